@@ -1,0 +1,65 @@
+"""Pins for the oracle's random-number generator (Philox4x32-10, SC'11) and its keying."""
+import os
+
+import numpy as np
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt")
+
+
+def _kat():
+    rows = []
+    for line in open(GOLDEN):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        w = [int(x, 16) for x in line.split()]
+        rows.append((w[0:4], w[4:6], w[6:10]))
+    return rows
+
+
+def test_known_answer_vectors(oracle):
+    rows = _kat()
+    assert len(rows) == 3
+    for ctr, key, out in rows:
+        got = oracle.philox4x32_10(ctr, key)
+        assert [int(x) for x in got] == out
+
+
+def test_keying_maps_to_counter_and_key(oracle):
+    """random_word(seed, step, worker, e) = word (e mod 4) of the block with
+    counter (lo(e/4), hi(e/4), worker, hi(seed)) and key (lo(seed), step)."""
+    seed = 0x0123456789ABCDEF
+    for e in (0, 1, 2, 3, 4, 7, 1 << 20, (1 << 34) + 5):
+        for worker in (0, 3):
+            for step in (0, 9):
+                q = e >> 2
+                blk = oracle.philox4x32_10([q & 0xFFFFFFFF, q >> 32, worker, seed >> 32],
+                                           [seed & 0xFFFFFFFF, step])
+                assert oracle.random_word(seed, step, worker, e) == int(blk[e & 3])
+
+
+def test_streams_differ_across_seed_step_worker(oracle):
+    base = [oracle.random_word(0, 0, 0, e) for e in range(64)]
+    for seed, step, worker in [(1, 0, 0), (0, 1, 0), (0, 0, 1), (1 << 32, 0, 0)]:
+        other = [oracle.random_word(seed, step, worker, e) for e in range(64)]
+        assert sum(a == b for a, b in zip(base, other)) == 0
+
+
+def test_uniform_grid_and_range(oracle):
+    assert oracle.uniform(0) == 0.0
+    assert oracle.uniform(0x1FF) == 0.0                    # low 9 bits are dropped
+    assert oracle.uniform(0x200) == 2.0 ** -23
+    assert oracle.uniform(0xFFFFFFFF) == 1.0 - 2.0 ** -23
+    assert oracle.uniform(0x80000000) == 0.5
+
+
+def test_uniform_moments(oracle):
+    n = 20000
+    u = np.array([oracle.uniform(oracle.random_word(7, 3, 1, e)) for e in range(n)])
+    assert abs(u.mean() - 0.5) < 5 * (1 / 12 ** 0.5) / n ** 0.5
+    assert abs(u.var() - 1 / 12) < 0.004
+    # bits look balanced
+    w = np.array([oracle.random_word(7, 3, 1, e) for e in range(4096)], dtype=np.uint64)
+    for bit in range(32):
+        frac = ((w >> np.uint64(bit)) & np.uint64(1)).mean()
+        assert abs(frac - 0.5) < 5 * 0.5 / 4096 ** 0.5
