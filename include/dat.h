@@ -1,0 +1,212 @@
+/*
+ * dat.h -- C ABI of the B200 (sm_100a) implementation of the data-parallel hot path of
+ * the outer-minimisation step of Distributed Adversarial Training (DAT):
+ *
+ *     M workers' per-layer fp32 gradients
+ *       -> randomized b-bit quantizer Q(.)              [Algorithm A1 Step 7; Eq. rand_q, Eq. xi]
+ *       -> aggregation  g_hat = (1/M) sum_i Q(g^(i))    [Algorithm A1 Step 9; Eq. grad_agg]
+ *       -> layer-wise adaptive learning-rate update      [Algorithm A1 Step 12, Eq. outer_min; Eq. 3]
+ *
+ * On one GPU the M workers are M gradient buffers in device memory.
+ *
+ * General conventions
+ *   - Every function returns an int: DAT_OK (0) or a negative DAT_ERR_* code.  Nothing throws,
+ *     aborts or prints.  Faults that the host can detect (null pointers, misalignment, bad
+ *     sizes) are returned BEFORE any kernel is launched.
+ *   - "device" pointers address memory of the CUDA device that was current when the plan was
+ *     created; that device must also be current in every later call with the plan.
+ *     "host" pointers address ordinary host memory.
+ *   - The caller owns every data buffer.  The library never allocates, frees or retains them;
+ *     after a call returns, only work already enqueued on `stream` refers to them.
+ *     A plan owns only its own small device workspace (layout tables, partial sums,
+ *     dependency counters, a status word) and, if dat_step_host is used, staging buffers.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All device work
+ *     is enqueued on it and is stream-ordered; calls return without synchronising unless
+ *     stated otherwise.
+ *   - Device data pointers must be 16-byte aligned (DAT_ERR_ALIGN otherwise).  Layer offsets
+ *     may be arbitrary (a layer need not start on a 16-byte boundary).
+ *   - A plan must not be used from two host threads at once, nor by two calls that overlap on
+ *     the device (its workspace is shared); distinct plans are independent.
+ *   - Conditions only the device can see (non-finite inputs, a bounded wait that ran out) set
+ *     bits in the plan's status word, read with dat_get_status; they never trap or hang.
+ *
+ * Notation: d = total number of parameters, h = number of layers (one per parameter tensor,
+ * given by the offset table), n_l = elements of layer l, M = workers, b = bits,
+ * S = 2^b - 1 (largest level), nu_l = the quantizer norm of layer l.
+ */
+#ifndef DAT_H_
+#define DAT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DAT_MAX_WORKERS 64
+
+typedef struct dat_plan dat_plan_t;
+
+/* Hyper-parameters of the update (Eq. 3): learning rate eta_t, momentum mu and weight decay of
+ * the descent direction u = mu*m + g_hat + wd*theta, and the clamp tau(x) = min{max{x,c_l},c_u}
+ * (the paper's experiments use c_l = 0, c_u = 10). */
+typedef struct dat_hparams {
+    float lr;
+    float momentum;
+    float weight_decay;
+    float c_l;
+    float c_u;
+} dat_hparams_t;
+
+/* Which l2 norm scales the quantizer of Eq. rand_q.
+ * SHARED_MAX: nu_l = max_i ||g_l^(i)||_2, one value per layer shared by all workers, so that
+ *             the workers' integer codes lie on one grid and Eq. grad_agg becomes an integer sum
+ *             followed by one scaling.  (Q stays unbiased for any nu >= max|g|.)              */
+enum { DAT_SCALE_SHARED_MAX = 0 };
+
+enum {
+    DAT_OK = 0,
+    DAT_ERR_ARG = -1,          /* null pointer, negative size, value out of range              */
+    DAT_ERR_ALIGN = -2,        /* a device data pointer is not 16-byte aligned                 */
+    DAT_ERR_BITS = -3,         /* bits not in {1,2,4,8,16,32}, or not valid for this call      */
+    DAT_ERR_LAYOUT = -4,       /* offsets[0] != 0 or offsets not strictly increasing           */
+    DAT_ERR_CUDA = -5,         /* a CUDA runtime call failed (see dat_last_cuda_error)         */
+    DAT_ERR_NOMEM = -6,        /* host or device allocation failed                              */
+    DAT_ERR_UNSUPPORTED = -7   /* valid request that this build does not implement             */
+};
+
+/* Bits of the device status word. */
+enum {
+    DAT_STATUS_NONFINITE = 1u, /* a quantizer norm or a layer norm was inf or NaN              */
+    DAT_STATUS_TIMEOUT = 2u,   /* a bounded device-side wait ran out; outputs of that call are
+                                  undefined, the plan stays usable                              */
+    DAT_STATUS_BOUNDS = 4u     /* reserved for self-checking builds                             */
+};
+
+/* ---------------------------------------------------------------------------------------------
+ * Plan: the layer partition theta = [theta_1^T ... theta_h^T]^T of Eq. 3 and the quantizer setup.
+ *   out            host pointer receiving the new plan.
+ *   num_layers     h >= 1.
+ *   layer_offsets  host array of h+1 element offsets; offsets[0] = 0, strictly increasing,
+ *                  offsets[h] = d.  Copied; the caller may free it after the call.
+ *   num_workers    M in [1, DAT_MAX_WORKERS].
+ *   bits           b in {1,2,4,8,16}, or 32 = no quantisation (Q is the identity and the
+ *                  aggregate is the plain worker average).
+ *   scale_mode     DAT_SCALE_SHARED_MAX.
+ * Allocates the plan's device workspace (synchronous).  Errors: ARG, BITS, LAYOUT, NOMEM, CUDA.
+ * ------------------------------------------------------------------------------------------- */
+int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64_t *layer_offsets,
+                    int num_workers, int bits, int scale_mode);
+
+/* Frees the plan and its workspace (synchronises the device).  NULL is accepted. */
+int dat_plan_destroy(dat_plan_t *plan);
+
+/* Sizes of the caller-owned buffers of the unfused calls (any output pointer may be NULL):
+ *   level_bytes_per_worker  bytes of one worker's level plane: ceil(d*b/8) rounded up to 16
+ *   sign_bytes_per_worker   bytes of one worker's sign plane:  ceil(d/8)   rounded up to 16
+ *   num_scales              number of fp32 norms in the message (h)
+ *   workspace_bytes         device bytes the plan itself holds
+ * Together: 32 bits per norm + d sign bits + b*d level bits per worker -- the
+ * "(32 + d + b d) bits" message of the paper's quantizer, with one norm per layer.            */
+int dat_plan_sizes(const dat_plan_t *plan, int64_t *level_bytes_per_worker,
+                   int64_t *sign_bytes_per_worker, int64_t *num_scales, int64_t *workspace_bytes);
+
+/* ---------------------------------------------------------------------------------------------
+ * dat_quantize -- Algorithm A1 Step 7: Q(g^(i)) for every worker (Eq. rand_q, Eq. xi).
+ *   For worker i, layer l, element e (global index in the flat vector), with x = S*|g_e|/nu_l:
+ *   level = floor(x) + 1 with probability x - floor(x), else floor(x); sign bit = (g_e < 0).
+ *   Randomness: Philox4x32-10, counter (lo(e/4), hi(e/4), i, hi(seed)), key (lo(seed), step),
+ *   word e mod 4; u = top 23 bits / 2^23; level = min(floor(fma(|g_e|, S/nu_l, u)), S).
+ *
+ *   grads      host array of M device pointers, each fp32[d], read-only.
+ *   seed,step  random-stream key; step must be < 2^32 (DAT_ERR_ARG).
+ *   levels     device, M * level_bytes_per_worker bytes, written.  Worker i's plane starts at
+ *              i*level_bytes_per_worker.  A plane is a little-endian bit stream over the global
+ *              element index: element e occupies bits [(e*b) mod 8, +b) of byte floor(e*b/8)
+ *              (b = 16: a little-endian uint16).  Padding bytes are written as zero.
+ *   signs      device, M * sign_bytes_per_worker bytes, written: bit (e mod 8) of byte
+ *              floor(e/8), 1 = negative.
+ *   scales     device fp32[h], written: nu_l.
+ *   scales_in  device fp32[h] or NULL.  If given, these norms are used instead of computing
+ *              ||g_l^(i)||_2 (and are copied to `scales`); may alias `scales`.
+ * Errors: ARG, ALIGN, BITS (b = 32 has no codes), CUDA.
+ * ------------------------------------------------------------------------------------------- */
+int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_t seed, uint64_t step,
+                 uint8_t *levels, uint8_t *signs, float *scales, const float *scales_in,
+                 void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * dat_aggregate -- Algorithm A1 Step 9, Eq. grad_agg, on the packed messages:
+ *   sum_e = sum_i (sign ? -level : level)  (exact, int32);  g_hat_e = sum_e * (nu_l / (S*M)).
+ *   levels, signs, scales   device, as written by dat_quantize, read-only.
+ *   code_sum                device int32[d] or NULL; written if given.
+ *   g_hat                   device fp32[d], written.
+ * Errors: ARG, ALIGN, BITS (b = 32), CUDA.
+ * ------------------------------------------------------------------------------------------- */
+int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint8_t *signs,
+                  const float *scales, int32_t *code_sum, float *g_hat, void *stream);
+
+/* dat_average -- Eq. grad_agg when Q is the identity (b = 32): g_hat_e = (sum_i g_e^(i)) / M,
+ * accumulated in fp32 in ascending worker order.  Valid for any plan.
+ *   grads  host array of M device pointers (fp32[d], read-only);  g_hat  device fp32[d], written. */
+int dat_average(dat_plan_t *plan, const float *const *grads, float *g_hat, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * dat_lalr_step -- Algorithm A1 Step 12 with the LALR rule of Eq. 3, for every layer l:
+ *   m'     = mu*m + (g_hat + wd*theta)                       (descent direction u = m')
+ *   theta' = theta - tau(||theta_l||_2) * lr / ||u_l||_2 * u,  tau(x) = min{max{x,c_l},c_u}
+ *   (||theta_l|| is the norm BEFORE the update; ||u_l|| = 0 gives a zero step.)
+ *   Two passes: pass 1 writes m' and reduces the two norms per layer, pass 2 updates theta.
+ *   theta, mom        device fp32[d], updated in place.
+ *   g_hat             device fp32[d], read-only.
+ *   hp                host pointer, read during the call.
+ *   layer_norms_out   device fp32[2h] or NULL: [2l] = ||theta_l||, [2l+1] = ||u_l||.
+ * Errors: ARG, ALIGN, CUDA.
+ * ------------------------------------------------------------------------------------------- */
+int dat_lalr_step(dat_plan_t *plan, float *theta, float *mom, const float *g_hat,
+                  const dat_hparams_t *hp, float *layer_norms_out, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * dat_step -- Steps 7, 9 and 12 of Algorithm A1 in one sweep: the result equals
+ * dat_quantize -> dat_aggregate -> dat_lalr_step (or dat_average -> dat_lalr_step when b = 32),
+ * but codes, code sums and g_hat are never written to device memory.
+ *   theta, mom        device fp32[d], updated in place.
+ *   grads             host array of M device pointers, fp32[d] each, read-only.
+ *   seed, step        as in dat_quantize.
+ *   hp                host pointer, read during the call.
+ *   code_sum_out      device int32[d] or NULL (checking aid; ignored when b = 32).
+ *   layer_norms_out   device fp32[2h] or NULL.
+ *   scales_out        device fp32[h] or NULL: nu_l (not written when b = 32).
+ * Errors: ARG, ALIGN, CUDA.
+ * ------------------------------------------------------------------------------------------- */
+int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+             uint64_t seed, uint64_t step, const dat_hparams_t *hp,
+             int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream);
+
+/* dat_step_host -- dat_step for callers whose data lives in HOST memory: copies theta, mom and
+ * the M gradient buffers to plan-owned device staging buffers, runs dat_step, copies theta and
+ * mom back, and synchronises `stream` before returning.
+ *   theta_host, mom_host   host fp32[d], updated in place (pinned memory makes the copies fast).
+ *   grads_host             host array of M host pointers, fp32[d] each.
+ * The first call allocates the staging buffers ((M+2)*d*4 bytes, kept until the plan is
+ * destroyed).  Errors: ARG, NOMEM, CUDA. */
+int dat_step_host(dat_plan_t *plan, float *theta_host, float *mom_host,
+                  const float *const *grads_host, uint64_t seed, uint64_t step,
+                  const dat_hparams_t *hp, void *stream);
+
+/* Synchronises `stream`, copies the plan's status word to *flags_out and clears it. */
+int dat_get_status(dat_plan_t *plan, uint32_t *flags_out, void *stream);
+
+/* Number of kernels the library has launched for this plan since it was created. */
+int64_t dat_plan_launch_count(const dat_plan_t *plan);
+
+/* Text for a DAT_ERR_* code (static storage). */
+const char *dat_strerror(int code);
+
+/* The cudaError_t value (as int) of the last failed CUDA call made for this plan, 0 if none. */
+int dat_last_cuda_error(const dat_plan_t *plan);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DAT_H_ */

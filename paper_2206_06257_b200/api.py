@@ -1,0 +1,172 @@
+"""ctypes binding of libdat.so: the same names and arguments as include/dat.h.
+
+Argument marshalling only -- every step of the path runs in the library's CUDA kernels.
+torch tensors are accepted wherever the C function takes a device (or host) pointer; the
+binding passes their data_ptr().  Importing this module loads the library and fails loudly
+if it has not been built (python -m paper_2206_06257_b200.build); there is no CPU fallback.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdat.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libdat.so is missing: build it with `python -m paper_2206_06257_b200.build` "
+        "(needs nvcc; the CUDA library is the only implementation of this path)")
+_lib = C.CDLL(LIB_PATH)
+
+DAT_MAX_WORKERS = 64
+DAT_SCALE_SHARED_MAX = 0
+DAT_OK, DAT_ERR_ARG, DAT_ERR_ALIGN, DAT_ERR_BITS = 0, -1, -2, -3
+DAT_ERR_LAYOUT, DAT_ERR_CUDA, DAT_ERR_NOMEM, DAT_ERR_UNSUPPORTED = -4, -5, -6, -7
+DAT_STATUS_NONFINITE, DAT_STATUS_TIMEOUT, DAT_STATUS_BOUNDS = 1, 2, 4
+
+# every symbol include/dat.h declares
+EXPORTS = ["dat_plan_create", "dat_plan_destroy", "dat_plan_sizes", "dat_quantize", "dat_aggregate",
+           "dat_average", "dat_lalr_step", "dat_step", "dat_step_host", "dat_get_status",
+           "dat_plan_launch_count", "dat_strerror", "dat_last_cuda_error"]
+
+
+class dat_hparams_t(C.Structure):
+    _fields_ = [("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
+                ("c_l", C.c_float), ("c_u", C.c_float)]
+
+
+_p, _i64, _u64, _int = C.c_void_p, C.c_int64, C.c_uint64, C.c_int
+_lib.dat_plan_create.argtypes = [C.POINTER(_p), _i64, _p, _int, _int, _int]
+_lib.dat_plan_destroy.argtypes = [_p]
+_lib.dat_plan_sizes.argtypes = [_p, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]
+_lib.dat_quantize.argtypes = [_p, _p, _u64, _u64, _p, _p, _p, _p, _p]
+_lib.dat_aggregate.argtypes = [_p, _p, _p, _p, _p, _p, _p]
+_lib.dat_average.argtypes = [_p, _p, _p, _p]
+_lib.dat_lalr_step.argtypes = [_p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
+_lib.dat_step.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
+_lib.dat_step_host.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p]
+_lib.dat_get_status.argtypes = [_p, C.POINTER(C.c_uint32), _p]
+_lib.dat_plan_launch_count.argtypes = [_p]
+_lib.dat_plan_launch_count.restype = _i64
+_lib.dat_strerror.argtypes = [_int]
+_lib.dat_strerror.restype = C.c_char_p
+_lib.dat_last_cuda_error.argtypes = [_p]
+for _n in EXPORTS:
+    if _n not in ("dat_plan_launch_count", "dat_strerror"):
+        getattr(_lib, _n).restype = _int
+
+
+class DatError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__("%s: %s (%d)" % (where, dat_strerror(code), code))
+
+
+def _ok(code, where):
+    if code != DAT_OK:
+        raise DatError(code, where)
+
+
+def _ptr(x):
+    """Address of a tensor / array / int / None, as c_void_p."""
+    if x is None:
+        return None
+    if isinstance(x, torch.Tensor):
+        return _p(x.data_ptr())
+    if isinstance(x, np.ndarray):
+        return _p(x.ctypes.data)
+    return _p(int(x))
+
+
+def _ptr_array(xs):
+    arr = (C.c_void_p * len(xs))()
+    for k, x in enumerate(xs):
+        arr[k] = _ptr(x).value if x is not None else None
+    return arr
+
+
+def _stream(stream):
+    if stream is None:
+        return _p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, torch.cuda.Stream):
+        return _p(stream.cuda_stream)
+    return _p(int(stream))
+
+
+def _hp(hp):
+    if isinstance(hp, dat_hparams_t):
+        return hp
+    return dat_hparams_t(*[float(v) for v in hp])
+
+
+def dat_strerror(code):
+    return _lib.dat_strerror(int(code)).decode()
+
+
+def dat_plan_create(layer_offsets, num_workers, bits, scale_mode=DAT_SCALE_SHARED_MAX):
+    """Returns the plan handle (an int).  layer_offsets: h+1 int64 values (any sequence)."""
+    offs = np.ascontiguousarray(layer_offsets, dtype=np.int64)
+    out = _p()
+    _ok(_lib.dat_plan_create(C.byref(out), offs.size - 1, _ptr(offs), int(num_workers), int(bits),
+                             int(scale_mode)), "dat_plan_create")
+    return out.value
+
+
+def dat_plan_destroy(plan):
+    _ok(_lib.dat_plan_destroy(_p(plan)), "dat_plan_destroy")
+
+
+def dat_plan_sizes(plan):
+    """(level_bytes_per_worker, sign_bytes_per_worker, num_scales, workspace_bytes)"""
+    a, b, c, d = _i64(), _i64(), _i64(), _i64()
+    _ok(_lib.dat_plan_sizes(_p(plan), C.byref(a), C.byref(b), C.byref(c), C.byref(d)), "dat_plan_sizes")
+    return a.value, b.value, c.value, d.value
+
+
+def dat_quantize(plan, grads, seed, step, levels, signs, scales, scales_in=None, stream=None):
+    _ok(_lib.dat_quantize(_p(plan), _ptr_array(grads), int(seed), int(step), _ptr(levels), _ptr(signs),
+                          _ptr(scales), _ptr(scales_in), _stream(stream)), "dat_quantize")
+
+
+def dat_aggregate(plan, levels, signs, scales, code_sum, g_hat, stream=None):
+    _ok(_lib.dat_aggregate(_p(plan), _ptr(levels), _ptr(signs), _ptr(scales), _ptr(code_sum), _ptr(g_hat),
+                           _stream(stream)), "dat_aggregate")
+
+
+def dat_average(plan, grads, g_hat, stream=None):
+    _ok(_lib.dat_average(_p(plan), _ptr_array(grads), _ptr(g_hat), _stream(stream)), "dat_average")
+
+
+def dat_lalr_step(plan, theta, mom, g_hat, hp, layer_norms_out=None, stream=None):
+    h = _hp(hp)
+    _ok(_lib.dat_lalr_step(_p(plan), _ptr(theta), _ptr(mom), _ptr(g_hat), C.byref(h), _ptr(layer_norms_out),
+                           _stream(stream)), "dat_lalr_step")
+
+
+def dat_step(plan, theta, mom, grads, seed, step, hp, code_sum_out=None, layer_norms_out=None,
+             scales_out=None, stream=None):
+    h = _hp(hp)
+    _ok(_lib.dat_step(_p(plan), _ptr(theta), _ptr(mom), _ptr_array(grads), int(seed), int(step), C.byref(h),
+                      _ptr(code_sum_out), _ptr(layer_norms_out), _ptr(scales_out), _stream(stream)), "dat_step")
+
+
+def dat_step_host(plan, theta_host, mom_host, grads_host, seed, step, hp, stream=None):
+    h = _hp(hp)
+    _ok(_lib.dat_step_host(_p(plan), _ptr(theta_host), _ptr(mom_host), _ptr_array(grads_host), int(seed),
+                           int(step), C.byref(h), _stream(stream)), "dat_step_host")
+
+
+def dat_get_status(plan, stream=None):
+    v = C.c_uint32()
+    _ok(_lib.dat_get_status(_p(plan), C.byref(v), _stream(stream)), "dat_get_status")
+    return v.value
+
+
+def dat_plan_launch_count(plan):
+    return int(_lib.dat_plan_launch_count(_p(plan)))
+
+
+def dat_last_cuda_error(plan):
+    return int(_lib.dat_last_cuda_error(_p(plan)))

@@ -1,0 +1,206 @@
+// Internal declarations shared by the translation units of libdat.so (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "dat.h"
+
+// Elements per tile of the per-layer tiling (tiles never cross a layer boundary; they start
+// on 4-element boundaries of the flat vector so that float4 accesses stay 16-byte aligned).
+#define DAT_TILE 4096
+#define DAT_THREADS 256
+
+struct GradPtrs {
+    const float *p[DAT_MAX_WORKERS];
+};
+
+// The ten round keys of Philox4x32-10 for one (seed, step): the same for every thread.
+struct PhiloxKeys {
+    uint32_t k0[10];
+    uint32_t k1[10];
+    uint32_t seed_hi;   // fourth counter word
+};
+
+struct FusedSchedule;   // dat_step.cu
+
+struct dat_plan {
+    int device = 0;
+    int64_t h = 0, d = 0;
+    int M = 0, bits = 0, scale_mode = 0;
+    uint32_t S = 0;
+    std::vector<int64_t> offsets;      // host copy, h+1
+    std::vector<int64_t> tile_base;    // host copy, h+1: first per-layer tile of each layer
+    int64_t n_tiles = 0;               // per-layer tiles in total
+    int64_t level_bytes = 0, sign_bytes = 0;
+
+    // device workspace (one allocation, carved up)
+    char *ws = nullptr;
+    size_t ws_bytes = 0;
+    int64_t *d_offsets = nullptr;      // h+1
+    int64_t *d_tile_base = nullptr;    // h+1
+    double *d_partials = nullptr;      // n_tiles * max(M,2)
+    float *d_worker_norms = nullptr;   // M*h
+    float *d_scales = nullptr;         // h     nu_l (fused path / scratch)
+    float *d_qmul = nullptr;           // h     S/nu_l (0 if nu_l = 0)
+    float *d_dq = nullptr;             // h     nu_l/(S*M)
+    float *d_step_a = nullptr;         // h     lr * tau/||u||
+    float *d_norms = nullptr;          // 2h
+    uint32_t *d_status = nullptr;      // 1
+
+    FusedSchedule *fused = nullptr;    // built lazily by dat_step
+
+    // staging buffers of dat_step_host
+    float *stage = nullptr;
+
+    int sm_count = 0;
+    int64_t launches = 0;
+    int last_cuda = 0;
+};
+
+// ---- host helpers (dat_plan.cu) -------------------------------------------------------------
+int dat_check_plan(dat_plan_t *plan);                       // device current, non-null
+int dat_cuda_fail(dat_plan_t *plan, cudaError_t e);          // records e, returns DAT_ERR_CUDA
+bool dat_aligned16(const void *p);
+int dat_check_grads(const dat_plan_t *plan, const float *const *grads, GradPtrs *out);
+PhiloxKeys dat_make_keys(uint64_t seed, uint64_t step);
+void dat_fused_destroy(dat_plan_t *plan);                    // dat_step.cu
+
+#define DAT_CUDA(plan, call)                                              \
+    do {                                                                  \
+        cudaError_t e__ = (call);                                         \
+        if (e__ != cudaSuccess) return dat_cuda_fail((plan), e__);        \
+    } while (0)
+
+#define DAT_LAUNCHED(plan)                                                \
+    do {                                                                  \
+        cudaError_t e__ = cudaGetLastError();                             \
+        if (e__ != cudaSuccess) return dat_cuda_fail((plan), e__);        \
+        (plan)->launches++;                                               \
+    } while (0)
+
+// ---- device helpers ---------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+// One Philox4x32-10 block (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and
+// two three-way XORs; round keys precomputed on the host.
+__device__ __forceinline__ void dat_philox(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                           const PhiloxKeys &k, uint32_t out[4])
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k.k0[r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k.k1[r];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// The random words of the four elements 4q .. 4q+3 of `worker`.
+__device__ __forceinline__ void dat_random_words(uint64_t q, uint32_t worker, const PhiloxKeys &k,
+                                                 uint32_t out[4])
+{
+    dat_philox((uint32_t)q, (uint32_t)(q >> 32), worker, k.seed_hi, k, out);
+}
+
+// Stochastic level of one element: floor(|g| * qmul + u) clamped to S, u = top 23 bits of w.
+// y lies in [0, 65535], so adding 2^23 rounding down leaves floor(y) in the low mantissa bits.
+__device__ __forceinline__ uint32_t dat_level(float g, float qmul, float S_f, uint32_t w)
+{
+    const float u = __uint_as_float(0x3F800000u | (w >> 9)) - 1.0f;
+    const float y = fminf(__fmaf_rn(fabsf(g), qmul, u), S_f);
+    return __float_as_uint(__fadd_rd(y, 8388608.0f)) & 0x007FFFFFu;
+}
+
+// Largest l in [0, h) with table[l] <= x (table[0] <= x < table[h] assumed).
+__device__ __forceinline__ int dat_find(const int64_t *__restrict__ table, int h, int64_t x)
+{
+    int lo = 0, hi = h;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(table + mid) <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ double dat_warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Sum over a block of DAT_THREADS threads in a fixed order; result valid in thread 0.
+// `scratch` holds at least DAT_THREADS/32 doubles; safe to call repeatedly.
+__device__ __forceinline__ double dat_block_sum(double v, double *scratch)
+{
+    v = dat_warp_sum(v);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    double r = 0.0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < DAT_THREADS / 32; ++w) r += scratch[w];
+    }
+    return r;
+}
+
+// ------------------------------------------------------------------------------------------
+// Per-layer tiling shared by the norm kernels: tile t belongs to layer l = find(tile_base, t);
+// it covers the flat elements [a + k*DAT_TILE, a + (k+1)*DAT_TILE) ∩ [lo, hi) where
+// lo/hi are the layer's bounds, a = lo rounded down to a multiple of 4 and k = t - tile_base[l].
+// ------------------------------------------------------------------------------------------
+struct TileRange {
+    int layer;
+    int64_t lo, hi;        // layer bounds
+    int64_t begin, end;    // begin is a multiple of 4; elements outside [lo, hi) are masked
+};
+
+__device__ __forceinline__ TileRange dat_tile_range(const int64_t *__restrict__ off,
+                                                    const int64_t *__restrict__ tile_base, int h,
+                                                    int64_t tile)
+{
+    TileRange r;
+    r.layer = dat_find(tile_base, h, tile);
+    r.lo = __ldg(off + r.layer);
+    r.hi = __ldg(off + r.layer + 1);
+    r.begin = (r.lo & ~(int64_t)3) + (tile - __ldg(tile_base + r.layer)) * DAT_TILE;
+    r.end = min(r.begin + (int64_t)DAT_TILE, r.hi);
+    return r;
+}
+
+// Loads the four elements e0..e0+3 (e0 a multiple of 4) that lie in [lo, hi); others read 0.
+__device__ __forceinline__ void dat_load4(const float *__restrict__ p, int64_t e0, int64_t lo,
+                                          int64_t hi, float v[4])
+{
+    if (e0 >= lo && e0 + 4 <= hi) {
+        const float4 f = *reinterpret_cast<const float4 *>(p + e0);
+        v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = (e0 + j >= lo && e0 + j < hi) ? p[e0 + j] : 0.0f;
+    }
+}
+
+__device__ __forceinline__ void dat_store4(float *__restrict__ p, int64_t e0, int64_t lo,
+                                           int64_t hi, const float v[4])
+{
+    if (e0 >= lo && e0 + 4 <= hi) {
+        *reinterpret_cast<float4 *>(p + e0) = make_float4(v[0], v[1], v[2], v[3]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (e0 + j >= lo && e0 + j < hi) p[e0 + j] = v[j];
+    }
+}
+
+#endif  // __CUDACC__

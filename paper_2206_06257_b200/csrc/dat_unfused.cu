@@ -1,0 +1,467 @@
+// The three steps as separate calls: dat_quantize (Algorithm A1 Step 7), dat_aggregate /
+// dat_average (Step 9, Eq. grad_agg) and dat_lalr_step (Step 12, Eq. 3).  Codes, scales and
+// g_hat are materialised in device memory between the calls.
+#include "dat_internal.cuh"
+
+// ------------------------------------------------------------------------------------------
+// S1: quantizer norms.  Pass A: one fp64 partial sum of squares per (tile, worker).
+// Pass B: per layer, fixed-order sum of the partials, nu_l = max_i sqrt(.), S/nu_l.
+// Squares of fp32 values are exact in fp64, so the result does not depend on the tiling
+// beyond the last bits of an fp64 sum.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DAT_THREADS)
+k_sumsq_partial(GradPtrs gp, const int64_t *__restrict__ off, const int64_t *__restrict__ tile_base,
+                int h, int M, double *__restrict__ partials)
+{
+    __shared__ double scratch[DAT_THREADS / 32];
+    const int64_t tile = blockIdx.x;
+    const int worker = blockIdx.y;
+    const TileRange r = dat_tile_range(off, tile_base, h, tile);
+    const float *__restrict__ g = gp.p[worker];
+    double acc = 0.0;
+#pragma unroll
+    for (int it = 0; it < DAT_TILE / 4 / DAT_THREADS; ++it) {
+        const int64_t e0 = r.begin + 4 * (int64_t)(it * DAT_THREADS + threadIdx.x);
+        if (e0 < r.end) {
+            float v[4];
+            dat_load4(g, e0, r.lo, r.hi, v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc = fma((double)v[j], (double)v[j], acc);
+        }
+    }
+    const double s = dat_block_sum(acc, scratch);
+    if (threadIdx.x == 0) partials[tile * M + worker] = s;
+}
+
+__global__ void __launch_bounds__(DAT_THREADS)
+k_scales_finalize(const int64_t *__restrict__ tile_base, int h, int M, float S_f,
+                  const double *__restrict__ partials, float *__restrict__ worker_norms,
+                  float *__restrict__ scales, float *__restrict__ qmul, uint32_t *status)
+{
+    __shared__ float s_norm[DAT_MAX_WORKERS];
+    const int l = blockIdx.x;
+    const int64_t t0 = tile_base[l], t1 = tile_base[l + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = warp; i < M; i += DAT_THREADS / 32) {
+        double acc = 0.0;
+        for (int64_t t = t0 + lane; t < t1; t += 32) acc += partials[t * M + i];
+        acc = dat_warp_sum(acc);
+        if (lane == 0) {
+            const float nrm = (float)sqrt(acc);
+            s_norm[i] = nrm;
+            worker_norms[(int64_t)i * h + l] = nrm;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float nu = s_norm[0];
+        bool bad = !isfinite(nu);
+        for (int i = 1; i < M; ++i) {
+            bad |= !isfinite(s_norm[i]);
+            nu = (s_norm[i] > nu) ? s_norm[i] : nu;
+        }
+        scales[l] = nu;
+        qmul[l] = (nu == 0.0f) ? 0.0f : S_f / nu;
+        if (bad) atomicOr(status, DAT_STATUS_NONFINITE);
+    }
+}
+
+// qmul from caller-supplied norms.
+__global__ void k_qmul_from_scales(int h, float S_f, const float *__restrict__ scales,
+                                   float *__restrict__ qmul, uint32_t *status)
+{
+    const int l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l >= h) return;
+    const float nu = scales[l];
+    qmul[l] = (nu == 0.0f) ? 0.0f : S_f / nu;
+    if (!isfinite(nu)) atomicOr(status, DAT_STATUS_NONFINITE);
+}
+
+// ------------------------------------------------------------------------------------------
+// S2 + S3: stochastic levels and the packed planes.  Tiles are DAT_TILE consecutive elements of
+// the FLAT vector (they may span layers); thread t of iteration k owns the aligned group of four
+// elements 4*(k*256+t).., which is exactly one Philox block.  The packed bits of a tile are
+// assembled in shared memory and written out with 128-bit stores.
+// ------------------------------------------------------------------------------------------
+template <int BITS>
+__global__ void __launch_bounds__(DAT_THREADS)
+k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h, int64_t d,
+           const float *__restrict__ qmul, uint8_t *__restrict__ levels, uint8_t *__restrict__ signs,
+           int64_t level_bytes, int64_t sign_bytes)
+{
+    constexpr int GROUPS = DAT_TILE / 4;                     // aligned groups per tile
+    constexpr int LEVEL_TILE_BYTES = DAT_TILE * BITS / 8;
+    constexpr int SIGN_TILE_BYTES = DAT_TILE / 8;
+    __shared__ uint4 s_level[LEVEL_TILE_BYTES / 16];
+    __shared__ uint4 s_sign[SIGN_TILE_BYTES / 16];
+    __shared__ int s_first;
+
+    const int64_t tile = blockIdx.x;
+    const int worker = blockIdx.y;
+    const int64_t e_tile = tile * DAT_TILE;
+    const float *__restrict__ g = gp.p[worker];
+    const float S_f = (float)((1u << BITS) - 1u);
+
+    if (threadIdx.x == 0) s_first = dat_find(off, h, e_tile);
+    __syncthreads();
+    int l = s_first;
+    int64_t l_hi = __ldg(off + l + 1);
+    float t = __ldg(qmul + l);
+
+#pragma unroll
+    for (int it = 0; it < GROUPS / DAT_THREADS; ++it) {
+        const int v = it * DAT_THREADS + threadIdx.x;
+        const int64_t e0 = e_tile + 4 * (int64_t)v;
+        float gv[4];
+        dat_load4(g, e0, 0, d, gv);
+        uint32_t w[4];
+        dat_random_words((uint64_t)e0 >> 2, (uint32_t)worker, keys, w);
+        uint32_t lev[4], neg = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t e = e0 + j;
+            while (e >= l_hi && l + 1 < h) {     // advance to the element's layer
+                ++l;
+                l_hi = __ldg(off + l + 1);
+                t = __ldg(qmul + l);
+            }
+            lev[j] = (e < d) ? dat_level(gv[j], t, S_f, w[j]) : 0u;
+            neg |= (uint32_t)(gv[j] < 0.0f) << j;
+        }
+        // pack the group's level bits
+        if (BITS == 16) {
+            reinterpret_cast<uint2 *>(s_level)[v] = make_uint2(lev[0] | (lev[1] << 16), lev[2] | (lev[3] << 16));
+        } else if (BITS == 8) {
+            reinterpret_cast<uint32_t *>(s_level)[v] = lev[0] | (lev[1] << 8) | (lev[2] << 16) | (lev[3] << 24);
+        } else if (BITS == 4) {
+            reinterpret_cast<uint16_t *>(s_level)[v] = (uint16_t)(lev[0] | (lev[1] << 4) | (lev[2] << 8) | (lev[3] << 12));
+        } else if (BITS == 2) {
+            reinterpret_cast<uint8_t *>(s_level)[v] = (uint8_t)(lev[0] | (lev[1] << 2) | (lev[2] << 4) | (lev[3] << 6));
+        } else {   // BITS == 1: two neighbouring groups share a byte
+            const uint32_t nib = lev[0] | (lev[1] << 1) | (lev[2] << 2) | (lev[3] << 3);
+            const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, nib, 1);
+            if ((threadIdx.x & 1) == 0) reinterpret_cast<uint8_t *>(s_level)[v >> 1] = (uint8_t)(nib | (other << 4));
+        }
+        const uint32_t other_neg = __shfl_xor_sync(0xFFFFFFFFu, neg, 1);
+        if ((threadIdx.x & 1) == 0) reinterpret_cast<uint8_t *>(s_sign)[v >> 1] = (uint8_t)(neg | (other_neg << 4));
+    }
+    __syncthreads();
+
+    // 128-bit stores of the finished tile (planes are padded to 16 bytes, so whole uint4 fit)
+    {
+        const int64_t base = tile * LEVEL_TILE_BYTES;
+        const int64_t left = level_bytes - base;
+        const int n16 = (int)((left < LEVEL_TILE_BYTES ? left : LEVEL_TILE_BYTES) / 16);
+        uint4 *dst = reinterpret_cast<uint4 *>(levels + (int64_t)worker * level_bytes + base);
+        for (int k = threadIdx.x; k < n16; k += DAT_THREADS) dst[k] = s_level[k];
+    }
+    {
+        const int64_t base = tile * SIGN_TILE_BYTES;
+        const int64_t left = sign_bytes - base;
+        const int n16 = (int)((left < SIGN_TILE_BYTES ? left : SIGN_TILE_BYTES) / 16);
+        uint4 *dst = reinterpret_cast<uint4 *>(signs + (int64_t)worker * sign_bytes + base);
+        for (int k = threadIdx.x; k < n16; k += DAT_THREADS) dst[k] = s_sign[k];
+    }
+}
+
+extern "C" int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_t seed, uint64_t step,
+                            uint8_t *levels, uint8_t *signs, float *scales, const float *scales_in,
+                            void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (plan->bits == 32) return DAT_ERR_BITS;
+    if (!levels || !signs || !scales) return DAT_ERR_ARG;
+    if (step >> 32) return DAT_ERR_ARG;
+    if (!dat_aligned16(levels) || !dat_aligned16(signs) || !dat_aligned16(scales)) return DAT_ERR_ALIGN;
+    if (scales_in && !dat_aligned16(scales_in)) return DAT_ERR_ALIGN;
+    GradPtrs gp;
+    rc = dat_check_grads(plan, grads, &gp);
+    if (rc != DAT_OK) return rc;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    const int h = (int)plan->h;
+    const float S_f = (float)plan->S;
+    if (scales_in) {
+        if (scales_in != scales)
+            DAT_CUDA(plan, cudaMemcpyAsync(scales, scales_in, (size_t)h * 4, cudaMemcpyDeviceToDevice, s));
+        k_qmul_from_scales<<<(h + 255) / 256, 256, 0, s>>>(h, S_f, scales, plan->d_qmul, plan->d_status);
+        DAT_LAUNCHED(plan);
+    } else {
+        dim3 grid((unsigned)plan->n_tiles, (unsigned)plan->M);
+        k_sumsq_partial<<<grid, DAT_THREADS, 0, s>>>(gp, plan->d_offsets, plan->d_tile_base, h, plan->M,
+                                                     plan->d_partials);
+        DAT_LAUNCHED(plan);
+        k_scales_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base, h, plan->M, S_f, plan->d_partials,
+                                                    plan->d_worker_norms, scales, plan->d_qmul, plan->d_status);
+        DAT_LAUNCHED(plan);
+    }
+    const PhiloxKeys keys = dat_make_keys(seed, step);
+    const int64_t flat_tiles = (plan->d + DAT_TILE - 1) / DAT_TILE;
+    dim3 grid((unsigned)flat_tiles, (unsigned)plan->M);
+#define DAT_Q(B)                                                                                           \
+    k_quantize<B><<<grid, DAT_THREADS, 0, s>>>(gp, keys, plan->d_offsets, h, plan->d, plan->d_qmul, levels, \
+                                               signs, plan->level_bytes, plan->sign_bytes)
+    switch (plan->bits) {
+    case 1: DAT_Q(1); break;
+    case 2: DAT_Q(2); break;
+    case 4: DAT_Q(4); break;
+    case 8: DAT_Q(8); break;
+    default: DAT_Q(16); break;
+    }
+#undef DAT_Q
+    DAT_LAUNCHED(plan);
+    return DAT_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// S4 + S5: unpack, integer sum over workers, one scaling.  Each thread owns 8 consecutive
+// elements (b bytes of levels and one sign byte per worker).
+// ------------------------------------------------------------------------------------------
+__global__ void k_dq_from_scales(int h, float SM_f, const float *__restrict__ scales, float *__restrict__ dq)
+{
+    const int l = blockIdx.x * blockDim.x + threadIdx.x;
+    if (l >= h) return;
+    const float nu = scales[l];
+    dq[l] = (nu == 0.0f) ? 0.0f : nu / SM_f;
+}
+
+template <int BITS>
+__device__ __forceinline__ void dat_unpack8(const uint8_t *__restrict__ plane, int64_t e0, uint32_t lev[8])
+{
+    const uint8_t *p = plane + e0 * BITS / 8;
+    if (BITS == 16) {
+        const uint4 q = *reinterpret_cast<const uint4 *>(p);
+        lev[0] = q.x & 0xFFFF; lev[1] = q.x >> 16; lev[2] = q.y & 0xFFFF; lev[3] = q.y >> 16;
+        lev[4] = q.z & 0xFFFF; lev[5] = q.z >> 16; lev[6] = q.w & 0xFFFF; lev[7] = q.w >> 16;
+    } else if (BITS == 8) {
+        const uint2 q = *reinterpret_cast<const uint2 *>(p);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { lev[j] = (q.x >> (8 * j)) & 0xFF; lev[4 + j] = (q.y >> (8 * j)) & 0xFF; }
+    } else {
+        uint32_t q;
+        if (BITS == 4) q = *reinterpret_cast<const uint32_t *>(p);
+        else if (BITS == 2) q = *reinterpret_cast<const uint16_t *>(p);
+        else q = *p;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) lev[j] = (q >> (BITS * j)) & ((1u << BITS) - 1u);
+    }
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(DAT_THREADS)
+k_aggregate(const uint8_t *__restrict__ levels, const uint8_t *__restrict__ signs, int64_t level_bytes,
+            int64_t sign_bytes, int M, const int64_t *__restrict__ off, int h, int64_t d,
+            const float *__restrict__ dq, int32_t *__restrict__ code_sum, float *__restrict__ g_hat)
+{
+    __shared__ int s_first;
+    const int64_t e_blk = (int64_t)blockIdx.x * (DAT_THREADS * 8);
+    if (threadIdx.x == 0) s_first = dat_find(off, h, e_blk);
+    __syncthreads();
+    const int64_t e0 = e_blk + 8 * (int64_t)threadIdx.x;
+    if (e0 >= d) return;
+    int sum[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sum[j] = 0;
+    for (int i = 0; i < M; ++i) {
+        uint32_t lev[8];
+        dat_unpack8<BITS>(levels + (int64_t)i * level_bytes, e0, lev);
+        const uint32_t sg = signs[(int64_t)i * sign_bytes + (e0 >> 3)];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) sum[j] += ((sg >> j) & 1u) ? -(int)lev[j] : (int)lev[j];
+    }
+    int l = s_first;
+    int64_t l_hi = __ldg(off + l + 1);
+    float f = __ldg(dq + l);
+    float out[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int64_t e = e0 + j;
+        while (e >= l_hi && l + 1 < h) {
+            ++l;
+            l_hi = __ldg(off + l + 1);
+            f = __ldg(dq + l);
+        }
+        out[j] = (float)sum[j] * f;
+    }
+    if (e0 + 8 <= d) {
+        reinterpret_cast<float4 *>(g_hat + e0)[0] = make_float4(out[0], out[1], out[2], out[3]);
+        reinterpret_cast<float4 *>(g_hat + e0)[1] = make_float4(out[4], out[5], out[6], out[7]);
+        if (code_sum) {
+            reinterpret_cast<int4 *>(code_sum + e0)[0] = make_int4(sum[0], sum[1], sum[2], sum[3]);
+            reinterpret_cast<int4 *>(code_sum + e0)[1] = make_int4(sum[4], sum[5], sum[6], sum[7]);
+        }
+    } else {
+        for (int j = 0; j < 8 && e0 + j < d; ++j) {
+            g_hat[e0 + j] = out[j];
+            if (code_sum) code_sum[e0 + j] = sum[j];
+        }
+    }
+}
+
+extern "C" int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint8_t *signs,
+                             const float *scales, int32_t *code_sum, float *g_hat, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (plan->bits == 32) return DAT_ERR_BITS;
+    if (!levels || !signs || !scales || !g_hat) return DAT_ERR_ARG;
+    if (!dat_aligned16(levels) || !dat_aligned16(signs) || !dat_aligned16(scales) || !dat_aligned16(g_hat) ||
+        (code_sum && !dat_aligned16(code_sum)))
+        return DAT_ERR_ALIGN;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int h = (int)plan->h;
+    const float SM_f = (float)((uint64_t)plan->S * (uint64_t)plan->M);
+    k_dq_from_scales<<<(h + 255) / 256, 256, 0, s>>>(h, SM_f, scales, plan->d_dq);
+    DAT_LAUNCHED(plan);
+    const unsigned grid = (unsigned)((plan->d + DAT_THREADS * 8 - 1) / (DAT_THREADS * 8));
+#define DAT_A(B)                                                                                         \
+    k_aggregate<B><<<grid, DAT_THREADS, 0, s>>>(levels, signs, plan->level_bytes, plan->sign_bytes, plan->M, \
+                                                plan->d_offsets, h, plan->d, plan->d_dq, code_sum, g_hat)
+    switch (plan->bits) {
+    case 1: DAT_A(1); break;
+    case 2: DAT_A(2); break;
+    case 4: DAT_A(4); break;
+    case 8: DAT_A(8); break;
+    default: DAT_A(16); break;
+    }
+#undef DAT_A
+    DAT_LAUNCHED(plan);
+    return DAT_OK;
+}
+
+// Eq. grad_agg with Q = identity: ordered fp32 sum over workers, then one division by M.
+__global__ void __launch_bounds__(DAT_THREADS)
+k_average(GradPtrs gp, int M, int64_t d, float *__restrict__ g_hat)
+{
+    const int64_t e0 = 4 * ((int64_t)blockIdx.x * DAT_THREADS + threadIdx.x);
+    if (e0 >= d) return;
+    float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    for (int i = 0; i < M; ++i) {
+        float v[4];
+        dat_load4(gp.p[i], e0, 0, d, v);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[j] += v[j];
+    }
+    const float Mf = (float)M;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[j] = acc[j] / Mf;
+    dat_store4(g_hat, e0, 0, d, acc);
+}
+
+extern "C" int dat_average(dat_plan_t *plan, const float *const *grads, float *g_hat, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (!g_hat) return DAT_ERR_ARG;
+    if (!dat_aligned16(g_hat)) return DAT_ERR_ALIGN;
+    GradPtrs gp;
+    rc = dat_check_grads(plan, grads, &gp);
+    if (rc != DAT_OK) return rc;
+    const unsigned grid = (unsigned)((plan->d + DAT_THREADS * 4 - 1) / (DAT_THREADS * 4));
+    k_average<<<grid, DAT_THREADS, 0, (cudaStream_t)stream>>>(gp, plan->M, plan->d, g_hat);
+    DAT_LAUNCHED(plan);
+    return DAT_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// S6-S8: LALR (Eq. 3).  Pass 1 (per-layer tiles): m' and the fp64 partial sums of theta^2 and
+// m'^2.  Finalize: per layer, a_l = lr * tau(||theta_l||)/||u_l||.  Pass 2: theta -= a_l * m'.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(DAT_THREADS)
+k_lalr_pass1(const float *__restrict__ theta, float *__restrict__ mom, const float *__restrict__ g_hat,
+             const int64_t *__restrict__ off, const int64_t *__restrict__ tile_base, int h, float mu, float wd,
+             double *__restrict__ partials)
+{
+    __shared__ double scratch[DAT_THREADS / 32];
+    const int64_t tile = blockIdx.x;
+    const TileRange r = dat_tile_range(off, tile_base, h, tile);
+    double ss_theta = 0.0, ss_u = 0.0;
+#pragma unroll
+    for (int it = 0; it < DAT_TILE / 4 / DAT_THREADS; ++it) {
+        const int64_t e0 = r.begin + 4 * (int64_t)(it * DAT_THREADS + threadIdx.x);
+        if (e0 < r.end) {
+            float th[4], m[4], g[4];
+            dat_load4(theta, e0, r.lo, r.hi, th);
+            dat_load4(mom, e0, r.lo, r.hi, m);
+            dat_load4(g_hat, e0, r.lo, r.hi, g);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                m[j] = __fmaf_rn(mu, m[j], __fmaf_rn(wd, th[j], g[j]));
+                ss_theta = fma((double)th[j], (double)th[j], ss_theta);
+                ss_u = fma((double)m[j], (double)m[j], ss_u);
+            }
+            dat_store4(mom, e0, r.lo, r.hi, m);
+        }
+    }
+    const double a = dat_block_sum(ss_theta, scratch);
+    const double b = dat_block_sum(ss_u, scratch);
+    if (threadIdx.x == 0) { partials[2 * tile] = a; partials[2 * tile + 1] = b; }
+}
+
+__global__ void __launch_bounds__(DAT_THREADS)
+k_lalr_finalize(const int64_t *__restrict__ tile_base, const double *__restrict__ partials,
+                float lr, float c_l, float c_u, float *__restrict__ step_a,
+                float *__restrict__ norms_out, uint32_t *status)
+{
+    __shared__ double scratch[DAT_THREADS / 32];
+    const int l = blockIdx.x;
+    const int64_t t0 = tile_base[l], t1 = tile_base[l + 1];
+    double a = 0.0, b = 0.0;
+    for (int64_t t = t0 + threadIdx.x; t < t1; t += DAT_THREADS) { a += partials[2 * t]; b += partials[2 * t + 1]; }
+    a = dat_block_sum(a, scratch);
+    b = dat_block_sum(b, scratch);
+    if (threadIdx.x == 0) {
+        const float n_theta = (float)sqrt(a), n_u = (float)sqrt(b);
+        const float tau = fminf(fmaxf(n_theta, c_l), c_u);
+        const float ratio = (n_u == 0.0f) ? 0.0f : tau / n_u;
+        step_a[l] = lr * ratio;
+        if (norms_out) { norms_out[2 * l] = n_theta; norms_out[2 * l + 1] = n_u; }
+        if (!isfinite(n_theta) || !isfinite(n_u)) atomicOr(status, DAT_STATUS_NONFINITE);
+    }
+}
+
+__global__ void __launch_bounds__(DAT_THREADS)
+k_lalr_pass2(float *__restrict__ theta, const float *__restrict__ mom, const int64_t *__restrict__ off,
+             const int64_t *__restrict__ tile_base, int h, const float *__restrict__ step_a)
+{
+    const int64_t tile = blockIdx.x;
+    const TileRange r = dat_tile_range(off, tile_base, h, tile);
+    const float na = -__ldg(step_a + r.layer);
+#pragma unroll
+    for (int it = 0; it < DAT_TILE / 4 / DAT_THREADS; ++it) {
+        const int64_t e0 = r.begin + 4 * (int64_t)(it * DAT_THREADS + threadIdx.x);
+        if (e0 < r.end) {
+            float th[4], m[4];
+            dat_load4(theta, e0, r.lo, r.hi, th);
+            dat_load4(mom, e0, r.lo, r.hi, m);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) th[j] = __fmaf_rn(na, m[j], th[j]);
+            dat_store4(theta, e0, r.lo, r.hi, th);
+        }
+    }
+}
+
+extern "C" int dat_lalr_step(dat_plan_t *plan, float *theta, float *mom, const float *g_hat,
+                             const dat_hparams_t *hp, float *layer_norms_out, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (!theta || !mom || !g_hat || !hp) return DAT_ERR_ARG;
+    if (!dat_aligned16(theta) || !dat_aligned16(mom) || !dat_aligned16(g_hat) ||
+        (layer_norms_out && !dat_aligned16(layer_norms_out)))
+        return DAT_ERR_ALIGN;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int h = (int)plan->h;
+    k_lalr_pass1<<<(unsigned)plan->n_tiles, DAT_THREADS, 0, s>>>(theta, mom, g_hat, plan->d_offsets,
+                                                                 plan->d_tile_base, h, hp->momentum,
+                                                                 hp->weight_decay, plan->d_partials);
+    DAT_LAUNCHED(plan);
+    k_lalr_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base, plan->d_partials, hp->lr, hp->c_l, hp->c_u,
+                                              plan->d_step_a, layer_norms_out, plan->d_status);
+    DAT_LAUNCHED(plan);
+    k_lalr_pass2<<<(unsigned)plan->n_tiles, DAT_THREADS, 0, s>>>(theta, mom, plan->d_offsets, plan->d_tile_base,
+                                                                 h, plan->d_step_a);
+    DAT_LAUNCHED(plan);
+    return DAT_OK;
+}

@@ -1,0 +1,327 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element.
+
+Bit-exact: packed level and sign planes, integer code sums, g_hat and m' (given equal scales).
+Scales: within 1 fp32 ulp of the oracle's (both accumulate exact squares in fp64; only the
+summation order differs); the oracle is then given the GPU's scale bits so that everything
+downstream is comparable bit for bit.  theta', m' end to end: 1e-5 relative.
+"""
+import numpy as np
+import pytest
+import torch
+
+from helpers import (REL_TOL, GpuPlan, assert_close_per_layer, hp_tuple, np_of, oracle_planes, to_dev,
+                     ulp_diff)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def api():
+    assert torch.cuda.is_available()
+    from paper_2206_06257_b200 import api as _api
+    return _api
+
+
+def _offs(sizes):
+    return np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+
+
+def _random_problem(seed, sizes, M, sigma_lo=-5, sigma_hi=-1, dist="normal"):
+    rng = np.random.RandomState(seed)
+    offs = _offs(sizes)
+    d = int(offs[-1])
+    sig = np.repeat(10.0 ** rng.uniform(sigma_lo, sigma_hi, size=len(sizes)), sizes)
+    grads = []
+    for _ in range(M):
+        z = rng.standard_t(3, d) if dist == "t3" else rng.randn(d)
+        grads.append((z * sig).astype(np.float32))
+    theta = (rng.randn(d) * 0.05).astype(np.float32)
+    mom = (rng.randn(d) * 1e-3).astype(np.float32)
+    return offs, grads, theta, mom
+
+
+def _check_unfused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5):
+    M = len(grads)
+    d = int(offs[-1])
+    g_dev = [torch.from_numpy(g).cuda() for g in grads]
+    with GpuPlan(api, offs, M, bits) as P:
+        lv, sg, sc = P.alloc_message()
+        api.dat_quantize(P.plan, g_dev, seed, step, lv, sg, sc)
+        torch.cuda.synchronize()
+        sc_gpu = np_of(sc)
+        # S1: scales within 1 ulp
+        sc_ref = oracle.scales(oracle.worker_norms(offs, grads))
+        assert ulp_diff(sc_gpu, sc_ref).max() <= 1
+        n_scale_mismatch = int((sc_gpu != sc_ref).sum())
+        # S2+S3: planes bit-exact given the GPU's scales
+        level, neg = oracle.quantize(offs, grads, bits, seed, step, sc_gpu)
+        lp_ref, sp_ref = oracle_planes(oracle, level, neg, bits)
+        assert np.array_equal(np_of(lv).reshape(M, -1), lp_ref)
+        assert np.array_equal(np_of(sg).reshape(M, -1), sp_ref)
+        # S4+S5
+        cs = torch.full((d + 8,), 12345, dtype=torch.int32, device="cuda")[:d]
+        gh = torch.zeros(d, dtype=torch.float32, device="cuda")
+        api.dat_aggregate(P.plan, lv, sg, sc, cs, gh)
+        cs_ref, gh_ref = oracle.aggregate(offs, level, neg, sc_gpu, bits)
+        assert np.array_equal(np_of(cs), cs_ref)
+        assert np.array_equal(np_of(gh).view(np.uint32), gh_ref.view(np.uint32))
+        # S6-S8
+        th_d, mo_d = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        norms = torch.zeros(2 * P.h, dtype=torch.float32, device="cuda")
+        api.dat_lalr_step(P.plan, th_d, mo_d, gh, hp, norms)
+        th_ref, mo_ref, norms_ref = oracle.lalr(offs, theta, mom, gh_ref, *hp)
+        assert np.array_equal(np_of(mo_d).view(np.uint32), mo_ref.view(np.uint32))
+        assert ulp_diff(np_of(norms).reshape(-1, 2), norms_ref).max() <= 1
+        assert_close_per_layer(np_of(th_d), th_ref, offs, "theta (unfused)")
+        assert P.status() == 0
+        return n_scale_mismatch
+
+
+def _check_fused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5):
+    M = len(grads)
+    d = int(offs[-1])
+    g_dev = [torch.from_numpy(g).cuda() for g in grads]
+    with GpuPlan(api, offs, M, bits) as P:
+        th_d, mo_d = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        cs = torch.full((d,), 777, dtype=torch.int32, device="cuda")
+        norms = torch.zeros(2 * P.h, dtype=torch.float32, device="cuda")
+        sc = torch.zeros(P.h, dtype=torch.float32, device="cuda")
+        api.dat_step(P.plan, th_d, mo_d, g_dev, seed, step, hp, cs, norms, sc)
+        torch.cuda.synchronize()
+        assert P.status() == 0
+        ref = oracle.step(offs, theta, mom, grads, bits, seed, step, *hp)
+        if bits != 32:
+            sc_gpu = np_of(sc)
+            assert ulp_diff(sc_gpu, ref["scales"]).max() <= 1
+            if not np.array_equal(sc_gpu, ref["scales"]):        # conditional protocol: same scale bits
+                ref = oracle.step(offs, theta, mom, grads, bits, seed, step, *hp, scales_in=sc_gpu)
+            assert np.array_equal(np_of(cs), ref["code_sum"])
+        assert np.array_equal(np_of(mo_d).view(np.uint32), ref["mom"].view(np.uint32))
+        assert ulp_diff(np_of(norms).reshape(-1, 2), ref["layer_norms"]).max() <= 1
+        assert_close_per_layer(np_of(th_d), ref["theta"], offs, "theta (fused)")
+        assert_close_per_layer(np_of(mo_d), ref["mom"], offs, "mom (fused)")
+        # a second call on fresh copies gives bit-identical results (run-to-run determinism)
+        th2, mo2 = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        api.dat_step(P.plan, th2, mo2, g_dev, seed, step, hp)
+        torch.cuda.synchronize()
+        assert torch.equal(th2, th_d) and torch.equal(mo2, mo_d)
+        return np_of(th_d), np_of(mo_d)
+
+
+HP = (0.1, 0.9, 5e-4, 0.0, 10.0)
+
+# several tiles + ragged tails + tiny and odd-sized layers (offsets not multiples of 4)
+SIZES_RAGGED = [1, 2, 3, 5, 31, 32, 33, 4096, 4097, 10, 12289, 7, 20001, 64, 8191]
+
+
+@pytest.mark.parametrize("bits", [1, 2, 4, 8, 16])
+def test_unfused_parity_ragged(api, oracle, bits):
+    offs, grads, theta, mom = _random_problem(bits, SIZES_RAGGED, 3)
+    _check_unfused(api, oracle, offs, grads, theta, mom, bits, HP)
+
+
+@pytest.mark.parametrize("bits", [1, 2, 4, 8, 16, 32])
+def test_fused_parity_ragged(api, oracle, bits):
+    offs, grads, theta, mom = _random_problem(100 + bits, SIZES_RAGGED, 3)
+    _check_fused(api, oracle, offs, grads, theta, mom, bits, HP)
+
+
+@pytest.mark.parametrize("M", [1, 2, 5, 8, 13, 32, 64])
+def test_fused_parity_worker_counts(api, oracle, M):
+    offs, grads, theta, mom = _random_problem(M, [1000, 5000, 3, 9000], M, dist="t3")
+    _check_fused(api, oracle, offs, grads, theta, mom, 4, HP)
+
+
+def test_fused_equals_unfused_on_gpu(api, oracle):
+    offs, grads, theta, mom = _random_problem(7, SIZES_RAGGED, 4)
+    M, d = 4, int(offs[-1])
+    g_dev = [torch.from_numpy(g).cuda() for g in grads]
+    with GpuPlan(api, offs, M, 8) as P:
+        lv, sg, sc = P.alloc_message()
+        gh = torch.zeros(d, dtype=torch.float32, device="cuda")
+        th1, mo1 = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        api.dat_quantize(P.plan, g_dev, 1, 2, lv, sg, sc)
+        api.dat_aggregate(P.plan, lv, sg, sc, None, gh)
+        api.dat_lalr_step(P.plan, th1, mo1, gh, HP)
+        th2, mo2 = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        api.dat_step(P.plan, th2, mo2, g_dev, 1, 2, HP)
+        torch.cuda.synchronize()
+        assert torch.equal(th1, th2) and torch.equal(mo1, mo2)
+
+
+def test_b32_unfused_average(api, oracle):
+    offs, grads, theta, mom = _random_problem(8, [100, 4099, 3], 5)
+    g_dev = [torch.from_numpy(g).cuda() for g in grads]
+    with GpuPlan(api, offs, 5, 32) as P:
+        gh = torch.zeros(int(offs[-1]), dtype=torch.float32, device="cuda")
+        api.dat_average(P.plan, g_dev, gh)
+        assert np.array_equal(np_of(gh).view(np.uint32), oracle.average(offs, grads).view(np.uint32))
+        with pytest.raises(api.DatError) as e:
+            api.dat_quantize(P.plan, g_dev, 0, 0, gh, gh, gh)
+        assert e.value.code == api.DAT_ERR_BITS
+
+
+def test_m1_b32_is_plain_lalr(api, oracle):
+    offs, grads, theta, mom = _random_problem(9, [300, 5000], 1)
+    th, mo = _check_fused(api, oracle, offs, grads, theta, mom, 32, HP)
+    th_ref, mo_ref, _ = oracle.lalr(offs, theta, mom, grads[0], *HP)
+    assert np.array_equal(mo, mo_ref)
+    assert_close_per_layer(th, th_ref, offs, "theta")
+
+
+def test_zero_norm_conventions(api, oracle):
+    offs, grads, theta, mom = _random_problem(10, [500, 700, 900, 64], 3)
+    for g in grads:
+        g[offs[1]:offs[2]] = 0.0            # a layer whose gradient is zero for every worker
+    theta[offs[2]:offs[3]] = 0.0            # an all-zero parameter tensor (momentum non-zero)
+    theta[offs[3]:] = 0.0
+    mom[offs[3]:] = 0.0                     # zero parameters, zero momentum: u = g_hat only
+    th, mo = _check_fused(api, oracle, offs, grads, theta, mom, 8, HP)
+    assert np.isfinite(th).all() and np.isfinite(mo).all()
+    assert not th[offs[2]:offs[3]].any()    # tau(0) = c_l = 0: does not move
+    assert mo[offs[2]:offs[3]].any()
+    _check_unfused(api, oracle, offs, grads, theta, mom, 8, HP)
+
+
+def test_all_zero_everything(api, oracle):
+    offs = _offs([10, 5000])
+    z = np.zeros(int(offs[-1]), dtype=np.float32)
+    th, mo = _check_fused(api, oracle, offs, [z, z.copy()], z.copy(), z.copy(), 8, HP)
+    assert not th.any() and not mo.any()
+
+
+def test_scales_in_is_used(api, oracle):
+    offs, grads, theta, mom = _random_problem(11, [1000, 3000], 2)
+    g_dev = [torch.from_numpy(g).cuda() for g in grads]
+    with GpuPlan(api, offs, 2, 8) as P:
+        lv, sg, sc = P.alloc_message()
+        mine = np.array([0.5, 2.0], dtype=np.float32)      # larger and (for layer 0 maybe) smaller than max|g|
+        mine[0] = np.abs(np.stack(grads)[:, :1000]).max() * 0.5   # forces the clamp to S
+        sin = torch.from_numpy(mine).cuda()
+        api.dat_quantize(P.plan, g_dev, 0, 0, lv, sg, sc, sin)
+        assert np.array_equal(np_of(sc), mine)
+        level, neg = oracle.quantize(offs, grads, 8, 0, 0, mine)
+        assert level.max() == 255
+        lp, sp = oracle_planes(oracle, level, neg, 8)
+        assert np.array_equal(np_of(lv).reshape(2, -1), lp) and np.array_equal(np_of(sg).reshape(2, -1), sp)
+
+
+@pytest.mark.parametrize("name", ["tiny_mlp", "flat_small"])
+def test_config_small(api, oracle, name):
+    from paper_2206_06257_b200 import synth
+    cfg = synth.config(name)
+    theta, mom = synth.make_params(cfg)
+    grads = [g.numpy() for g in synth.make_grads(cfg, 0)]
+    _check_unfused(api, oracle, cfg.offsets, grads, theta.numpy(), mom.numpy(), cfg.bits, hp_tuple(cfg), 0, 0)
+    _check_fused(api, oracle, cfg.offsets, grads, theta.numpy(), mom.numpy(), cfg.bits, hp_tuple(cfg), 0, 0)
+
+
+def test_resnet18_ten_steps_and_resume(api, oracle):
+    """Ten consecutive steps, the step counter advancing the random key; state compared with the
+    oracle after every step; then resume exactness (5 + copy + 5 == 10 straight)."""
+    from paper_2206_06257_b200 import synth
+    cfg = synth.config("resnet18")
+    theta, mom = synth.make_params(cfg)
+    hp = hp_tuple(cfg)
+    th_ref, mo_ref = theta.numpy().copy(), mom.numpy().copy()
+    sigma = synth._per_element(cfg, synth.layer_sigmas(cfg), "cpu")
+    with GpuPlan(api, cfg.offsets, cfg.M, cfg.bits) as P:
+        th_d, mo_d = theta.cuda(), mom.cuda()
+        th_r, mo_r = theta.cuda(), mom.cuda()            # the resumed run
+        sc = torch.zeros(cfg.h, dtype=torch.float32, device="cuda")
+        for t in range(cfg.steps):
+            grads = synth.make_grads(cfg, t, sigma_elem=sigma)
+            g_dev = to_dev(grads)
+            api.dat_step(P.plan, th_d, mo_d, g_dev, cfg.seed, t, hp, None, None, sc)
+            if t == 5:                                   # "checkpoint": copy the state out and back
+                th_r, mo_r = th_r.cpu().cuda(), mo_r.cpu().cuda()
+            api.dat_step(P.plan, th_r, mo_r, g_dev, cfg.seed, t, hp)
+            if t < 3 or t == cfg.steps - 1:
+                # the oracle continues from the GPU's previous state, so that one step is compared
+                ref = oracle.step(cfg.offsets, th_ref, mo_ref, [g.numpy() for g in grads], cfg.bits, cfg.seed, t,
+                                  *hp, scales_in=np_of(sc), want_code_sum=False)
+                assert np.array_equal(np_of(mo_d).view(np.uint32), ref["mom"].view(np.uint32))
+                assert_close_per_layer(np_of(th_d), ref["theta"], cfg.offsets, "theta step %d" % t)
+            th_ref, mo_ref = np_of(th_d).copy(), np_of(mo_d).copy()
+        assert torch.equal(th_d, th_r) and torch.equal(mo_d, mo_r)
+        assert P.status() == 0
+
+
+def test_step_counter_changes_codes(api):
+    offs, grads, theta, mom = _random_problem(12, [5000], 2)
+    g_dev = [torch.from_numpy(g).cuda() for g in grads]
+    with GpuPlan(api, offs, 2, 8) as P:
+        outs = []
+        for seed, step in [(0, 0), (0, 1), (1, 0), (0, 0)]:
+            cs = torch.zeros(5000, dtype=torch.int32, device="cuda")
+            api.dat_step(P.plan, torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda(), g_dev, seed, step,
+                         HP, cs)
+            outs.append(cs.cpu())
+        assert not torch.equal(outs[0], outs[1]) and not torch.equal(outs[0], outs[2])
+        assert torch.equal(outs[0], outs[3])
+
+
+def test_host_detected_errors(api):
+    offs = _offs([100, 200])
+    with pytest.raises(api.DatError) as e:
+        api.dat_plan_create([0, 5, 5], 2, 8)
+    assert e.value.code == api.DAT_ERR_LAYOUT
+    with pytest.raises(api.DatError) as e:
+        api.dat_plan_create(offs, 2, 3)
+    assert e.value.code == api.DAT_ERR_BITS
+    with pytest.raises(api.DatError) as e:
+        api.dat_plan_create(offs, 0, 8)
+    assert e.value.code == api.DAT_ERR_ARG
+    with pytest.raises(api.DatError) as e:
+        api.dat_plan_create(offs, 65, 8)
+    assert e.value.code == api.DAT_ERR_ARG
+    with GpuPlan(api, offs, 2, 8) as P:
+        buf = torch.zeros(400, dtype=torch.float32, device="cuda")
+        th, mo = torch.zeros(300, device="cuda"), torch.zeros(300, device="cuda")
+        g = [torch.zeros(300, device="cuda"), torch.zeros(300, device="cuda")]
+        before = api.dat_plan_launch_count(P.plan)
+        with pytest.raises(api.DatError) as e:                 # misaligned gradient pointer
+            api.dat_step(P.plan, th, mo, [g[0], buf[1:301]], 0, 0, HP)
+        assert e.value.code == api.DAT_ERR_ALIGN
+        with pytest.raises(api.DatError) as e:                 # step does not fit 32 bits
+            api.dat_step(P.plan, th, mo, g, 0, 1 << 32, HP)
+        assert e.value.code == api.DAT_ERR_ARG
+        with pytest.raises(api.DatError) as e:                 # null pointer
+            api.dat_step(P.plan, None, mo, g, 0, 0, HP)
+        assert e.value.code == api.DAT_ERR_ARG
+        with pytest.raises(api.DatError) as e:
+            api.dat_lalr_step(P.plan, th, mo, buf[1:301], HP)
+        assert e.value.code == api.DAT_ERR_ALIGN
+        assert api.dat_plan_launch_count(P.plan) == before     # nothing was launched
+        api.dat_step(P.plan, th, mo, g, 0, 0, HP)              # and the plan still works
+        torch.cuda.synchronize()
+        assert api.dat_plan_launch_count(P.plan) == before + 1
+        assert P.status() == 0
+
+
+def test_nonfinite_input_sets_status_bit(api):
+    offs = _offs([1000, 1000])
+    g = [torch.randn(2000, device="cuda") * 0.01 for _ in range(2)]
+    g[1][1500] = float("inf")
+    with GpuPlan(api, offs, 2, 8) as P:
+        th, mo = torch.randn(2000, device="cuda"), torch.zeros(2000, device="cuda")
+        api.dat_step(P.plan, th, mo, g, 0, 0, HP)
+        assert P.status() & api.DAT_STATUS_NONFINITE
+        assert P.status() == 0                                   # reading clears it
+        assert torch.isfinite(th[:1000]).all()                   # the finite layer is untouched by it
+        g[1][1500] = 0.0
+        api.dat_step(P.plan, torch.randn(2000, device="cuda"), mo.zero_(), g, 0, 1, HP)
+        assert P.status() == 0
+
+
+def test_step_host_matches_device_call(api):
+    offs, grads, theta, mom = _random_problem(13, [3000, 50, 9001], 3)
+    g_dev = [torch.from_numpy(g).cuda() for g in grads]
+    with GpuPlan(api, offs, 3, 8) as P:
+        th_d, mo_d = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        api.dat_step(P.plan, th_d, mo_d, g_dev, 4, 4, HP)
+        th_h = torch.from_numpy(theta.copy()).pin_memory()
+        mo_h = torch.from_numpy(mom.copy()).pin_memory()
+        g_h = [torch.from_numpy(g).pin_memory() for g in grads]
+        api.dat_step_host(P.plan, th_h, mo_h, g_h, 4, 4, HP)
+        assert torch.equal(th_h, th_d.cpu()) and torch.equal(mo_h, mo_d.cpu())
