@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the fused DAT outer-minimisation step (quantize + aggregate + LALR).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config resnet50] [--impl reference]
+
+One "step" is one pass of the whole hot path (dat_step) over one batch of synthetic input:
+the M worker gradient buffers, parameters and momentum of the chosen workload, resident in HBM.
+Prints ONE JSON line (rank 0).  With N > 1 (torchrun) every rank runs an independent replica
+of the workload on its own GPU (the path has no exchange step on one node: replicas only);
+the time is the maximum over ranks and the value the sum of all ranks' elements.
+
+--impl reference times the CPU oracle (the only reference implementation that exists for this
+path) on the host cores, on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "worker-grad elems/s through quantize+aggregate+LALR"
+UNIT = "elems/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy read+write)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+# ------------------------------------------------------------------------------------------
+# clocks during the timed region (read-only NVML queries)
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, device_index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:          # no NVML: report that, do not fail the benchmark
+            self.err = repr(e)
+            self.h = None
+
+    def sample(self):
+        if self.h is None:
+            return
+        try:
+            self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+            try:
+                r = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+            except Exception:
+                r = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            for bit, name in self.REASONS.items():
+                if r & bit and name != "gpu_idle":
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def start(self):
+        if self.h is None:
+            return
+        def loop():
+            while not self._stop.is_set():
+                self.sample()
+                time.sleep(0.01)
+        self._thread = threading.Thread(target=loop, daemon=True)
+        self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+        return {"sm_mhz": int(np.median(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle timing (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------
+def oracle_layer_sample(cfg, max_worker_elems):
+    """A prefix-free sample of layers: every k-th layer, largest stride that keeps the sample
+    below max_worker_elems (whole workload if it fits)."""
+    sizes = np.diff(cfg.offsets)
+    total = int(sizes.sum()) * cfg.M
+    if total <= max_worker_elems:
+        return list(range(cfg.h)), "whole workload (%d layers, %.3g worker-elems)" % (cfg.h, total)
+    stride = 1
+    while True:
+        stride += 1
+        idx = list(range(0, cfg.h, stride))
+        n = int(sizes[idx].sum()) * cfg.M
+        if n <= max_worker_elems or stride >= cfg.h:
+            return idx, "every %d-th layer of the workload (%d of %d layers, %.3g of %.3g worker-elems)" % (
+                stride, len(idx), cfg.h, n, total)
+
+
+def time_oracle(cfg, theta, mom, grads, layers, threads, step=0):
+    """One oracle step restricted to `layers` (numpy inputs).  Returns (seconds, worker_elems)."""
+    import oracle
+    offs = cfg.offsets
+    hp = (cfg.lr, cfg.momentum, cfg.weight_decay, cfg.c_l, cfg.c_u)
+
+    def run(l):
+        a, b = int(offs[l]), int(offs[l + 1])
+        oracle.step(offs, theta[a:b], mom[a:b], [g[a:b] for g in grads], cfg.bits, cfg.seed, step, *hp,
+                    l0=l, l1=l + 1, window=True, want_code_sum=False)
+        return (b - a) * cfg.M
+    order = sorted(layers, key=lambda l: -(offs[l + 1] - offs[l]))     # big layers first
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        n = sum(ex.map(run, order))
+    return time.perf_counter() - t0, n
+
+
+def host_threads():
+    try:
+        n = len(os.sched_getaffinity(0))
+    except Exception:
+        n = os.cpu_count() or 1
+    return max(1, min(n, 32))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    from paper_2206_06257_b200 import synth
+    oracle.lib()
+    cfg = synth.config(args.config)
+    theta, mom = synth.make_params(cfg)
+    grads = [g.numpy() for g in synth.make_grads(cfg, 0)]
+    theta, mom = theta.numpy(), mom.numpy()
+    threads = host_threads()
+    # calibrate on a small sample, then size each step for a run of a few minutes at most
+    cal_layers, _ = oracle_layer_sample(cfg, 4_000_000)
+    t_cal, n_cal = time_oracle(cfg, theta, mom, grads, cal_layers, threads)
+    rate = n_cal / t_cal
+    budget_s = 150.0 / max(1, args.steps + args.warmup)
+    layers, what = oracle_layer_sample(cfg, max(2_000_000, int(rate * min(budget_s, 20.0))))
+    for w in range(args.warmup):
+        time_oracle(cfg, theta, mom, grads, layers, threads, step=w)
+    t_tot, n_tot = 0.0, 0
+    for k in range(args.steps):
+        t, n = time_oracle(cfg, theta, mom, grads, layers, threads, step=k)
+        t_tot += t
+        n_tot += n
+    value = n_tot / t_tot
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": workload_config(cfg, "n/a (host)"),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(cfg, l2_note):
+    return {"workload": cfg.name, "d": cfg.d, "layers": cfg.h, "workers_M": cfg.M, "bits": cfg.bits,
+            "lr": cfg.lr, "momentum": cfg.momentum, "weight_decay": cfg.weight_decay,
+            "grad_dist": cfg.grad_dist, "parallelism": "replicas", "l2": l2_note}
+
+
+# ------------------------------------------------------------------------------------------
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2206_06257_b200 import api, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for this path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = synth.config(args.config)
+    if args.bits:
+        cfg.bits = args.bits
+    theta, mom = synth.make_params(cfg, device=dev)
+    grads = synth.make_grads(cfg, 0, device=dev)
+    hp = (cfg.lr, cfg.momentum, cfg.weight_decay, cfg.c_l, cfg.c_u)
+    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits)
+    stream = torch.cuda.current_stream()
+    working_set = (cfg.M + 2) * cfg.d * 4
+    l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
+    l2_note = ("inputs larger than L2 (%.0f MB touched per step vs %.0f MB L2), no flush" %
+               (working_set / 1e6, l2_bytes / 1e6))
+    flush = None
+    if working_set < 2 * l2_bytes:       # cache-resident workload: flush L2 between timed steps
+        flush = torch.empty(int(2.5 * l2_bytes) // 4, dtype=torch.float32, device=dev)
+        l2_note = "L2 flushed between timed steps (%.0f MB buffer written)" % (flush.numel() * 4 / 1e6)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- warm-up
+    step_no = 0
+    for _ in range(max(args.warmup, 3)):
+        api.dat_step(plan, theta, mom, grads, cfg.seed, step_no, hp)
+        step_no += 1
+    torch.cuda.synchronize()
+    status = api.dat_get_status(plan)
+    if status:
+        raise SystemExit("device status word not clean after warm-up: %d" % status)
+
+    # ---- timed region: exactly K steps, per-step CUDA events on the launching stream
+    K = args.steps
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K)]
+    sampler = ClockSampler(local)
+    launches0 = api.dat_plan_launch_count(plan)
+    barrier()
+    sampler.start()
+    t_wall0 = time.perf_counter()
+    for k in range(K):
+        if flush is not None:
+            flush.fill_(1.0)
+        ev[2 * k].record(stream)
+        api.dat_step(plan, theta, mom, grads, cfg.seed, step_no, hp)
+        ev[2 * k + 1].record(stream)
+        step_no += 1
+    sampler.sample()
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop()
+    launches = api.dat_plan_launch_count(plan) - launches0
+    step_ms = np.array([ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(K)])
+    region_ms = ev[0].elapsed_time(ev[2 * K - 1]) if flush is None else float(step_ms.sum())
+    status = api.dat_get_status(plan)
+    finite = bool(torch.isfinite(theta).all().item() and torch.isfinite(mom).all().item())
+
+    t = torch.tensor([region_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    region_ms_max = float(t.item())
+    elems_per_step = cfg.M * cfg.d
+    value = world * elems_per_step * K / (region_ms_max * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (H2D + step + D2H inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        th_h = theta.detach().cpu().pin_memory()
+        mo_h = mom.detach().cpu().pin_memory()
+        g_h = [g.detach().cpu().pin_memory() for g in grads]
+        n_e2e = max(2, min(K, args.e2e_steps))
+        api.dat_step_host(plan, th_h, mo_h, g_h, cfg.seed, step_no, hp)      # allocates the staging buffers
+        barrier()
+        t0 = time.perf_counter()
+        for k in range(n_e2e):
+            api.dat_step_host(plan, th_h, mo_h, g_h, cfg.seed, step_no + 1 + k, hp)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        tt = torch.tensor([dt], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * elems_per_step * n_e2e / float(tt.item()), "unit": UNIT,
+               "h2d_bytes_per_step": (cfg.M + 2) * cfg.d * 4, "d2h_bytes_per_step": 2 * cfg.d * 4,
+               "steps": n_e2e, "ms_per_step": 1e3 * float(tt.item()) / n_e2e}
+
+    # ---- CPU oracle beside it (rank 0, N = 1 only), on a bounded sample of the same workload
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        import oracle
+        oracle.lib()
+        th_c, mo_c = synth.make_params(cfg)
+        g_c = [g.numpy() for g in synth.make_grads(cfg, 0)]
+        threads = host_threads()
+        cal_layers, _ = oracle_layer_sample(cfg, 4_000_000)
+        t_cal, n_cal = time_oracle(cfg, th_c.numpy(), mo_c.numpy(), g_c, cal_layers, threads)
+        layers, what = oracle_layer_sample(cfg, int(n_cal / t_cal * 15.0))
+        t_or, n_or = time_oracle(cfg, th_c.numpy(), mo_c.numpy(), g_c, layers, threads)
+        cpu = {"value": n_or / t_or, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": what + ", one step, %.1f s" % t_or}
+
+    api.dat_plan_destroy(plan)
+    if rank == 0:
+        peak, peak_src = measured_peaks()
+        kernel_ms = float(step_ms.mean())
+        algo_bytes = (4 * cfg.M + 16) * cfg.d
+        achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
+        prof = os.path.join(ROOT, "profiles", "traffic.json")
+        traffic = None
+        if os.path.exists(prof):
+            try:
+                traffic = json.load(open(prof)).get("%s_b%d" % (cfg.name, cfg.bits))
+            except Exception:
+                traffic = None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+            "ms_per_step": region_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": workload_config(cfg, l2_note),
+            "step_latency_us": {"median": 1e3 * float(np.median(step_ms)), "min": 1e3 * float(step_ms.min()),
+                                "mean": 1e3 * kernel_ms},
+            "pct_of_8TBps": 100.0 * achieved / NOMINAL_HBM_GBS,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "algorithmic_bytes_per_launch": algo_bytes,
+                         "kernel": "k_fused_step (one launch per step)", "peak_source": peak_src},
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "status_word": int(status), "outputs_finite": finite, "wall_s_timed_region": t_wall,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="resnet50",
+                    choices=["tiny_mlp", "resnet18", "resnet50", "resnet50_m32", "flat1b", "flat_small"])
+    ap.add_argument("--bits", type=int, default=0, help="override the config's bits")
+    ap.add_argument("--impl", default="dat", choices=["dat", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
