@@ -116,7 +116,7 @@ int dat_plan_sizes(const dat_plan_t *plan, int64_t *level_bytes_per_worker,
  *   For worker i, layer l, element e (global index in the flat vector), with x = S*|g_e|/nu_l:
  *   level = floor(x) + 1 with probability x - floor(x), else floor(x); sign bit = (g_e < 0).
  *   Randomness: Philox4x32-10, counter (lo(e/4), hi(e/4), i, hi(seed)), key (lo(seed), step),
- *   word e mod 4; u = top 23 bits / 2^23; level = min(floor(fma(|g_e|, S/nu_l, u)), S).
+ *   word e mod 4; u1 = 1 + (low 23 bits)/2^23; level = min(floor(fma(|g_e|, S/nu_l, u1)) - 1, S).
  *
  *   grads      host array of M device pointers, each fp32[d], read-only.
  *   seed,step  random-stream key; step must be < 2^32 (DAT_ERR_ARG).

@@ -45,8 +45,8 @@ def _declare(L):
     L.dat_oracle_philox4x32_10.restype = None
     L.dat_oracle_random_word.argtypes = [_u64, _u64, _u32, _u64]
     L.dat_oracle_random_word.restype = _u32
-    L.dat_oracle_uniform.argtypes = [_u32]
-    L.dat_oracle_uniform.restype = _f32
+    L.dat_oracle_uniform12.argtypes = [_u32]
+    L.dat_oracle_uniform12.restype = _f32
     L.dat_oracle_worker_norms.argtypes = [_i64, _p, _i64, _i64, _int, _p, _p]
     L.dat_oracle_worker_norms.restype = None
     L.dat_oracle_scales.argtypes = [_i64, _i64, _i64, _int, _int, _p, _p]
@@ -125,8 +125,9 @@ def random_word(seed, step, worker, e):
     return int(lib().dat_oracle_random_word(int(seed), int(step), int(worker), int(e)))
 
 
-def uniform(w):
-    return float(lib().dat_oracle_uniform(int(w) & 0xFFFFFFFF))
+def uniform12(w):
+    """1 + u in [1, 2), u from the low 23 bits of w."""
+    return float(lib().dat_oracle_uniform12(int(w) & 0xFFFFFFFF))
 
 
 # ---------------------------------------------------------------- S1

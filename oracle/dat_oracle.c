@@ -30,7 +30,8 @@
  *       workers' integer codes live on one grid and can be summed as integers.
  *       PER_WORKER mode is Eq. grad_agg / Eq. rand_q taken literally per layer.
  *   R3  Randomness: Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11), keyed on
- *       (seed, step, worker, element); 23-bit uniform; level = floor(x + u).
+ *       (seed, step, worker, element); 23-bit uniform u from the low 23 bits of the
+ *       element's word; level = floor(x + u), evaluated as floor(x + (1 + u)) - 1.
  *   R4  Descent direction u_t (which Eq. 3 leaves to "the optimizer employed"):
  *       heavy-ball momentum with coupled weight decay, u = m' = mu*m + g_hat + wd*theta.
  *   R5  Zero norms: tau(0) = c_l (0 by default, so an all-zero tensor does not move);
@@ -92,13 +93,14 @@ uint32_t dat_oracle_random_word(uint64_t seed, uint64_t step, uint32_t worker, u
     return out[e & 3u];
 }
 
-/* Uniform on {0, 2^-23, ..., 1 - 2^-23} from the top 23 bits of a word (exact). */
-float dat_oracle_uniform(uint32_t w)
+/* 1 + u, with u uniform on {0, 2^-23, ..., 1 - 2^-23} taken from the low 23 bits of a word:
+ * the bits become the mantissa of a float in [1, 2) (exact, no arithmetic). */
+float dat_oracle_uniform12(uint32_t w)
 {
-    uint32_t bits = 0x3F800000u | (w >> 9);       /* a float in [1, 2) */
+    uint32_t bits = 0x3F800000u | (w & 0x007FFFFFu);
     float f;
     memcpy(&f, &bits, sizeof f);
-    return f - 1.0f;
+    return f;
 }
 
 /* ------------------------------------------------------------------------- */
@@ -151,10 +153,11 @@ static float scale_of(const float *scales, int scale_mode, int64_t h, int i, int
 
 /* With S = 2^b - 1 and x = S*|g_e|/nu in [0, S]: xi = level/S where
  * level = floor(x) + 1 with probability x - floor(x), else floor(x).
- * Drawn as level = floor(x + u), u uniform on [0,1).  x + u is ONE fused operation
- * fmaf(|g|, S/nu, u), so x itself is never rounded.  The clamp to S covers the two
- * ways the sum can reach S+1: rounding at x = S, and caller-supplied scales
- * smaller than max|g|.
+ * Drawn as level = floor(x + u), u uniform on [0,1).  The random bits give u1 = 1 + u
+ * directly, so the draw is written level = floor(x + u1) - 1; x + u1 is ONE fused
+ * operation fmaf(|g|, S/nu, u1), so x itself is never rounded.  The clamp (of x + u1 to
+ * S + 1, i.e. of the level to S) covers the two ways the sum can exceed it: rounding at
+ * x = S, and caller-supplied scales smaller than max|g|.
  * level[i][e] in {0..S}; neg[i][e] = 1 iff g < 0 (so -0.0 and NaN give 0).       */
 void dat_oracle_quantize(int64_t h, const int64_t *offsets, int64_t l0, int64_t l1,
                          int M, int bits, int scale_mode,
@@ -170,9 +173,9 @@ void dat_oracle_quantize(int64_t h, const int64_t *offsets, int64_t l0, int64_t 
             float t = (nu == 0.0f) ? 0.0f : S_f / nu;
             for (int64_t e = offsets[l]; e < offsets[l + 1]; ++e) {
                 float g = grads[i][e];
-                float u = dat_oracle_uniform(dat_oracle_random_word(seed, step, (uint32_t)i, (uint64_t)e));
-                float y = fminf(fmaf(fabsf(g), t, u), S_f);
-                level[i][e] = (uint32_t)floorf(y);
+                float u1 = dat_oracle_uniform12(dat_oracle_random_word(seed, step, (uint32_t)i, (uint64_t)e));
+                float y = fminf(fmaf(fabsf(g), t, u1), S_f + 1.0f);
+                level[i][e] = (uint32_t)floorf(y) - 1u;
                 neg[i][e] = (uint8_t)(g < 0.0f);
             }
         }

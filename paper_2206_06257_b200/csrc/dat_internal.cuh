@@ -110,13 +110,29 @@ __device__ __forceinline__ void dat_random_words(uint64_t q, uint32_t worker, co
     dat_philox((uint32_t)q, (uint32_t)(q >> 32), worker, k.seed_hi, k, out);
 }
 
-// Stochastic level of one element: floor(|g| * qmul + u) clamped to S, u = top 23 bits of w.
-// y lies in [0, 65535], so adding 2^23 rounding down leaves floor(y) in the low mantissa bits.
-__device__ __forceinline__ uint32_t dat_level(float g, float qmul, float S_f, uint32_t w)
+// Stochastic level of one element (Eq. xi): level = min(floor(|g|*qmul + u), S) with u uniform
+// on [0,1).  The low 23 bits of the random word w are the mantissa of u1 = 1 + u in [1,2), so
+// y = fma(|g|, qmul, u1) is clamped to S+1 and level = floor(y) - 1.  y lies in [1, 65537):
+// adding 2^23 - 1 with rounding toward -inf leaves floor(y) - 1 in the low mantissa bits.
+// Returns those float bits, 0x4B000000 + level.
+__device__ __forceinline__ uint32_t dat_level_bits(float g, float qmul, float S1_f, uint32_t w)
 {
-    const float u = __uint_as_float(0x3F800000u | (w >> 9)) - 1.0f;
-    const float y = fminf(__fmaf_rn(fabsf(g), qmul, u), S_f);
-    return __float_as_uint(__fadd_rd(y, 8388608.0f)) & 0x007FFFFFu;
+    const float u1 = __uint_as_float(0x3F800000u | (w & 0x007FFFFFu));
+    const float y = fminf(__fmaf_rn(fabsf(g), qmul, u1), S1_f);
+    return __float_as_uint(__fadd_rd(y, 8388607.0f));
+}
+
+__device__ __forceinline__ uint32_t dat_level(float g, float qmul, float S1_f, uint32_t w)
+{
+    return dat_level_bits(g, qmul, S1_f, w) & 0x007FFFFFu;
+}
+
+// sum += sign(g) * level, from the bits of dat_level_bits: with sm = 0 or -1 (all ones) for
+// g's sign bit, (level ^ sm) - sm is level or -level.  (-0.0 has level 0, so its sign is moot.)
+__device__ __forceinline__ int dat_add_signed_level(int sum, float g, uint32_t level_bits)
+{
+    const int sm = (int)__float_as_uint(g) >> 31;
+    return sum + (int)((level_bits & 0x007FFFFFu) ^ (uint32_t)sm) - sm;
 }
 
 // Largest l in [0, h) with table[l] <= x (table[0] <= x < table[h] assumed).

@@ -100,7 +100,7 @@ k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h,
     const int worker = blockIdx.y;
     const int64_t e_tile = tile * DAT_TILE;
     const float *__restrict__ g = gp.p[worker];
-    const float S_f = (float)((1u << BITS) - 1u);
+    const float S1_f = (float)(1u << BITS);                  // S + 1
 
     if (threadIdx.x == 0) s_first = dat_find(off, h, e_tile);
     __syncthreads();
@@ -125,7 +125,7 @@ k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h,
                 l_hi = __ldg(off + l + 1);
                 t = __ldg(qmul + l);
             }
-            lev[j] = (e < d) ? dat_level(gv[j], t, S_f, w[j]) : 0u;
+            lev[j] = (e < d) ? dat_level(gv[j], t, S1_f, w[j]) : 0u;
             neg |= (uint32_t)(gv[j] < 0.0f) << j;
         }
         // pack the group's level bits

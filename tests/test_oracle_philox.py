@@ -46,16 +46,20 @@ def test_streams_differ_across_seed_step_worker(oracle):
 
 
 def test_uniform_grid_and_range(oracle):
-    assert oracle.uniform(0) == 0.0
-    assert oracle.uniform(0x1FF) == 0.0                    # low 9 bits are dropped
-    assert oracle.uniform(0x200) == 2.0 ** -23
-    assert oracle.uniform(0xFFFFFFFF) == 1.0 - 2.0 ** -23
-    assert oracle.uniform(0x80000000) == 0.5
+    """uniform12 = 1 + u, u = (low 23 bits) / 2^23: exact, in [1, 2)."""
+    assert oracle.uniform12(0) == 1.0
+    assert oracle.uniform12(0xFF800000) == 1.0              # high 9 bits are dropped
+    assert oracle.uniform12(1) == 1.0 + 2.0 ** -23
+    assert oracle.uniform12(0xFFFFFFFF) == 2.0 - 2.0 ** -23
+    assert oracle.uniform12(0x00400000) == 1.5
+    for w in (0x12345678, 0x9ABCDEF0, 0x007FFFFF):
+        assert oracle.uniform12(w) == 1.0 + (w & 0x7FFFFF) / 2.0 ** 23
 
 
 def test_uniform_moments(oracle):
     n = 20000
-    u = np.array([oracle.uniform(oracle.random_word(7, 3, 1, e)) for e in range(n)])
+    u = np.array([oracle.uniform12(oracle.random_word(7, 3, 1, e)) for e in range(n)]) - 1.0
+    assert u.min() >= 0.0 and u.max() < 1.0
     assert abs(u.mean() - 0.5) < 5 * (1 / 12 ** 0.5) / n ** 0.5
     assert abs(u.var() - 1 / 12) < 0.004
     # bits look balanced
