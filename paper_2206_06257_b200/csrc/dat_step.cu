@@ -1,7 +1,7 @@
 // dat_step: Steps 7, 9 and 12 of Algorithm A1 in ONE persistent, warp-specialised kernel.
 //
 // The flat vector is cut into per-layer tiles of FT elements.  Every tile passes through three
-// stages of work, each a work item:
+// work items:
 //   N  read the M gradient tiles, fp64 sums of squares per worker.  When a layer's last
 //      contribution has arrived, nu_l, S/nu_l and nu_l/(S*M) are published  [||g||_2 of Eq. rand_q]
 //   Q  (needs nu_l) re-read the gradient tiles -- by construction still in L2 for layers that
@@ -10,36 +10,47 @@
 //      and m'^2.  When a layer is complete, a_l = lr*tau(||theta_l||)/||u_l|| is published [Eq. 3]
 //   U  (needs a_l) theta -= a_l * m'                                                    [Eq. 3]
 //
-// The host lays the items out as a software pipeline: the N items of one window of layers are
-// interleaved with the Q items of the previous window and the U items of the one before, so
-// that HBM streaming (N) overlaps the L2- and ALU-bound work (Q, U) and a layer's dependency
-// is normally met long before its consumers are reached.  CTA c (one per SM) executes items
-// c, c+G, c+2G, ... in order.  Inside a CTA one producer warp walks the list ahead of the
-// consumers and moves every tile into a ring of shared-memory stages with bulk asynchronous
-// copies (cp.async.bulk, completion counted on an mbarrier; no multicast); eight consumer
-// warps take the stages in order.  Tiles that touch a layer boundary or are not full are read
-// with ordinary masked loads instead.
+// The host lays the items out as one list in which N runs ahead of Q and Q ahead of U by just
+// enough for the dependencies (and no more than L2 can hold); CTA c (two per SM) owns items
+// c, c+G, c+2G, ...  Inside a CTA the work is split by role:
+//   - two NORM warps stream the CTA's N items straight from HBM with wide loads (HBM-bound,
+//     fp64/conversion pipes);
+//   - a PRODUCER warp walks the Q and U items ahead of the consumers, waits for the layer flags
+//     and moves every tile (M gradient rows, theta, m) into a ring of shared-memory stages with
+//     bulk asynchronous copies (cp.async.bulk, completion counted on an mbarrier; no multicast);
+//   - eight CONSUMER warps take the stages in order (integer/fp32 pipes: Philox, levels, sums);
+//   - a REDUCER warp takes the per-warp partial sums of both groups, keeps the CTA's running
+//     sums per layer, publishes them, and -- for the contribution that completes a layer --
+//     reduces all contributions in a fixed order and releases the layer's flag.  This keeps the
+//     global-memory round trips of the reductions off the streaming and computing warps.
+// Tiles that touch a layer boundary or are not full are read with ordinary masked loads.
 //
 // An item depends only on items earlier in the list and all CTAs are co-resident (cooperative
-// launch), so the list cannot deadlock.  Every wait -- on an mbarrier, on a layer flag -- is
-// bounded all the same: when one runs out the thread sets DAT_STATUS_TIMEOUT and the CTA's abort
-// flag, every other waiter sees it and leaves, the producer waits (bounded) for its copies in
-// flight, and the kernel returns; the last CTA out clears the dependency counters.
+// launch), so the list cannot deadlock.  Every wait -- on an mbarrier, on a layer flag, on the
+// norm warps' throttle -- is bounded all the same: when one runs out the thread sets
+// DAT_STATUS_TIMEOUT and the CTA's abort flag, every other waiter sees it and leaves, the
+// producer waits (bounded) for its copies in flight, and the kernel returns; the last CTA out
+// clears the dependency counters.
 #include <algorithm>
 #include <new>
 
 #include "dat_internal.cuh"
 
 #define FT 1024                                  // elements per fused tile
-#define F_CW 8                                   // consumer warps
+#define F_CW 8                                   // consumer warps (Q and U items)
 #define F_CT (F_CW * 32)                         // consumer threads; thread t owns elements 4t..4t+3
-#define F_THREADS (F_CT + 64)                    // + one producer warp + one reducer warp
+#define F_NW 2                                   // norm warps (N items)
+#define F_NT (F_NW * 32)
+#define F_THREADS (F_CT + F_NT + 64)             // + one producer warp + one reducer warp
 #define F_ROWS 4                                 // worker rows per stage
-#define F_STAGES 4
-#define F_RED 2                                  // reduction hand-off buffers
+#define F_STAGES 3
+#define F_NBUF 2                                 // norm warps' own tile buffers (F_ROWS rows each)
+#define F_RED 2                                  // reduction hand-off buffers per group
+#define F_NLEAD 6                                // list items the norm warps may run ahead of the producer
 #define F_CTAS_PER_SM 2
 #define F_STAGE_FLOATS ((F_ROWS + 2) * FT)       // gradient rows + theta row + momentum row
 #define F_STAGE_BYTES (F_STAGE_FLOATS * 4)
+#define F_NBUF_FLOATS (F_ROWS * FT)
 #define F_WAIT_CYCLES (1ll << 31)                // bound of every device-side wait (about a second)
 
 enum { ITEM_N = 0u, ITEM_Q = 1u, ITEM_U = 2u, ITEM_END = 3u };
@@ -56,6 +67,7 @@ struct FusedSchedule {
     double *d_npart = nullptr;        // slots * M
     double *d_qpart = nullptr;        // slots * 2
     size_t sync_words = 0;
+    int64_t n_slots = 0;
     uint32_t epoch = 0;
     int grid = 0;
     int64_t window_bytes = 0;
@@ -80,11 +92,15 @@ struct FusedArgs {
 #ifdef DAT_PROF
     unsigned long long *prof;                    // development builds only
 #endif
+#ifdef DAT_SELFCHECK
+    long long d, n_slots;                        // self-checking builds: bounds of the flat vector and of the slots
+    long long *check_log;                        // [0] = number of violations, then (site, value) pairs
+#endif
 };
 
 // What a stage holds: written by the producer (four 16-byte stores), read by every consumer thread.
 struct __align__(16) StageHdr {
-    uint32_t kind;                               // ITEM_*
+    uint32_t kind;                               // ITEM_Q, ITEM_U or ITEM_END
     uint32_t flags;                              // HDR_*
     int layer;
     int chunk;                                   // which group of F_ROWS workers
@@ -95,7 +111,7 @@ struct __align__(16) StageHdr {
 };
 enum { HDR_FAST = 1u, HDR_FLUSH = 2u, HDR_LAST_CHUNK = 4u };
 
-// What the consumers hand to the reducer warp with a buffer of per-warp partial sums.
+// What a group hands to the reducer warp with a buffer of per-warp partial sums.
 struct RedDesc {
     uint32_t kind;                               // ITEM_N, ITEM_Q or ITEM_END
     uint32_t flush;
@@ -104,8 +120,9 @@ struct RedDesc {
 };
 
 #ifdef DAT_PROF
+// counters: 0 c.wait_full 1 n.wait 2 c.Q 3 c.U 4 n.work 5 r.work 6 p.wait_empty 7 p.wait_flag 8 p.issue 9 total
 #define PROF_T0() const long long prof_t0 = clock64()
-#define PROF_ADD(k) do { if (a.prof && (threadIdx.x & 31) == 0 && (threadIdx.x == 0 || threadIdx.x >= F_CT)) a.prof[blockIdx.x * 16 + (k)] += (unsigned long long)(clock64() - prof_t0); } while (0)
+#define PROF_ADD(k) do { if (a.prof && (threadIdx.x & 31) == 0 && (threadIdx.x == 0 || threadIdx.x == F_CT || threadIdx.x >= F_CT + F_NT)) a.prof[blockIdx.x * 16 + (k)] += (unsigned long long)(clock64() - prof_t0); } while (0)
 #define PROF_TRACE(role, idx, col, val) do { if (a.prof && blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (idx) < 4096) a.prof[296 * 16 + ((role) * 4096 + (idx)) * 8 + (col)] = (unsigned long long)(val); } while (0)
 #else
 #define PROF_TRACE(role, idx, col, val) do {} while (0)
@@ -113,14 +130,46 @@ struct RedDesc {
 #define PROF_ADD(k) do {} while (0)
 #endif
 
+// What a norm buffer holds: written by the issuing norm warp, read by both.
+struct __align__(16) NormHdr {
+    uint32_t kind;                               // ITEM_N or ITEM_END
+    uint32_t flags;                              // HDR_FAST | HDR_FLUSH | HDR_LAST_CHUNK
+    int layer;
+    int row0;                                    // first worker row of this pass
+    long long begin, lo;
+    long long hi, slot;
+};
+
+#ifdef DAT_SELFCHECK
+// Self-checking build: a failed check records (site, value), sets DAT_STATUS_BOUNDS and the
+// guarded access is skipped.
+#define DAT_CHECK(cond, site, value) ((cond) ? true : (dat_check_fail(a, (site), (long long)(value)), false))
+__device__ __noinline__ void dat_check_fail(const FusedArgs &a, int site, long long value)
+{
+    atomicOr(a.status, DAT_STATUS_BOUNDS);
+    if (a.check_log) {
+        const unsigned long long k = atomicAdd((unsigned long long *)a.check_log, 1ull);
+        if (k < 64) { a.check_log[1 + 2 * k] = ((long long)blockIdx.x << 32) | (threadIdx.x << 8) | site; a.check_log[2 + 2 * k] = value; }
+    }
+}
+#else
+#define DAT_CHECK(cond, site, value) (true)
+#endif
+
 struct Shared {
     unsigned long long full[F_STAGES], empty[F_STAGES];
-    unsigned long long red_full[F_RED], red_empty[F_RED];
+    unsigned long long nfull[F_NBUF], nempty[F_NBUF];         // norm warps' buffers
+    unsigned long long nred_full[F_RED], nred_empty[F_RED];   // norm warps -> reducer
+    unsigned long long qred_full[F_RED], qred_empty[F_RED];   // consumer warps -> reducer
     StageHdr hdr[F_STAGES];
-    RedDesc rdesc[F_RED];
-    double red[F_RED][F_CW][DAT_MAX_WORKERS];    // per-warp partial sums handed to the reducer
+    NormHdr nhdr[F_NBUF];
+    RedDesc ndesc[F_RED], qdesc[F_RED];
+    double red_n[F_RED][F_NW][DAT_MAX_WORKERS];  // per-warp sums of squares of one N item
+    double red_q[F_RED][F_CW][2];                // per-warp sums of theta^2 and m'^2 of one Q item
     double acc_n[DAT_MAX_WORKERS];               // the CTA's running sums for its current layer (reducer)
     double acc_q[2];
+    int q_pos;                                   // list position of the producer (throttles the norm warps)
+    int n_issued;                                // passes the norm warps have started
     int abort_flag;
 };
 
@@ -145,6 +194,16 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, uint32_t 
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_test_wait(unsigned long long *bar, uint32_t parity)      // never blocks
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
@@ -208,9 +267,9 @@ __device__ __forceinline__ bool wait_flag(Shared &sh, const uint32_t *flag, uint
     return false;
 }
 
-// ---- producer warp -------------------------------------------------------------------------------
+// ---- walking the item list -----------------------------------------------------------------------
 // The layer a kind of item is working in (items of one kind come in layer order), with what
-// the producer has already learnt about it.
+// the walker has already learnt about it.
 struct LayerCursor {
     int layer = -1;
     long long t0 = 0, t1 = 0, lo = 0, hi = 0;
@@ -230,35 +289,279 @@ __device__ __forceinline__ void cursor_seek(const FusedArgs &a, LayerCursor &c, 
     c.flag_seen = false;
 }
 
-// All 32 lanes walk the CTA's item list together (warp-uniform control flow).  Per stage: wait
-// until the slot is free, announce the bytes, start the copies (lane r moves row r), write the
-// stage header, arrive.  Layer flags are waited for here, ahead of the consumers; a flag already
-// seen is not read again.  Returns the number of stages issued.
+// Where the CTA's running sums of a layer go: layers with at most G tiles use one slot per tile
+// (the CTA's first tile of the run names it), larger layers one slot per CTA.
+__device__ __forceinline__ long long cursor_slot(const FusedArgs &a, LayerCursor &c, long long tile, bool flush)
+{
+    if (c.first_tile < 0) c.first_tile = tile;
+    const long long nt = c.t1 - c.t0;
+    const long long slot = __ldg(a.slot_base + c.layer) + ((nt <= (long long)gridDim.x) ? (c.first_tile - c.t0) : (long long)blockIdx.x);
+    if (flush) c.first_tile = -1;
+    return slot;
+}
+
+// Cross-lane sum of four per-lane values: after the call, lanes with (lane & 7) == 0 hold the
+// warp total of value number (lane >> 3).  Fixed order: 2 exchange-and-halve steps, 3 plain.
+__device__ __forceinline__ double warp_sum4(double v[4], int lane)
+{
+    {
+        const bool up = lane & 16;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const double send = up ? v[k] : v[k + 2], keep = up ? v[k + 2] : v[k];
+            v[k] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 16);
+        }
+    }
+    {
+        const bool up = lane & 8;
+        const double send = up ? v[0] : v[1], keep = up ? v[1] : v[0];
+        v[0] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 8);
+    }
+    v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 4);
+    v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 2);
+    v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
+    return v[0];
+}
+
+// ---- norm warps ------------------------------------------------------------------------------------
+// Each pass over F_ROWS worker rows of a tile goes through one of the norm warps' own
+// shared-memory buffers.  The first norm warp walks the CTA's N items and starts the bulk copies
+// up to F_NBUF passes ahead (lane r moves row r); both warps then add the exact fp64 squares of
+// their halves of every pass, in order, and hand the per-warp sums of each item to the reducer.
+struct NormWalk {
+    long long it;                                // list index of next_item
+    int pos;                                     // its position in the CTA's list
+    uint32_t next_item;
+    LayerCursor cn;
+    bool have_item = false;                      // an N item has been found and waits for the throttle
+    uint32_t item = 0;
+    int item_pos = 0;
+    // the item being cut into passes
+    int row0 = -1;
+    long long begin = 0, slot = 0;
+    bool fast = false, flush = false;
+};
+
+enum { NORM_ISSUED = 0, NORM_END = 1, NORM_LATER = 2, NORM_FAIL = 3 };
+
+// Tries to start pass number `seq` (buffer seq % F_NBUF): the next F_ROWS rows of the current
+// item, or of the next N item of the list -- unless that item is still too far ahead of the
+// producer (NORM_LATER: the caller goes on with what is already in flight; what is streamed here
+// must still be in L2 when the consumers re-read it).  Writes the buffer's header; ITEM_END when
+// the list is exhausted.  Called by the whole first norm warp.
+__device__ __forceinline__ int norm_issue(const FusedArgs &a, Shared &sh, float *nbuf, NormWalk &w, uint32_t seq, int lane)
+{
+    const uint32_t b = seq % F_NBUF, use = seq / F_NBUF;
+    const long long G = gridDim.x;
+    if (w.row0 < 0) {                            // next N item
+        if (!w.have_item) {
+            while (w.it < a.n_items) {
+                const uint32_t item = w.next_item;
+                const int pos = w.pos;
+                if (w.it + G < a.n_items) w.next_item = __ldg(a.items + w.it + G);
+                w.it += G; w.pos++;
+                if ((item >> 30) == ITEM_N) { w.have_item = true; w.item = item; w.item_pos = pos; break; }
+            }
+        }
+        if (!w.have_item) {
+            if (!wait_mbar(sh, &sh.nempty[b], (use & 1u) ^ 1u, a.status)) return NORM_FAIL;
+            if (lane == 0) { sh.nhdr[b].kind = ITEM_END; sh.n_issued = (int)seq + 1; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.nfull[b]);
+            return NORM_END;
+        }
+        if (w.item_pos > *(volatile int *)&sh.q_pos + F_NLEAD) return NORM_LATER;
+        const long long tile = w.item & ITEM_TILE_MASK;
+        cursor_seek(a, w.cn, tile);
+        w.flush = (w.item & ITEM_FLUSH) != 0;
+        w.slot = cursor_slot(a, w.cn, tile, w.flush);
+        w.begin = (w.cn.lo & ~3ll) + (tile - w.cn.t0) * FT;
+        w.fast = (w.begin >= w.cn.lo) && (w.begin + FT <= w.cn.hi);
+        w.row0 = 0;
+        w.have_item = false;
+    }
+    const int rows = min(F_ROWS, a.M - w.row0);
+    const bool last = (w.row0 + F_ROWS >= a.M);
+    if (!wait_mbar(sh, &sh.nempty[b], (use & 1u) ^ 1u, a.status)) return NORM_FAIL;
+    if (w.fast) {
+        if (lane == 0) mbar_expect_tx(&sh.nfull[b], (uint32_t)rows * (FT * 4));
+        __syncwarp();
+        if (lane < rows) {
+            if (DAT_CHECK(w.begin >= 0 && w.begin + FT <= a.d && w.row0 + lane < a.M && (w.begin & 3) == 0, 1, w.begin))
+                bulk_g2s(nbuf + (size_t)b * F_NBUF_FLOATS + lane * FT, a.gp.p[w.row0 + lane] + w.begin, FT * 4, &sh.nfull[b]);
+        }
+    }
+    if (lane == 0) {
+        uint4 *H = reinterpret_cast<uint4 *>(&sh.nhdr[b]);
+        const uint32_t flags = (w.fast ? HDR_FAST : 0u) | (w.flush ? HDR_FLUSH : 0u) | (last ? HDR_LAST_CHUNK : 0u);
+        H[0] = make_uint4(ITEM_N, flags, (uint32_t)w.cn.layer, (uint32_t)w.row0);
+        H[1] = make_uint4((uint32_t)w.begin, (uint32_t)(w.begin >> 32), (uint32_t)w.cn.lo, (uint32_t)(w.cn.lo >> 32));
+        H[2] = make_uint4((uint32_t)w.cn.hi, (uint32_t)(w.cn.hi >> 32), (uint32_t)w.slot, (uint32_t)(w.slot >> 32));
+        sh.n_issued = (int)seq + 1;
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.nfull[b]);
+    w.row0 = last ? -1 : w.row0 + F_ROWS;
+    return NORM_ISSUED;
+}
+
+// F_ROWS rows of a full tile from a norm buffer: thread nt owns the 16-byte groups nt + 64k.
+template <bool FULL>
+__device__ __forceinline__ void norm_rows(const float *buf, int rows, int nt, double acc[F_ROWS])
+{
+#pragma unroll
+    for (int r = 0; r < F_ROWS; ++r) {
+        acc[r] = 0.0;
+        if (FULL || r < rows) {
+            const float4 *g = reinterpret_cast<const float4 *>(buf + r * FT) + nt;
+#pragma unroll
+            for (int k = 0; k < FT / 4 / F_NT; ++k) {
+                const float4 v = g[F_NT * k];
+                acc[r] = fma((double)v.x, (double)v.x, acc[r]);
+                acc[r] = fma((double)v.y, (double)v.y, acc[r]);
+                acc[r] = fma((double)v.z, (double)v.z, acc[r]);
+                acc[r] = fma((double)v.w, (double)v.w, acc[r]);
+            }
+        }
+    }
+}
+
+// The same for a tile at a layer boundary: masked global loads, one group at a time.
+__device__ __noinline__ void norm_rows_masked(const FusedArgs &a, int row0, int rows, long long begin, long long lo,
+                                               long long hi, int nt, double acc[F_ROWS])
+{
+#pragma unroll 1
+    for (int r = 0; r < F_ROWS; ++r) {
+        double s = 0.0;
+        if (r < rows) {
+            const float *__restrict__ g = a.gp.p[row0 + r];
+#pragma unroll 1
+            for (int k = 0; k < FT / 4 / F_NT; ++k) {
+                float v[4];
+                dat_load4(g, begin + 4 * (long long)(nt + F_NT * k), lo, hi, v);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) s = fma((double)v[j], (double)v[j], s);
+            }
+        }
+        acc[r] = s;
+    }
+}
+
+// One pass: both norm warps.  Returns false at the end marker or when a wait gave up.
+__device__ __forceinline__ bool norm_consume(const FusedArgs &a, Shared &sh, const float *nbuf, uint32_t seq,
+                                             uint32_t &nred, int nt)
+{
+    const int lane = nt & 31, nw = nt >> 5;
+    const uint32_t b = seq % F_NBUF, use = seq / F_NBUF;
+    if (!wait_mbar(sh, &sh.nfull[b], use & 1u, a.status)) return false;
+    PROF_T0();
+    const NormHdr &H = sh.nhdr[b];
+    if (H.kind != ITEM_N) return false;
+    const uint32_t flags = H.flags;
+    const int row0 = H.row0, rows = min(F_ROWS, a.M - row0);
+    const uint32_t rb = nred % F_RED, ruse = nred / F_RED;
+    double acc[F_ROWS];
+    if ((flags & HDR_FAST) && rows == F_ROWS) norm_rows<true>(nbuf + (size_t)b * F_NBUF_FLOATS, rows, nt, acc);
+    else if (flags & HDR_FAST) norm_rows<false>(nbuf + (size_t)b * F_NBUF_FLOATS, rows, nt, acc);
+    else norm_rows_masked(a, row0, rows, H.begin, H.lo, H.hi, nt, acc);
+    const int layer = H.layer;
+    const long long slot = H.slot;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.nempty[b]);
+    // the item's first pass claims a hand-off buffer
+    if (row0 == 0 && !wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return false;
+    const double s = warp_sum4(acc, lane);
+    if ((lane & 7) == 0 && (lane >> 3) < rows) sh.red_n[rb][nw][row0 + (lane >> 3)] = s;
+    if (flags & HDR_LAST_CHUNK) {
+        if (nt == 0) {
+            sh.ndesc[rb].kind = ITEM_N; sh.ndesc[rb].flush = flags & HDR_FLUSH;
+            sh.ndesc[rb].layer = layer; sh.ndesc[rb].slot = slot;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.nred_full[rb]);
+        nred++;
+    }
+    PROF_ADD(4);
+    return true;
+}
+
+__device__ __forceinline__ void norm_warps(const FusedArgs &a, Shared &sh, float *nbuf)
+{
+    static_assert(F_ROWS == 4, "the cross-lane sum is written for four rows");
+    const int nt = threadIdx.x - F_CT, lane = nt & 31, nw = nt >> 5;
+    uint32_t nred = 0, consumed = 0;
+    if (nw != 0) {
+        // the second warp only takes the passes in order
+        while (norm_consume(a, sh, nbuf, consumed, nred, nt)) ++consumed;
+    } else {
+        NormWalk w;
+        w.it = blockIdx.x;
+        w.pos = 0;
+        w.next_item = (blockIdx.x < a.n_items) ? __ldg(a.items + blockIdx.x) : 0u;
+        uint32_t issued = 0;
+        bool ended = false;
+        long long t_idle = 0;
+        for (;;) {
+            // start as many passes as the buffers and the throttle allow; never wait for the
+            // throttle while a started pass has not been taken (its item may be what the
+            // producer is waiting for)
+            while (!ended && issued < consumed + F_NBUF) {
+                const int r = norm_issue(a, sh, nbuf, w, issued, lane);
+                if (r == NORM_FAIL) return;
+                if (r == NORM_LATER) break;
+                issued++;
+                ended = (r == NORM_END);
+            }
+            if (consumed < issued) {
+                if (!norm_consume(a, sh, nbuf, consumed, nred, nt)) break;
+                ++consumed;
+                t_idle = 0;
+            } else {
+                // nothing in flight and the next item is still ahead of the producer
+                PROF_T0();
+                if (t_idle == 0) t_idle = clock64();
+                __nanosleep(64);
+                if (*(volatile int *)&sh.abort_flag) return;
+                if (clock64() - t_idle > F_WAIT_CYCLES) { raise_timeout(sh, a.status); return; }
+                PROF_ADD(1);
+            }
+        }
+    }
+    if (*(volatile int *)&sh.abort_flag) return;
+    const uint32_t rb = nred % F_RED, ruse = nred / F_RED;
+    if (!wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
+    if (nt == 0) sh.ndesc[rb].kind = ITEM_END;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sh.nred_full[rb]);
+}
+
+// ---- producer warp -------------------------------------------------------------------------------
+// All 32 lanes walk the CTA's item list together (warp-uniform control flow), skipping the N
+// items.  Per stage: wait until the slot is free, announce the bytes, start the copies (lane r
+// moves row r), write the stage header, arrive.  Layer flags are waited for here, ahead of the
+// consumers; a flag already seen is not read again.  Returns the number of stages issued.
 template <bool IDENTITY>
 __device__ __forceinline__ uint32_t producer(const FusedArgs &a, Shared &sh, float *stages)
 {
     const int lane = threadIdx.x & 31;
-    LayerCursor cn, cq, cu;
+    LayerCursor cq, cu;
     uint32_t issued = 0;
+    int pos = 0;
     const int nchunks = (a.M + F_ROWS - 1) / F_ROWS;
     const long long G = gridDim.x;
     uint32_t next_item = (blockIdx.x < a.n_items) ? __ldg(a.items + blockIdx.x) : 0u;
-    for (long long it = blockIdx.x; it < a.n_items; it += G) {
+    for (long long it = blockIdx.x; it < a.n_items; it += G, ++pos) {
         const uint32_t item = next_item;
         if (it + G < a.n_items) next_item = __ldg(a.items + it + G);
         const uint32_t type = item >> 30;
+        if (lane == 0) *(volatile int *)&sh.q_pos = pos;
+        if (type == ITEM_N) continue;
         const long long tile = item & ITEM_TILE_MASK;
-        LayerCursor cur = (type == ITEM_N) ? cn : (type == ITEM_Q) ? cq : cu;     // by value: stays in registers
+        LayerCursor cur = (type == ITEM_Q) ? cq : cu;          // by value: stays in registers
         cursor_seek(a, cur, tile);
         const long long begin = (cur.lo & ~3ll) + (tile - cur.t0) * FT;
         const bool fast = (begin >= cur.lo) && (begin + FT <= cur.hi);
-        long long slot_idx = 0;
-        if (type != ITEM_U) {
-            if (cur.first_tile < 0) cur.first_tile = tile;
-            const long long nt = cur.t1 - cur.t0;
-            slot_idx = __ldg(a.slot_base + cur.layer) + ((nt <= G) ? (cur.first_tile - cur.t0) : (long long)blockIdx.x);
-            if (item & ITEM_FLUSH) cur.first_tile = -1;
-        }
+        const long long slot_idx = (type == ITEM_Q) ? cursor_slot(a, cur, tile, (item & ITEM_FLUSH) != 0) : 0;
         if (type == ITEM_U && !cur.flag_seen) {
             // m' of this tile was written by the tile's Q item: the layer's flag orders it
             { PROF_T0();
@@ -280,22 +583,22 @@ __device__ __forceinline__ uint32_t producer(const FusedArgs &a, Shared &sh, flo
             PROF_T0();
             float *st = stages + (size_t)slot * F_STAGE_FLOATS;
             if (fast) {
-                const bool params = (type == ITEM_U) || (type == ITEM_Q && c == nst - 1);   // theta and m rows
+                const bool params = (type == ITEM_U) || (c == nst - 1);                     // theta and m rows
                 const int rows = (type == ITEM_U) ? 0 : min(F_ROWS, a.M - c * F_ROWS);
                 if (lane == 0) mbar_expect_tx(&sh.full[slot], (uint32_t)(rows + (params ? 2 : 0)) * (FT * 4));
                 __syncwarp();
-                PROF_TRACE(1, issued, 4, clock64());
-                if (lane < rows) bulk_g2s(st + lane * FT, a.gp.p[c * F_ROWS + lane] + begin, FT * 4, &sh.full[slot]);
-                if (params && lane == F_ROWS) bulk_g2s(st + F_ROWS * FT, a.theta + begin, FT * 4, &sh.full[slot]);
-                if (params && lane == F_ROWS + 1) bulk_g2s(st + (F_ROWS + 1) * FT, a.mom + begin, FT * 4, &sh.full[slot]);
+                const bool in_range = DAT_CHECK(begin >= 0 && begin + FT <= a.d && (begin & 3) == 0 && c * F_ROWS + rows <= a.M, 2, begin);
+                if (in_range && lane < rows) bulk_g2s(st + lane * FT, a.gp.p[c * F_ROWS + lane] + begin, FT * 4, &sh.full[slot]);
+                if (in_range && params && lane == F_ROWS) bulk_g2s(st + F_ROWS * FT, a.theta + begin, FT * 4, &sh.full[slot]);
+                if (in_range && params && lane == F_ROWS + 1) bulk_g2s(st + (F_ROWS + 1) * FT, a.mom + begin, FT * 4, &sh.full[slot]);
             }
-            PROF_TRACE(1, issued, 5, clock64());
             issued++;
             if (type == ITEM_Q && !IDENTITY && !cur.flag_seen) {
                 // every copy announced above has been started, so the stage completes even if
                 // this wait gives up
                 PROF_T0();
                 if (!wait_flag(sh, a.flag_n + cur.layer, a.epoch, a.status)) {
+                    if (lane == 0) sh.hdr[slot].kind = ITEM_END;      // nothing valid to consume in this stage
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sh.full[slot]);
                     return issued;
@@ -314,14 +617,14 @@ __device__ __forceinline__ uint32_t producer(const FusedArgs &a, Shared &sh, flo
                 H[2] = make_uint4((uint32_t)cur.hi, (uint32_t)(cur.hi >> 32), (uint32_t)slot_idx, (uint32_t)(slot_idx >> 32));
                 H[3] = make_uint4(__float_as_uint(cur.f0), __float_as_uint(cur.f1), 0u, 0u);
             }
-            PROF_TRACE(1, issued - 1, 6, clock64());
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.full[slot]);      // release: the header is visible once the stage completes
             PROF_ADD(8);
             PROF_TRACE(1, issued - 1, 3, clock64());
         }
-        if (type == ITEM_N) cn = cur; else if (type == ITEM_Q) cq = cur; else cu = cur;
+        if (type == ITEM_Q) cq = cur; else cu = cur;
     }
+    if (lane == 0) *(volatile int *)&sh.q_pos = 0x3FFFFFFF;          // nothing left to stay close to
     {   // end marker
         const uint32_t slot = issued % F_STAGES, use = issued / F_STAGES;
         if (!wait_mbar(sh, &sh.empty[slot], (use & 1u) ^ 1u, a.status)) return issued;
@@ -334,22 +637,20 @@ __device__ __forceinline__ uint32_t producer(const FusedArgs &a, Shared &sh, flo
 }
 
 // ---- reducer warp ----------------------------------------------------------------------------------
-// Takes the consumers' per-warp sums of an item, folds them into the CTA's running sums of the
-// layer and, on a flush item, publishes those to global memory.  The CTA whose contribution
-// completes a layer reduces all contributions in a fixed order and publishes the layer's scale
-// (N) or step length (Q) behind a release flag.  All of this costs several global round trips;
-// keeping it in a warp of its own keeps them off the consumers' path.
+// N: fold the norm warps' sums into the CTA's running sums of the layer; on a flush item publish
+// them and, if that completed the layer, reduce all contributions and publish the scale.
 __device__ __forceinline__ void finish_norm(const FusedArgs &a, Shared &sh, int layer, long long slot, int buf,
                                             bool flush, int lane)
 {
     for (int i = lane; i < a.M; i += 32) {
         double s = sh.acc_n[i];
 #pragma unroll
-        for (int w = 0; w < F_CW; ++w) s += sh.red[buf][w][i];
+        for (int w = 0; w < F_NW; ++w) s += sh.red_n[buf][w][i];
         sh.acc_n[i] = s;
     }
     __syncwarp();
     if (!flush) return;
+    if (!DAT_CHECK(slot >= 0 && slot < a.n_slots && layer >= 0 && layer < a.h, 8, slot)) return;
     for (int i = lane; i < a.M; i += 32) { a.npart[slot * a.M + i] = sh.acc_n[i]; sh.acc_n[i] = 0.0; }
     __threadfence();
     __syncwarp();
@@ -384,17 +685,19 @@ __device__ __forceinline__ void finish_norm(const FusedArgs &a, Shared &sh, int 
     }
 }
 
+// Q: the same for the sums of theta^2 and m'^2; completing a layer publishes its step length.
 __device__ __forceinline__ void finish_quant(const FusedArgs &a, Shared &sh, int layer, long long slot, int buf,
                                              bool flush, int lane)
 {
     if (lane < 2) {
         double s = sh.acc_q[lane];
 #pragma unroll
-        for (int w = 0; w < F_CW; ++w) s += sh.red[buf][w][lane];
+        for (int w = 0; w < F_CW; ++w) s += sh.red_q[buf][w][lane];
         sh.acc_q[lane] = s;
     }
     __syncwarp();
     if (!flush) return;
+    if (!DAT_CHECK(slot >= 0 && slot < a.n_slots && layer >= 0 && layer < a.h, 9, slot)) return;
     if (lane < 2) { a.qpart[slot * 2 + lane] = sh.acc_q[lane]; sh.acc_q[lane] = 0.0; }
     __threadfence();
     __syncwarp();
@@ -423,51 +726,56 @@ __device__ __forceinline__ void finish_quant(const FusedArgs &a, Shared &sh, int
     }
 }
 
-__device__ __forceinline__ void reducer(const FusedArgs &a, Shared &sh)
+// Serves both hand-off rings in turn (non-blocking tests), until both groups have said END.
+__device__ __forceinline__ void reducer(const FusedArgs &a, Shared &sh, bool have_norm_warps)
 {
     const int lane = threadIdx.x & 31;
-    for (uint32_t k = 0;; ++k) {
-        const uint32_t b = k % F_RED, use = k / F_RED;
-        if (!wait_mbar(sh, &sh.red_full[b], use & 1u, a.status)) return;
-        const uint32_t kind = sh.rdesc[b].kind;
-        if (kind == ITEM_END) return;
-        PROF_T0();
-        const bool flush = sh.rdesc[b].flush != 0;
-        const int layer = sh.rdesc[b].layer;
-        const long long slot = sh.rdesc[b].slot;
-        if (kind == ITEM_N) finish_norm(a, sh, layer, slot, (int)b, flush, lane);
-        else finish_quant(a, sh, layer, slot, (int)b, flush, lane);
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.red_empty[b]);
-        PROF_ADD(5);
+    uint32_t kn = 0, kq = 0;
+    bool done_n = !have_norm_warps, done_q = false;
+    long long t_last = clock64();
+    while (!(done_n && done_q)) {
+        bool progress = false;
+        if (!done_n) {
+            const uint32_t b = kn % F_RED;
+            if (mbar_test_wait(&sh.nred_full[b], (kn / F_RED) & 1u)) {
+                PROF_T0();
+                if (sh.ndesc[b].kind == ITEM_END) done_n = true;
+                else {
+                    finish_norm(a, sh, sh.ndesc[b].layer, sh.ndesc[b].slot, (int)b, sh.ndesc[b].flush != 0, lane);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh.nred_empty[b]);
+                }
+                kn++;
+                progress = true;
+                PROF_ADD(5);
+            }
+        }
+        if (!done_q) {
+            const uint32_t b = kq % F_RED;
+            if (mbar_test_wait(&sh.qred_full[b], (kq / F_RED) & 1u)) {
+                PROF_T0();
+                if (sh.qdesc[b].kind == ITEM_END) done_q = true;
+                else {
+                    finish_quant(a, sh, sh.qdesc[b].layer, sh.qdesc[b].slot, (int)b, sh.qdesc[b].flush != 0, lane);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sh.qred_empty[b]);
+                }
+                kq++;
+                progress = true;
+                PROF_ADD(5);
+            }
+        }
+        if (progress) {
+            t_last = clock64();
+        } else {
+            if (*(volatile int *)&sh.abort_flag) return;
+            if (clock64() - t_last > F_WAIT_CYCLES) { raise_timeout(sh, a.status); return; }
+            __nanosleep(20);
+        }
     }
 }
 
 // ---- consumer warps -----------------------------------------------------------------------------------
-// Cross-lane sum of F_ROWS (= 4) per-lane values: after the call, lanes with (lane & 7) == 0 hold
-// the warp total of value number (lane >> 3).  Fixed order: 2 exchange-and-halve steps, 3 plain.
-__device__ __forceinline__ double warp_sum_rows(double v[F_ROWS], int lane)
-{
-    static_assert(F_ROWS == 4, "warp_sum_rows is written for four rows");
-    {
-        const bool up = lane & 16;
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            const double send = up ? v[k] : v[k + 2], keep = up ? v[k + 2] : v[k];
-            v[k] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 16);
-        }
-    }
-    {
-        const bool up = lane & 8;
-        const double send = up ? v[0] : v[1], keep = up ? v[1] : v[0];
-        v[0] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 8);
-    }
-    v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 4);
-    v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 2);
-    v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
-    return v[0];
-}
-
 // The four elements of consumer thread `ct` in one row of a tile: from the stage (bulk-copied
 // tiles) or, masked, from global memory (tiles at a layer boundary).
 template <bool FAST>
@@ -482,32 +790,17 @@ __device__ __forceinline__ void load_group(const float *stage_row, const float *
     }
 }
 
-template <bool FAST, bool FULL>
-__device__ __forceinline__ void rows_sumsq(const FusedArgs &a, const float *st, int chunk, int rows, long long e0,
-                                           long long lo, long long hi, int ct, double acc[F_ROWS])
-{
-#pragma unroll
-    for (int r = 0; r < F_ROWS; ++r) {
-        acc[r] = 0.0;
-        if (FULL || r < rows) {
-            float v[4];
-            load_group<FAST>(st + r * FT, a.gp.p[chunk * F_ROWS + r], e0, lo, hi, ct, v);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc[r] = fma((double)v[j], (double)v[j], acc[r]);
-        }
-    }
-}
-
-template <bool IDENTITY, bool FAST, bool FULL>
+// The F_ROWS worker rows of one chunk of a full tile, from the stage.
+template <bool IDENTITY, bool FULL>
 __device__ __forceinline__ void rows_quant(const FusedArgs &a, const float *st, int chunk, int rows, long long e0,
-                                           long long lo, long long hi, int ct, float qmul, int sum[4], float facc[4])
+                                           int ct, float qmul, int sum[4], float facc[4])
 {
     const float S1_f = a.S_f + 1.0f;
 #pragma unroll
     for (int r = 0; r < F_ROWS; ++r) {
         if (FULL || r < rows) {
-            float v[4];
-            load_group<FAST>(st + r * FT, a.gp.p[chunk * F_ROWS + r], e0, lo, hi, ct, v);
+            const float4 f = *reinterpret_cast<const float4 *>(st + r * FT + 4 * ct);
+            const float v[4] = {f.x, f.y, f.z, f.w};
             if (IDENTITY) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) facc[j] += v[j];
@@ -522,10 +815,32 @@ __device__ __forceinline__ void rows_quant(const FusedArgs &a, const float *st, 
     }
 }
 
+// The same for a tile at a layer boundary: masked global loads, one row at a time.
+template <bool IDENTITY>
+__device__ __noinline__ void rows_quant_masked(const FusedArgs &a, int chunk, int rows, long long e0, long long lo,
+                                               long long hi, float qmul, int sum[4], float facc[4])
+{
+    const float S1_f = a.S_f + 1.0f;
+#pragma unroll 1
+    for (int r = 0; r < rows; ++r) {
+        float v[4];
+        dat_load4(a.gp.p[chunk * F_ROWS + r], e0, lo, hi, v);
+        if (IDENTITY) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) facc[j] += v[j];
+        } else {
+            uint32_t w[4];
+            dat_random_words((uint64_t)e0 >> 2, (uint32_t)(chunk * F_ROWS + r), a.keys, w);
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                sum[j] = dat_add_signed_level(sum[j], v[j], dat_level_bits(v[j], qmul, S1_f, w[j]));
+        }
+    }
+}
+
 // Eight warps; consumer thread ct owns elements 4ct..4ct+3 of every tile.  Everything a stage
 // needs to know comes from its header, so the consumers touch global memory only for the
-// results (and for the masked loads of boundary tiles).  Per-warp partial sums go to the
-// reducer warp through a small ring of buffers; the consumers never wait for global memory.
+// results (and for the masked loads of boundary tiles).
 template <bool IDENTITY>
 __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const float *stages)
 {
@@ -547,10 +862,10 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
         taken++;
         const uint32_t rb = nred % F_RED, ruse = nred / F_RED;
         if (kind == ITEM_END) {
-            if (!wait_mbar(sh, &sh.red_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
-            if (ct == 0) sh.rdesc[rb].kind = ITEM_END;
+            if (!wait_mbar(sh, &sh.qred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
+            if (ct == 0) sh.qdesc[rb].kind = ITEM_END;
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.red_full[rb]);
+            if (lane == 0) mbar_arrive(&sh.qred_full[rb]);
             return;
         }
         const uint32_t flags = H.flags;
@@ -559,37 +874,17 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
         const long long lo = H.lo, hi = H.hi, e0 = H.begin + 4 * (long long)ct;
         const float f0 = H.f0, f1 = H.f1;
         const float *st = stages + (size_t)slot * F_STAGE_FLOATS;
-        const int rows = min(F_ROWS, a.M - chunk * F_ROWS);
+        if (!DAT_CHECK(kind <= ITEM_U && chunk >= 0 && chunk * F_ROWS < a.M && lo >= 0 && lo < hi && hi <= a.d, 7, chunk)) return;
 
-        if (kind == ITEM_N) {
-            double acc[F_ROWS];
-            if (fast && rows == F_ROWS) rows_sumsq<true, true>(a, st, chunk, rows, e0, lo, hi, ct, acc);
-            else if (fast) rows_sumsq<true, false>(a, st, chunk, rows, e0, lo, hi, ct, acc);
-            else rows_sumsq<false, false>(a, st, chunk, rows, e0, lo, hi, ct, acc);
-            // the item's first chunk claims a hand-off buffer
-            if (chunk == 0 && !wait_mbar(sh, &sh.red_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
-            if (ct == 0 && last_chunk) {
-                sh.rdesc[rb].kind = ITEM_N; sh.rdesc[rb].flush = flags & HDR_FLUSH;
-                sh.rdesc[rb].layer = H.layer; sh.rdesc[rb].slot = H.slot;
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.empty[slot]);
-            const double s = warp_sum_rows(acc, lane);
-            if ((lane & 7) == 0 && (lane >> 3) < rows) sh.red[rb][warp][chunk * F_ROWS + (lane >> 3)] = s;
-            if (last_chunk) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.red_full[rb]);
-                nred++;
-            }
-            PROF_ADD(1);
-        } else if (kind == ITEM_Q) {
+        if (kind == ITEM_Q) {
+            const int rows = min(F_ROWS, a.M - chunk * F_ROWS);
             if (chunk == 0) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) { sum[j] = 0; facc[j] = 0.0f; }
             }
-            if (fast && rows == F_ROWS) rows_quant<IDENTITY, true, true>(a, st, chunk, rows, e0, lo, hi, ct, f0, sum, facc);
-            else if (fast) rows_quant<IDENTITY, true, false>(a, st, chunk, rows, e0, lo, hi, ct, f0, sum, facc);
-            else rows_quant<IDENTITY, false, false>(a, st, chunk, rows, e0, lo, hi, ct, f0, sum, facc);
+            if (fast && rows == F_ROWS) rows_quant<IDENTITY, true>(a, st, chunk, rows, e0, ct, f0, sum, facc);
+            else if (fast) rows_quant<IDENTITY, false>(a, st, chunk, rows, e0, ct, f0, sum, facc);
+            else rows_quant_masked<IDENTITY>(a, chunk, rows, e0, lo, hi, f0, sum, facc);
             if (!last_chunk) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.empty[slot]);
@@ -604,10 +899,9 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
                 load_group<false>(st, a.theta, e0, lo, hi, ct, th);
                 load_group<false>(st, a.mom, e0, lo, hi, ct, m);
             }
-            if (ct == 0) {
-                sh.rdesc[rb].kind = ITEM_Q; sh.rdesc[rb].flush = flags & HDR_FLUSH;
-                sh.rdesc[rb].layer = H.layer; sh.rdesc[rb].slot = H.slot;
-            }
+            const uint32_t hflush = flags & HDR_FLUSH;
+            const int hlayer = H.layer;
+            const long long hslot = H.slot;
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.empty[slot]);
             if (IDENTITY) {
@@ -629,13 +923,17 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
                 ss0 = fma((double)th[j], (double)th[j], ss0);
                 ss1 = fma((double)m[j], (double)m[j], ss1);
             }
-            if (e0 < hi) dat_store4(a.mom, e0, lo, hi, m);
+            if (e0 < hi && DAT_CHECK(lo >= 0 && hi <= a.d && e0 >= 0, 5, e0)) dat_store4(a.mom, e0, lo, hi, m);
             ss0 = dat_warp_sum(ss0);
             ss1 = dat_warp_sum(ss1);
-            if (!wait_mbar(sh, &sh.red_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
-            if (lane == 0) { sh.red[rb][warp][0] = ss0; sh.red[rb][warp][1] = ss1; }
+            if (!wait_mbar(sh, &sh.qred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
+            if (lane == 0) { sh.red_q[rb][warp][0] = ss0; sh.red_q[rb][warp][1] = ss1; }
+            if (ct == 0) {
+                sh.qdesc[rb].kind = ITEM_Q; sh.qdesc[rb].flush = hflush;
+                sh.qdesc[rb].layer = hlayer; sh.qdesc[rb].slot = hslot;
+            }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.red_full[rb]);
+            if (lane == 0) mbar_arrive(&sh.qred_full[rb]);
             nred++;
             PROF_ADD(2);
         } else {
@@ -652,7 +950,7 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
             if (lane == 0) mbar_arrive(&sh.empty[slot]);
 #pragma unroll
             for (int j = 0; j < 4; ++j) th[j] = __fmaf_rn(f0, m[j], th[j]);
-            if (e0 < hi) dat_store4(a.theta, e0, lo, hi, th);
+            if (e0 < hi && DAT_CHECK(lo >= 0 && hi <= a.d && e0 >= 0, 6, e0)) dat_store4(a.theta, e0, lo, hi, th);
             PROF_ADD(3);
         }
     }
@@ -664,12 +962,21 @@ k_fused_step(const __grid_constant__ FusedArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     float *stages = reinterpret_cast<float *>(smem_raw);
-    Shared &sh = *reinterpret_cast<Shared *>(smem_raw + (size_t)F_STAGES * F_STAGE_BYTES);
+    float *nbuf = stages + (size_t)F_STAGES * F_STAGE_FLOATS;
+    Shared &sh = *reinterpret_cast<Shared *>(smem_raw + (size_t)F_STAGES * F_STAGE_BYTES + (size_t)F_NBUF * F_NBUF_FLOATS * 4);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < F_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], F_CW); }
-        for (int b = 0; b < F_RED; ++b) { mbar_init(&sh.red_full[b], F_CW); mbar_init(&sh.red_empty[b], 1); }
+        for (int b = 0; b < F_NBUF; ++b) { mbar_init(&sh.nfull[b], 1); mbar_init(&sh.nempty[b], F_NW); }
+        for (int b = 0; b < F_RED; ++b) {
+            mbar_init(&sh.nred_full[b], F_NW); mbar_init(&sh.nred_empty[b], 1);
+            mbar_init(&sh.qred_full[b], F_CW); mbar_init(&sh.qred_empty[b], 1);
+        }
+        for (int s = 0; s < F_STAGES; ++s) sh.hdr[s].kind = ITEM_END;
+        for (int b = 0; b < F_NBUF; ++b) sh.nhdr[b].kind = ITEM_END;
         sh.abort_flag = 0;
+        sh.q_pos = 0;
+        sh.n_issued = 0;
         sh.acc_q[0] = sh.acc_q[1] = 0.0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -680,12 +987,22 @@ k_fused_step(const __grid_constant__ FusedArgs a)
     uint32_t issued = 0;
     const int warp = threadIdx.x >> 5;
     if (warp < F_CW) consumer<IDENTITY>(a, sh, stages);
-    else if (warp == F_CW) issued = producer<IDENTITY>(a, sh, stages);
-    else reducer(a, sh);
+    else if (warp < F_CW + F_NW) { if (!IDENTITY) norm_warps(a, sh, nbuf); }
+    else if (warp == F_CW + F_NW) issued = producer<IDENTITY>(a, sh, stages);
+    else reducer(a, sh, !IDENTITY);
     __syncthreads();
-    PROF_ADD(threadIdx.x == 0 ? 9 : 10);
+    PROF_ADD(9);
 
-    if (threadIdx.x == F_CT) {
+    if (threadIdx.x == F_CT && !IDENTITY && *(volatile int *)&sh.abort_flag) {
+        // after an abort the norm warps' last copies may still be in flight: wait (bounded) for the
+        // last use of each of their buffers
+        const uint32_t n = (uint32_t)sh.n_issued, first = n > F_NBUF ? n - F_NBUF : 0;
+        for (uint32_t q = first; q < n; ++q) {
+            const long long t0 = clock64();
+            while (!mbar_test_wait(&sh.nfull[q % F_NBUF], (q / F_NBUF) & 1u) && clock64() - t0 < F_WAIT_CYCLES) {}
+        }
+    }
+    if (threadIdx.x == F_CT + F_NT) {
         // After an abort copies may still be in flight: wait (bounded) for the last use of every
         // stage before the shared memory is given back.
         if (*(volatile int *)&sh.abort_flag) {
@@ -710,6 +1027,10 @@ k_fused_step(const __grid_constant__ FusedArgs a)
 }
 
 // ---- host side -------------------------------------------------------------------------------
+#ifdef DAT_SELFCHECK
+static long long *g_dat_check_log = nullptr;
+extern "C" void dat_selfcheck_set_log(long long *device_buffer) { g_dat_check_log = device_buffer; }
+#endif
 #ifdef DAT_PROF
 static unsigned long long *g_dat_prof = nullptr;
 extern "C" void dat_prof_set_buffer(unsigned long long *device_buffer) { g_dat_prof = device_buffer; }
@@ -768,7 +1089,7 @@ static int fused_prepare(dat_plan_t *plan)
     const int64_t h = plan->h;
     const int G = plan->sm_count * F_CTAS_PER_SM;
     f->grid = G;
-    f->smem_bytes = (size_t)F_STAGES * F_STAGE_BYTES + sizeof(Shared);
+    f->smem_bytes = (size_t)F_STAGES * F_STAGE_BYTES + (size_t)F_NBUF * F_NBUF_FLOATS * 4 + sizeof(Shared);
 
     int l2 = 0;
     cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, plan->device);
@@ -789,6 +1110,7 @@ static int fused_prepare(dat_plan_t *plan)
         }
         tile_base[h] = nt;
         slot_base[h] = ns;
+        f->n_slots = ns;
         if (nt > (int64_t)ITEM_TILE_MASK) return DAT_ERR_UNSUPPORTED;
 
         // how far N may run ahead of Q: the gradient tiles in between must stay in L2
@@ -908,6 +1230,11 @@ extern "C" int dat_step(dat_plan_t *plan, float *theta, float *mom, const float 
 
 #ifdef DAT_PROF
     a.prof = g_dat_prof;
+#endif
+#ifdef DAT_SELFCHECK
+    a.d = plan->d;
+    a.n_slots = f->n_slots;
+    a.check_log = g_dat_check_log;
 #endif
     void *params[] = {(void *)&a};
     const void *fn = identity ? (const void *)k_fused_step<true> : (const void *)k_fused_step<false>;
