@@ -72,7 +72,8 @@ enum {
     DAT_ERR_LAYOUT = -4,       /* offsets[0] != 0 or offsets not strictly increasing           */
     DAT_ERR_CUDA = -5,         /* a CUDA runtime call failed (see dat_last_cuda_error)         */
     DAT_ERR_NOMEM = -6,        /* host or device allocation failed                              */
-    DAT_ERR_UNSUPPORTED = -7   /* valid request that this build does not implement             */
+    DAT_ERR_UNSUPPORTED = -7,  /* valid request that this build does not implement             */
+    DAT_ERR_TOO_LARGE = -8     /* problem exceeds a fixed capacity (dat_lalr_step_static)       */
 };
 
 /* Bits of the device status word. */
@@ -165,6 +166,42 @@ int dat_average(dat_plan_t *plan, const float *const *grads, float *g_hat, void 
  * ------------------------------------------------------------------------------------------- */
 int dat_lalr_step(dat_plan_t *plan, float *theta, float *mom, const float *g_hat,
                   const dat_hparams_t *hp, float *layer_norms_out, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * dat_lalr_step_static -- the update of dat_lalr_step for callers that must not allocate.
+ * (The paper has no counterpart; this is a deployment variant of the same arithmetic.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or impossible -- inside a
+ * framework's own allocator callbacks or a memory-pool's critical section, in a process whose
+ * device memory was handed out completely at start-up, or in a host thread that is not allowed
+ * to take the driver's allocation lock (a latency-critical serving loop).  Creating a plan
+ * calls cudaMalloc; this entry point needs no plan and calls no cudaMalloc, cudaFree or any
+ * other allocating routine.  Its scratch memory (the layer table, two fp64 partial sums per
+ * 4096-element tile, one step length per layer; about 0.6 MB) is a fixed array inside the
+ * library image, so every GPU that loads the library holds it until the process exits.
+ *
+ *   num_layers      h, 1 <= h <= DAT_STATIC_MAX_LAYERS.
+ *   layer_offsets   HOST array of h+1 element offsets (as for dat_plan_create); copied during
+ *                   the call.  The layers may span at most DAT_STATIC_MAX_TILES tiles of 4096
+ *                   elements (each layer occupies ceil((n_l + 3)/4096) or fewer); larger
+ *                   problems are refused with DAT_ERR_TOO_LARGE before anything is launched.
+ *   theta, mom      device fp32[d], updated in place.      g_hat  device fp32[d], read-only.
+ *   hp              host pointer, read during the call.
+ *   layer_norms_out device fp32[2h] or NULL, as in dat_lalr_step.
+ * The result is bit-identical to dat_lalr_step on the same inputs.
+ * First call on a device: it looks up the device address of the scratch array (once per device,
+ * with that device current); make this first call outside any stream capture.  The call is
+ * not thread-safe with respect to other first calls on the same device.
+ * All calls on a device share the one scratch array, which keeps the previous call's contents;
+ * the call clears what has to start at zero.  Two calls whose device work overlaps (different
+ * streams, or different host threads) race on it: serialise them.  Non-finite norms are not
+ * reported (there is no plan whose status word could carry the bit).
+ * Errors: ARG, ALIGN, LAYOUT, TOO_LARGE, UNSUPPORTED (device ordinal >= 64), CUDA.
+ * ------------------------------------------------------------------------------------------- */
+#define DAT_STATIC_MAX_LAYERS 4096
+#define DAT_STATIC_MAX_TILES 32768
+int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_offsets, float *theta, float *mom,
+                         const float *g_hat, const dat_hparams_t *hp, float *layer_norms_out, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * dat_step -- Steps 7, 9 and 12 of Algorithm A1 in one sweep: the result equals

@@ -23,12 +23,13 @@ _lib = C.CDLL(LIB_PATH)
 DAT_MAX_WORKERS = 64
 DAT_SCALE_SHARED_MAX = 0
 DAT_OK, DAT_ERR_ARG, DAT_ERR_ALIGN, DAT_ERR_BITS = 0, -1, -2, -3
-DAT_ERR_LAYOUT, DAT_ERR_CUDA, DAT_ERR_NOMEM, DAT_ERR_UNSUPPORTED = -4, -5, -6, -7
+DAT_ERR_LAYOUT, DAT_ERR_CUDA, DAT_ERR_NOMEM, DAT_ERR_UNSUPPORTED, DAT_ERR_TOO_LARGE = -4, -5, -6, -7, -8
+DAT_STATIC_MAX_LAYERS, DAT_STATIC_MAX_TILES = 4096, 32768
 DAT_STATUS_NONFINITE, DAT_STATUS_TIMEOUT, DAT_STATUS_BOUNDS = 1, 2, 4
 
 # every symbol include/dat.h declares
 EXPORTS = ["dat_plan_create", "dat_plan_destroy", "dat_plan_sizes", "dat_quantize", "dat_aggregate",
-           "dat_average", "dat_lalr_step", "dat_step", "dat_step_host", "dat_get_status",
+           "dat_average", "dat_lalr_step", "dat_lalr_step_static", "dat_step", "dat_step_host", "dat_get_status",
            "dat_plan_launch_count", "dat_strerror", "dat_last_cuda_error"]
 
 
@@ -45,6 +46,7 @@ _lib.dat_quantize.argtypes = [_p, _p, _u64, _u64, _p, _p, _p, _p, _p]
 _lib.dat_aggregate.argtypes = [_p, _p, _p, _p, _p, _p, _p]
 _lib.dat_average.argtypes = [_p, _p, _p, _p]
 _lib.dat_lalr_step.argtypes = [_p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
+_lib.dat_lalr_step_static.argtypes = [_i64, _p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
 _lib.dat_step.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_step_host.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p]
 _lib.dat_get_status.argtypes = [_p, C.POINTER(C.c_uint32), _p]
@@ -143,6 +145,15 @@ def dat_lalr_step(plan, theta, mom, g_hat, hp, layer_norms_out=None, stream=None
     h = _hp(hp)
     _ok(_lib.dat_lalr_step(_p(plan), _ptr(theta), _ptr(mom), _ptr(g_hat), C.byref(h), _ptr(layer_norms_out),
                            _stream(stream)), "dat_lalr_step")
+
+
+def dat_lalr_step_static(layer_offsets, theta, mom, g_hat, hp, layer_norms_out=None, stream=None):
+    """The LALR update without a plan and without any allocation (see include/dat.h).
+    layer_offsets: h+1 int64 values in host memory (any sequence)."""
+    offs = np.ascontiguousarray(layer_offsets, dtype=np.int64)
+    h = _hp(hp)
+    _ok(_lib.dat_lalr_step_static(offs.size - 1, _ptr(offs), _ptr(theta), _ptr(mom), _ptr(g_hat), C.byref(h),
+                                  _ptr(layer_norms_out), _stream(stream)), "dat_lalr_step_static")
 
 
 def dat_step(plan, theta, mom, grads, seed, step, hp, code_sum_out=None, layer_norms_out=None,

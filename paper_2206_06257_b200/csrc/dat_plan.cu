@@ -186,6 +186,7 @@ extern "C" const char *dat_strerror(int code)
     case DAT_ERR_CUDA: return "a CUDA runtime call failed";
     case DAT_ERR_NOMEM: return "out of memory";
     case DAT_ERR_UNSUPPORTED: return "not implemented in this build";
+    case DAT_ERR_TOO_LARGE: return "problem exceeds the fixed capacity of this entry point (see DAT_STATIC_MAX_*)";
     default: return "unknown error code";
     }
 }

@@ -465,3 +465,73 @@ extern "C" int dat_lalr_step(dat_plan_t *plan, float *theta, float *mom, const f
     DAT_LAUNCHED(plan);
     return DAT_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// dat_lalr_step_static: the LALR update for callers that cannot allocate device memory.
+// No plan, no cudaMalloc: the layer table, the per-tile partial sums and the per-layer step
+// lengths live in one fixed array that is part of the library image on every device.
+// ------------------------------------------------------------------------------------------
+struct StaticScratch {
+    int64_t off[DAT_STATIC_MAX_LAYERS + 1];
+    int64_t tile_base[DAT_STATIC_MAX_LAYERS + 1];
+    double partials[2 * DAT_STATIC_MAX_TILES];
+    float step_a[DAT_STATIC_MAX_LAYERS];
+    uint32_t status;
+};
+
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+// In host code `g_static_scratch` is only a handle; the device address has to be asked for,
+// once per device, with that device current.
+#define DAT_STATIC_MAX_DEVICES 64
+static StaticScratch *g_static_ptr[DAT_STATIC_MAX_DEVICES];
+
+extern "C" int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_offsets, float *theta, float *mom,
+                                    const float *g_hat, const dat_hparams_t *hp, float *layer_norms_out,
+                                    void *stream)
+{
+    if (!layer_offsets || !theta || !mom || !g_hat || !hp) return DAT_ERR_ARG;
+    if (num_layers < 1) return DAT_ERR_ARG;
+    if (num_layers > DAT_STATIC_MAX_LAYERS) return DAT_ERR_TOO_LARGE;
+    if (!dat_aligned16(theta) || !dat_aligned16(mom) || !dat_aligned16(g_hat) ||
+        (layer_norms_out && !dat_aligned16(layer_norms_out)))
+        return DAT_ERR_ALIGN;
+    if (layer_offsets[0] != 0) return DAT_ERR_LAYOUT;
+    int64_t tile_base[DAT_STATIC_MAX_LAYERS + 1];              // host stack, 32 KB
+    int64_t nt = 0;
+    for (int64_t l = 0; l < num_layers; ++l) {
+        if (layer_offsets[l + 1] <= layer_offsets[l]) return DAT_ERR_LAYOUT;
+        tile_base[l] = nt;
+        const int64_t a = layer_offsets[l] & ~(int64_t)3;
+        nt += (layer_offsets[l + 1] - a + DAT_TILE - 1) / DAT_TILE;
+        if (nt > DAT_STATIC_MAX_TILES) return DAT_ERR_TOO_LARGE;
+    }
+    tile_base[num_layers] = nt;
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return DAT_ERR_CUDA; }
+    if (dev < 0 || dev >= DAT_STATIC_MAX_DEVICES) return DAT_ERR_UNSUPPORTED;
+    if (!g_static_ptr[dev]) {
+        StaticScratch *p = nullptr;
+        if (cudaGetSymbolAddress((void **)&p, g_static_scratch) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return DAT_ERR_CUDA;
+        }
+        g_static_ptr[dev] = p;
+    }
+    StaticScratch *sc = g_static_ptr[dev];
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t table = (size_t)(num_layers + 1) * sizeof(int64_t);
+    cudaError_t e = cudaMemcpyAsync(sc->off, layer_offsets, table, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(sc->tile_base, tile_base, table, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(&sc->status, 0, sizeof(uint32_t), s);   // the one word that must start at zero
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return DAT_ERR_CUDA; }
+    const int h = (int)num_layers;
+    k_lalr_pass1<<<(unsigned)nt, DAT_THREADS, 0, s>>>(theta, mom, g_hat, sc->off, sc->tile_base, h, hp->momentum,
+                                                      hp->weight_decay, sc->partials);
+    k_lalr_finalize<<<h, DAT_THREADS, 0, s>>>(sc->tile_base, sc->partials, hp->lr, hp->c_l, hp->c_u, sc->step_a,
+                                              layer_norms_out, &sc->status);
+    k_lalr_pass2<<<(unsigned)nt, DAT_THREADS, 0, s>>>(theta, mom, sc->off, sc->tile_base, h, sc->step_a);
+    if (cudaGetLastError() != cudaSuccess) return DAT_ERR_CUDA;
+    return DAT_OK;
+}

@@ -30,7 +30,7 @@ def test_binding_lists_the_same_names():
 
 def test_strerror_and_cpu_side_validation():
     from paper_2206_06257_b200 import api
-    for code in range(-7, 1):
+    for code in range(-8, 1):
         assert api.dat_strerror(code) and "unknown" not in api.dat_strerror(code)
     assert "unknown" in api.dat_strerror(-99)
     # layout faults are reported before any CUDA call, so this works without a GPU
