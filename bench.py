@@ -28,6 +28,9 @@ sys.path.insert(0, ROOT)
 METRIC = "worker-grad elems/s through quantize+aggregate+LALR"
 UNIT = "elems/s"
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_fused_step launch, from the ncu capture
+# summarised under profiles/ (None until taken for the kernel as it stands).
+NCU_DRAM_BYTES_PER_LAUNCH = {"resnet50_b8": None}
 
 
 def measured_peaks():
@@ -188,6 +191,21 @@ def run_reference(args):
     return 0
 
 
+def max_over_ranks(value, world, device):
+    """Maximum of a per-rank scalar over all ranks (the slowest rank sets the job's time)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world, elems_per_step, steps, seconds):
+    """Whole-job throughput of `world` independent replicas that all took `seconds` (the maximum)."""
+    return world * elems_per_step * steps / seconds
+
+
 def workload_config(cfg, l2_note):
     return {"workload": cfg.name, "d": cfg.d, "layers": cfg.h, "workers_M": cfg.M, "bits": cfg.bits,
             "lr": cfg.lr, "momentum": cfg.momentum, "weight_decay": cfg.weight_decay,
@@ -267,12 +285,9 @@ def run_gpu(args):
     status = api.dat_get_status(plan)
     finite = bool(torch.isfinite(theta).all().item() and torch.isfinite(mom).all().item())
 
-    t = torch.tensor([region_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    region_ms_max = float(t.item())
+    region_ms_max = max_over_ranks(region_ms, world, dev)
     elems_per_step = cfg.M * cfg.d
-    value = world * elems_per_step * K / (region_ms_max * 1e-3)
+    value = job_value(world, elems_per_step, K, region_ms_max * 1e-3)
 
     # ---- end to end through the host-buffer entry point (H2D + step + D2H inside the timed region)
     e2e = None
@@ -288,12 +303,10 @@ def run_gpu(args):
             api.dat_step_host(plan, th_h, mo_h, g_h, cfg.seed, step_no + 1 + k, hp)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        tt = torch.tensor([dt], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * elems_per_step * n_e2e / float(tt.item()), "unit": UNIT,
+        dt_max = max_over_ranks(dt, world, dev)
+        e2e = {"value": job_value(world, elems_per_step, n_e2e, dt_max), "unit": UNIT,
                "h2d_bytes_per_step": (cfg.M + 2) * cfg.d * 4, "d2h_bytes_per_step": 2 * cfg.d * 4,
-               "steps": n_e2e, "ms_per_step": 1e3 * float(tt.item()) / n_e2e}
+               "steps": n_e2e, "ms_per_step": 1e3 * dt_max / n_e2e}
 
     # ---- CPU oracle beside it (rank 0, N = 1 only), on a bounded sample of the same workload
     cpu = None
@@ -316,13 +329,7 @@ def run_gpu(args):
         kernel_ms = float(step_ms.mean())
         algo_bytes = (4 * cfg.M + 16) * cfg.d
         achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-        prof = os.path.join(ROOT, "profiles", "traffic.json")
-        traffic = None
-        if os.path.exists(prof):
-            try:
-                traffic = json.load(open(prof)).get("%s_b%d" % (cfg.name, cfg.bits))
-            except Exception:
-                traffic = None
+        traffic = NCU_DRAM_BYTES_PER_LAUNCH.get("%s_b%d" % (cfg.name, cfg.bits))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": region_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
