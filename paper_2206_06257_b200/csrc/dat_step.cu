@@ -32,6 +32,7 @@
 // producer waits (bounded) for its copies in flight, and the kernel returns; the last CTA out
 // clears the dependency counters.
 #include <algorithm>
+#include <cstdlib>
 #include <new>
 
 #include "dat_internal.cuh"
@@ -46,7 +47,7 @@
 #define F_STAGES 3
 #define F_NBUF 2                                 // norm warps' own tile buffers (F_ROWS rows each)
 #define F_RED 2                                  // reduction hand-off buffers per group
-#define F_NLEAD 6                                // list items the norm warps may run ahead of the producer
+#define F_NLEAD 6                                // default: list items the norm warps may run ahead of the producer
 #define F_CTAS_PER_SM 2
 #define F_STAGE_FLOATS ((F_ROWS + 2) * FT)       // gradient rows + theta row + momentum row
 #define F_STAGE_BYTES (F_STAGE_FLOATS * 4)
@@ -58,18 +59,21 @@ enum { ITEM_N = 0u, ITEM_Q = 1u, ITEM_U = 2u, ITEM_END = 3u };
 #define ITEM_TILE_MASK 0x1FFFFFFFu
 
 struct FusedSchedule {
-    uint32_t *d_items = nullptr;
+    uint4 *d_recs = nullptr;          // the item records, grouped by CTA
+    int64_t *d_cta_first = nullptr;   // G+1: first record of each CTA
     int64_t n_items = 0;
-    int64_t *d_tile_base = nullptr;   // h+1, tiles of FT elements
     int64_t *d_slot_base = nullptr;   // h+1, partial-sum slots per layer
     uint32_t *d_expect = nullptr;     // 2h: contributions expected per layer (N, Q)
-    uint32_t *d_sync = nullptr;       // cnt_n[h] cnt_q[h] flag_n[h] flag_q[h] done[1]
+    uint32_t *d_sync = nullptr;       // cnt_n[h] cnt_q[h] done[1]
+    unsigned long long *d_flags = nullptr;   // per layer: (epoch, S/nu) (epoch, nu/(S*M)) (epoch, -a_l)
     double *d_npart = nullptr;        // slots * M
     double *d_qpart = nullptr;        // slots * 2
     size_t sync_words = 0;
     int64_t n_slots = 0;
     uint32_t epoch = 0;
     int grid = 0;
+    int nlead = F_NLEAD;
+    int64_t slack = 0;
     int64_t window_bytes = 0;
     size_t smem_bytes = 0;
 };
@@ -78,15 +82,16 @@ struct FusedArgs {
     GradPtrs gp;
     PhiloxKeys keys;
     float *theta, *mom;
-    const int64_t *off, *tile_base, *slot_base;
-    const uint32_t *items, *expect;
-    int64_t n_items;
+    const int64_t *off, *slot_base, *cta_first;
+    const uint4 *recs;
+    const uint32_t *expect;
     double *npart, *qpart;
-    uint32_t *cnt_n, *cnt_q, *flag_n, *flag_q, *done, *status;
-    float *worker_norms, *scales, *qmul, *dq, *step_a;
+    uint32_t *cnt_n, *cnt_q, *done, *status;
+    unsigned long long *flags;                   // 3 words per layer, each (epoch << 32) | float bits
+    float *worker_norms, *scales;
     int32_t *code_sum;
     float *norms_out, *scales_out;
-    int h, M;
+    int h, M, nlead;
     uint32_t epoch;
     float S_f, SM_f, lr, mu, wd, c_l, c_u;
 #ifdef DAT_PROF
@@ -248,14 +253,73 @@ __device__ __forceinline__ bool wait_mbar(Shared &sh, unsigned long long *bar, u
     return false;
 }
 
-__device__ __forceinline__ bool wait_flag(Shared &sh, const uint32_t *flag, uint32_t epoch, uint32_t *status)
+// ---- the item list -----------------------------------------------------------------------------
+// One 16-byte record per item, written by the host, grouped by CTA in execution order:
+//   x = kind | flush << 2 | fast << 3 | layer << 8     y = partial-sum slot (N, Q)
+//   z, w = first element of the tile (a multiple of 4)
+// "fast" = a full tile inside its layer (moved by bulk copies); other tiles are masked with the
+// layer's bounds.  A warp fetches 32 records with one coalesced load.
+#define REC_FLUSH 4u
+#define REC_FAST 8u
+
+struct Item {
+    uint32_t kind, flags;
+    int layer;
+    long long slot, begin;
+};
+
+__device__ __forceinline__ Item item_from(uint4 r)
 {
-    if (ld_acquire(flag) == epoch) return true;
+    Item it;
+    it.kind = r.x & 3u;
+    it.flags = r.x & (REC_FLUSH | REC_FAST);
+    it.layer = (int)(r.x >> 8);
+    it.slot = r.y;
+    it.begin = (long long)(((unsigned long long)r.w << 32) | r.z);
+    return it;
+}
+
+__device__ __forceinline__ uint4 shfl_rec(uint4 r, int src)
+{
+    return make_uint4(__shfl_sync(0xFFFFFFFFu, r.x, src), __shfl_sync(0xFFFFFFFFu, r.y, src),
+                      __shfl_sync(0xFFFFFFFFu, r.z, src), __shfl_sync(0xFFFFFFFFu, r.w, src));
+}
+
+// The layer's bounds as the consumers need them: exact for masked tiles, the tile itself otherwise.
+__device__ __forceinline__ void item_bounds(const FusedArgs &a, const Item &it, long long &lo, long long &hi)
+{
+    if (it.flags & REC_FAST) { lo = it.begin; hi = it.begin + FT; }
+    else { lo = __ldg(a.off + it.layer); hi = __ldg(a.off + it.layer + 1); }
+}
+
+// Per-layer result words: (epoch << 32) | float bits.  Valid once the epoch matches.
+__device__ __forceinline__ unsigned long long ld_acquire64(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release64(unsigned long long *p, unsigned long long v)
+{
+    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// Waits (bounded) until the `nwords` result words at p carry this call's epoch; returns their
+// float payloads.  One round trip when they are already there.
+__device__ __forceinline__ bool wait_words(Shared &sh, const unsigned long long *p, int nwords, uint32_t epoch,
+                                           uint32_t *status, float out[2])
+{
     const long long t0 = clock64();
-    for (uint32_t spins = 1;; ++spins) {
+    for (uint32_t spins = 0;; ++spins) {
+        const unsigned long long w0 = ld_acquire64(p);
+        const unsigned long long w1 = (nwords > 1) ? ld_acquire64(p + 1) : w0;
+        if ((uint32_t)(w0 >> 32) == epoch && (uint32_t)(w1 >> 32) == epoch) {
+            out[0] = __uint_as_float((uint32_t)w0);
+            out[1] = __uint_as_float((uint32_t)w1);
+            return true;
+        }
         __nanosleep(32);
-        if (ld_acquire(flag) == epoch) return true;
-        if ((spins & 15u) == 0u) {
+        if ((spins & 15u) == 15u) {
             if (*(volatile int *)&sh.abort_flag || (ld_acquire(status) & DAT_STATUS_TIMEOUT)) {
                 atomicExch(&sh.abort_flag, 1);
                 return false;
@@ -265,39 +329,6 @@ __device__ __forceinline__ bool wait_flag(Shared &sh, const uint32_t *flag, uint
     }
     raise_timeout(sh, status);
     return false;
-}
-
-// ---- walking the item list -----------------------------------------------------------------------
-// The layer a kind of item is working in (items of one kind come in layer order), with what
-// the walker has already learnt about it.
-struct LayerCursor {
-    int layer = -1;
-    long long t0 = 0, t1 = 0, lo = 0, hi = 0;
-    long long first_tile = -1;                   // the CTA's first tile of its running sums in this layer
-    bool flag_seen = false;
-    float f0 = 0.0f, f1 = 0.0f;
-};
-
-__device__ __forceinline__ void cursor_seek(const FusedArgs &a, LayerCursor &c, long long tile)
-{
-    if (c.layer >= 0 && tile >= c.t0 && tile < c.t1) return;
-    c.layer = dat_find(a.tile_base, a.h, tile);
-    c.t0 = __ldg(a.tile_base + c.layer);
-    c.t1 = __ldg(a.tile_base + c.layer + 1);
-    c.lo = __ldg(a.off + c.layer);
-    c.hi = __ldg(a.off + c.layer + 1);
-    c.flag_seen = false;
-}
-
-// Where the CTA's running sums of a layer go: layers with at most G tiles use one slot per tile
-// (the CTA's first tile of the run names it), larger layers one slot per CTA.
-__device__ __forceinline__ long long cursor_slot(const FusedArgs &a, LayerCursor &c, long long tile, bool flush)
-{
-    if (c.first_tile < 0) c.first_tile = tile;
-    const long long nt = c.t1 - c.t0;
-    const long long slot = __ldg(a.slot_base + c.layer) + ((nt <= (long long)gridDim.x) ? (c.first_tile - c.t0) : (long long)blockIdx.x);
-    if (flush) c.first_tile = -1;
-    return slot;
 }
 
 // Cross-lane sum of four per-lane values: after the call, lanes with (lane & 7) == 0 hold the
@@ -329,17 +360,15 @@ __device__ __forceinline__ double warp_sum4(double v[4], int lane)
 // up to F_NBUF passes ahead (lane r moves row r); both warps then add the exact fp64 squares of
 // their halves of every pass, in order, and hand the per-warp sums of each item to the reducer.
 struct NormWalk {
-    long long it;                                // list index of next_item
-    int pos;                                     // its position in the CTA's list
-    uint32_t next_item;
-    LayerCursor cn;
+    long long first, n;                          // this CTA's records
+    int pos = 0;                                 // list position of the next record to look at
+    uint4 batch;                                 // lane j holds record (pos rounded down to 32) + j
+    int batch_base = -1;
     bool have_item = false;                      // an N item has been found and waits for the throttle
-    uint32_t item = 0;
+    Item item;
     int item_pos = 0;
-    // the item being cut into passes
-    int row0 = -1;
-    long long begin = 0, slot = 0;
-    bool fast = false, flush = false;
+    int row0 = -1;                               // next worker row of the item being cut into passes
+    long long lo = 0, hi = 0;
 };
 
 enum { NORM_ISSUED = 0, NORM_END = 1, NORM_LATER = 2, NORM_FAIL = 3 };
@@ -352,16 +381,15 @@ enum { NORM_ISSUED = 0, NORM_END = 1, NORM_LATER = 2, NORM_FAIL = 3 };
 __device__ __forceinline__ int norm_issue(const FusedArgs &a, Shared &sh, float *nbuf, NormWalk &w, uint32_t seq, int lane)
 {
     const uint32_t b = seq % F_NBUF, use = seq / F_NBUF;
-    const long long G = gridDim.x;
     if (w.row0 < 0) {                            // next N item
-        if (!w.have_item) {
-            while (w.it < a.n_items) {
-                const uint32_t item = w.next_item;
-                const int pos = w.pos;
-                if (w.it + G < a.n_items) w.next_item = __ldg(a.items + w.it + G);
-                w.it += G; w.pos++;
-                if ((item >> 30) == ITEM_N) { w.have_item = true; w.item = item; w.item_pos = pos; break; }
+        while (!w.have_item && w.pos < w.n) {
+            if ((w.pos & ~31) != w.batch_base) {
+                w.batch_base = w.pos & ~31;
+                w.batch = (w.batch_base + lane < w.n) ? __ldg(a.recs + w.first + w.batch_base + lane) : make_uint4(ITEM_U, 0, 0, 0);
             }
+            const uint4 r = shfl_rec(w.batch, w.pos & 31);
+            if ((r.x & 3u) == ITEM_N) { w.have_item = true; w.item = item_from(r); w.item_pos = w.pos; }
+            w.pos++;
         }
         if (!w.have_item) {
             if (!wait_mbar(sh, &sh.nempty[b], (use & 1u) ^ 1u, a.status)) return NORM_FAIL;
@@ -370,33 +398,29 @@ __device__ __forceinline__ int norm_issue(const FusedArgs &a, Shared &sh, float 
             if (lane == 0) mbar_arrive(&sh.nfull[b]);
             return NORM_END;
         }
-        if (w.item_pos > *(volatile int *)&sh.q_pos + F_NLEAD) return NORM_LATER;
-        const long long tile = w.item & ITEM_TILE_MASK;
-        cursor_seek(a, w.cn, tile);
-        w.flush = (w.item & ITEM_FLUSH) != 0;
-        w.slot = cursor_slot(a, w.cn, tile, w.flush);
-        w.begin = (w.cn.lo & ~3ll) + (tile - w.cn.t0) * FT;
-        w.fast = (w.begin >= w.cn.lo) && (w.begin + FT <= w.cn.hi);
+        if (w.item_pos > *(volatile int *)&sh.q_pos + a.nlead) return NORM_LATER;
+        item_bounds(a, w.item, w.lo, w.hi);
         w.row0 = 0;
         w.have_item = false;
     }
     const int rows = min(F_ROWS, a.M - w.row0);
     const bool last = (w.row0 + F_ROWS >= a.M);
+    const bool fast = (w.item.flags & REC_FAST) != 0;
     if (!wait_mbar(sh, &sh.nempty[b], (use & 1u) ^ 1u, a.status)) return NORM_FAIL;
-    if (w.fast) {
+    if (fast) {
         if (lane == 0) mbar_expect_tx(&sh.nfull[b], (uint32_t)rows * (FT * 4));
         __syncwarp();
         if (lane < rows) {
-            if (DAT_CHECK(w.begin >= 0 && w.begin + FT <= a.d && w.row0 + lane < a.M && (w.begin & 3) == 0, 1, w.begin))
-                bulk_g2s(nbuf + (size_t)b * F_NBUF_FLOATS + lane * FT, a.gp.p[w.row0 + lane] + w.begin, FT * 4, &sh.nfull[b]);
+            if (DAT_CHECK(w.item.begin >= 0 && w.item.begin + FT <= a.d && w.row0 + lane < a.M && (w.item.begin & 3) == 0, 1, w.item.begin))
+                bulk_g2s(nbuf + (size_t)b * F_NBUF_FLOATS + lane * FT, a.gp.p[w.row0 + lane] + w.item.begin, FT * 4, &sh.nfull[b]);
         }
     }
     if (lane == 0) {
         uint4 *H = reinterpret_cast<uint4 *>(&sh.nhdr[b]);
-        const uint32_t flags = (w.fast ? HDR_FAST : 0u) | (w.flush ? HDR_FLUSH : 0u) | (last ? HDR_LAST_CHUNK : 0u);
-        H[0] = make_uint4(ITEM_N, flags, (uint32_t)w.cn.layer, (uint32_t)w.row0);
-        H[1] = make_uint4((uint32_t)w.begin, (uint32_t)(w.begin >> 32), (uint32_t)w.cn.lo, (uint32_t)(w.cn.lo >> 32));
-        H[2] = make_uint4((uint32_t)w.cn.hi, (uint32_t)(w.cn.hi >> 32), (uint32_t)w.slot, (uint32_t)(w.slot >> 32));
+        const uint32_t flags = (fast ? HDR_FAST : 0u) | ((w.item.flags & REC_FLUSH) ? HDR_FLUSH : 0u) | (last ? HDR_LAST_CHUNK : 0u);
+        H[0] = make_uint4(ITEM_N, flags, (uint32_t)w.item.layer, (uint32_t)w.row0);
+        H[1] = make_uint4((uint32_t)w.item.begin, (uint32_t)(w.item.begin >> 32), (uint32_t)w.lo, (uint32_t)(w.lo >> 32));
+        H[2] = make_uint4((uint32_t)w.hi, (uint32_t)(w.hi >> 32), (uint32_t)w.item.slot, (uint32_t)(w.item.slot >> 32));
         sh.n_issued = (int)seq + 1;
     }
     __syncwarp();
@@ -495,9 +519,8 @@ __device__ __forceinline__ void norm_warps(const FusedArgs &a, Shared &sh, float
         while (norm_consume(a, sh, nbuf, consumed, nred, nt)) ++consumed;
     } else {
         NormWalk w;
-        w.it = blockIdx.x;
-        w.pos = 0;
-        w.next_item = (blockIdx.x < a.n_items) ? __ldg(a.items + blockIdx.x) : 0u;
+        w.first = __ldg(a.cta_first + blockIdx.x);
+        w.n = __ldg(a.cta_first + blockIdx.x + 1) - w.first;
         uint32_t issued = 0;
         bool ended = false;
         long long t_idle = 0;
@@ -544,31 +567,29 @@ template <bool IDENTITY>
 __device__ __forceinline__ uint32_t producer(const FusedArgs &a, Shared &sh, float *stages)
 {
     const int lane = threadIdx.x & 31;
-    LayerCursor cq, cu;
     uint32_t issued = 0;
-    int pos = 0;
     const int nchunks = (a.M + F_ROWS - 1) / F_ROWS;
-    const long long G = gridDim.x;
-    uint32_t next_item = (blockIdx.x < a.n_items) ? __ldg(a.items + blockIdx.x) : 0u;
-    for (long long it = blockIdx.x; it < a.n_items; it += G, ++pos) {
-        const uint32_t item = next_item;
-        if (it + G < a.n_items) next_item = __ldg(a.items + it + G);
-        const uint32_t type = item >> 30;
+    const long long first = __ldg(a.cta_first + blockIdx.x);
+    const int n = (int)(__ldg(a.cta_first + blockIdx.x + 1) - first);
+    int q_layer = -1, u_layer = -1;              // layers whose result words this warp has seen
+    float q_f[2] = {0.0f, 0.0f}, u_f[2] = {0.0f, 0.0f};
+    uint4 batch = make_uint4(0, 0, 0, 0);
+    for (int pos = 0; pos < n; ++pos) {
+        if ((pos & 31) == 0) batch = (pos + lane < n) ? __ldg(a.recs + first + pos + lane) : make_uint4(0, 0, 0, 0);
+        const uint4 rec = shfl_rec(batch, pos & 31);
         if (lane == 0) *(volatile int *)&sh.q_pos = pos;
-        if (type == ITEM_N) continue;
-        const long long tile = item & ITEM_TILE_MASK;
-        LayerCursor cur = (type == ITEM_Q) ? cq : cu;          // by value: stays in registers
-        cursor_seek(a, cur, tile);
-        const long long begin = (cur.lo & ~3ll) + (tile - cur.t0) * FT;
-        const bool fast = (begin >= cur.lo) && (begin + FT <= cur.hi);
-        const long long slot_idx = (type == ITEM_Q) ? cursor_slot(a, cur, tile, (item & ITEM_FLUSH) != 0) : 0;
-        if (type == ITEM_U && !cur.flag_seen) {
-            // m' of this tile was written by the tile's Q item: the layer's flag orders it
+        if ((rec.x & 3u) == ITEM_N) continue;
+        const Item item = item_from(rec);
+        const uint32_t type = item.kind;
+        const bool fast = (item.flags & REC_FAST) != 0;
+        long long lo, hi;
+        item_bounds(a, item, lo, hi);
+        if (type == ITEM_U && u_layer != item.layer) {
+            // m' of this tile was written by the tile's Q item: the layer's result word orders it
             { PROF_T0();
-            if (!wait_flag(sh, a.flag_q + cur.layer, a.epoch, a.status)) return issued;
+            if (!wait_words(sh, a.flags + 3 * (long long)item.layer + 2, 1, a.epoch, a.status, u_f)) return issued;
             PROF_ADD(7); }
-            cur.f0 = -__ldcg(a.step_a + cur.layer);
-            cur.flag_seen = true;
+            u_layer = item.layer;
             asm volatile("fence.proxy.async;" ::: "memory");
         }
         const int nst = (type == ITEM_U) ? 1 : nchunks;
@@ -579,10 +600,11 @@ __device__ __forceinline__ uint32_t producer(const FusedArgs &a, Shared &sh, flo
             if (!wait_mbar(sh, &sh.empty[slot], (use & 1u) ^ 1u, a.status)) return issued;
             PROF_ADD(6); }
             PROF_TRACE(1, issued, 1, clock64());
-            PROF_TRACE(1, issued, 2, type | ((unsigned long long)cur.layer << 16));
+            PROF_TRACE(1, issued, 2, type | ((unsigned long long)item.layer << 16));
             PROF_T0();
             float *st = stages + (size_t)slot * F_STAGE_FLOATS;
             if (fast) {
+                const long long begin = item.begin;
                 const bool params = (type == ITEM_U) || (c == nst - 1);                     // theta and m rows
                 const int rows = (type == ITEM_U) ? 0 : min(F_ROWS, a.M - c * F_ROWS);
                 if (lane == 0) mbar_expect_tx(&sh.full[slot], (uint32_t)(rows + (params ? 2 : 0)) * (FT * 4));
@@ -593,36 +615,33 @@ __device__ __forceinline__ uint32_t producer(const FusedArgs &a, Shared &sh, flo
                 if (in_range && params && lane == F_ROWS + 1) bulk_g2s(st + (F_ROWS + 1) * FT, a.mom + begin, FT * 4, &sh.full[slot]);
             }
             issued++;
-            if (type == ITEM_Q && !IDENTITY && !cur.flag_seen) {
+            if (type == ITEM_Q && !IDENTITY && q_layer != item.layer) {
                 // every copy announced above has been started, so the stage completes even if
                 // this wait gives up
                 PROF_T0();
-                if (!wait_flag(sh, a.flag_n + cur.layer, a.epoch, a.status)) {
+                if (!wait_words(sh, a.flags + 3 * (long long)item.layer, 2, a.epoch, a.status, q_f)) {
                     if (lane == 0) sh.hdr[slot].kind = ITEM_END;      // nothing valid to consume in this stage
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sh.full[slot]);
                     return issued;
                 }
                 PROF_ADD(7);
-                cur.f0 = __ldcg(a.qmul + cur.layer);
-                cur.f1 = __ldcg(a.dq + cur.layer);
-                cur.flag_seen = true;
+                q_layer = item.layer;
             }
             if (lane == 0) {
                 uint4 *H = reinterpret_cast<uint4 *>(&sh.hdr[slot]);
-                const uint32_t flags = (fast ? HDR_FAST : 0u) | ((item & ITEM_FLUSH) ? HDR_FLUSH : 0u) |
+                const uint32_t flags = (fast ? HDR_FAST : 0u) | ((item.flags & REC_FLUSH) ? HDR_FLUSH : 0u) |
                                        ((c == nst - 1) ? HDR_LAST_CHUNK : 0u);
-                H[0] = make_uint4(type, flags, (uint32_t)cur.layer, (uint32_t)c);
-                H[1] = make_uint4((uint32_t)begin, (uint32_t)(begin >> 32), (uint32_t)cur.lo, (uint32_t)(cur.lo >> 32));
-                H[2] = make_uint4((uint32_t)cur.hi, (uint32_t)(cur.hi >> 32), (uint32_t)slot_idx, (uint32_t)(slot_idx >> 32));
-                H[3] = make_uint4(__float_as_uint(cur.f0), __float_as_uint(cur.f1), 0u, 0u);
+                H[0] = make_uint4(type, flags, (uint32_t)item.layer, (uint32_t)c);
+                H[1] = make_uint4((uint32_t)item.begin, (uint32_t)(item.begin >> 32), (uint32_t)lo, (uint32_t)(lo >> 32));
+                H[2] = make_uint4((uint32_t)hi, (uint32_t)(hi >> 32), (uint32_t)item.slot, (uint32_t)(item.slot >> 32));
+                H[3] = make_uint4(__float_as_uint(type == ITEM_U ? u_f[0] : q_f[0]), __float_as_uint(q_f[1]), 0u, 0u);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.full[slot]);      // release: the header is visible once the stage completes
             PROF_ADD(8);
             PROF_TRACE(1, issued - 1, 3, clock64());
         }
-        if (type == ITEM_Q) cq = cur; else cu = cur;
     }
     if (lane == 0) *(volatile int *)&sh.q_pos = 0x3FFFFFFF;          // nothing left to stay close to
     {   // end marker
@@ -664,24 +683,40 @@ __device__ __forceinline__ void finish_norm(const FusedArgs &a, Shared &sh, int 
     if (!last) return;
     const long long s0 = __ldg(a.slot_base + layer);
     const int ns = (int)(__ldg(a.slot_base + layer + 1) - s0);
+    // Every lane sums its slots (lane, lane+32, ...) in order, eight workers at a time so that many
+    // independent loads are in flight; then a fixed butterfly across the lanes.
     float nu = 0.0f;
     bool bad = false;
-    for (int i = 0; i < a.M; ++i) {
-        double acc = 0.0;
-        for (int s = lane; s < ns; s += 32) acc += __ldcg(a.npart + (s0 + s) * a.M + i);
-        acc = dat_warp_sum(acc);
-        const float nrm = (float)sqrt(acc);
-        if (lane == 0) a.worker_norms[(long long)i * a.h + layer] = nrm;
-        bad |= !isfinite(nrm);
-        nu = (i == 0 || nrm > nu) ? nrm : nu;
+    for (int i0 = 0; i0 < a.M; i0 += 8) {
+        double acc[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+#pragma unroll 2
+        for (int s = lane; s < ns; s += 32) {
+            const double *p = a.npart + (s0 + s) * a.M + i0;
+            double v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = (i0 + j < a.M) ? __ldcg(p + j) : 0.0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] += v[j];
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (i0 + j < a.M) {
+                const float nrm = (float)sqrt(dat_warp_sum(acc[j]));
+                if (lane == 0) a.worker_norms[(long long)(i0 + j) * a.h + layer] = nrm;
+                bad |= !isfinite(nrm);
+                nu = (i0 + j == 0 || nrm > nu) ? nrm : nu;
+            }
+        }
     }
     if (lane == 0) {
         a.scales[layer] = nu;
-        a.qmul[layer] = (nu == 0.0f) ? 0.0f : a.S_f / nu;
-        a.dq[layer] = (nu == 0.0f) ? 0.0f : nu / a.SM_f;
+        const float qmul = (nu == 0.0f) ? 0.0f : a.S_f / nu;
+        const float dq = (nu == 0.0f) ? 0.0f : nu / a.SM_f;
         if (a.scales_out) a.scales_out[layer] = nu;
         if (bad) atomicOr(a.status, DAT_STATUS_NONFINITE);
-        st_release(a.flag_n + layer, a.epoch);
+        unsigned long long *w = a.flags + 3 * (long long)layer;
+        st_release64(w, ((unsigned long long)a.epoch << 32) | __float_as_uint(qmul));
+        st_release64(w + 1, ((unsigned long long)a.epoch << 32) | __float_as_uint(dq));
     }
 }
 
@@ -712,17 +747,22 @@ __device__ __forceinline__ void finish_quant(const FusedArgs &a, Shared &sh, int
     const long long s0 = __ldg(a.slot_base + layer);
     const int ns = (int)(__ldg(a.slot_base + layer + 1) - s0);
     double x = 0.0, y = 0.0;
-    for (int s = lane; s < ns; s += 32) { x += __ldcg(a.qpart + (s0 + s) * 2); y += __ldcg(a.qpart + (s0 + s) * 2 + 1); }
+#pragma unroll 4
+    for (int s = lane; s < ns; s += 32) {
+        const double2 v = __ldcg(reinterpret_cast<const double2 *>(a.qpart + (s0 + s) * 2));
+        x += v.x;
+        y += v.y;
+    }
     x = dat_warp_sum(x);
     y = dat_warp_sum(y);
     if (lane == 0) {
         const float n_theta = (float)sqrt(x), n_u = (float)sqrt(y);
         const float tau = fminf(fmaxf(n_theta, a.c_l), a.c_u);
         const float ratio = (n_u == 0.0f) ? 0.0f : tau / n_u;
-        a.step_a[layer] = a.lr * ratio;
+        const float neg_a = -(a.lr * ratio);
         if (a.norms_out) { a.norms_out[2 * layer] = n_theta; a.norms_out[2 * layer + 1] = n_u; }
         if (!isfinite(n_theta) || !isfinite(n_u)) atomicOr(a.status, DAT_STATUS_NONFINITE);
-        st_release(a.flag_q + layer, a.epoch);
+        st_release64(a.flags + 3 * (long long)layer + 2, ((unsigned long long)a.epoch << 32) | __float_as_uint(neg_a));
     }
 }
 
@@ -1040,7 +1080,7 @@ void dat_fused_destroy(dat_plan_t *plan)
 {
     FusedSchedule *f = plan->fused;
     if (!f) return;
-    void *ptrs[] = {f->d_items, f->d_tile_base, f->d_slot_base, f->d_expect, f->d_sync, f->d_npart, f->d_qpart};
+    void *ptrs[] = {f->d_recs, f->d_cta_first, f->d_slot_base, f->d_expect, f->d_sync, f->d_flags, f->d_npart, f->d_qpart};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     delete f;
@@ -1094,6 +1134,12 @@ static int fused_prepare(dat_plan_t *plan)
     int l2 = 0;
     cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, plan->device);
     f->window_bytes = l2 > 0 ? (int64_t)l2 / 10 * 7 : (int64_t)32 << 20;
+    f->slack = 2 * (int64_t)G;
+#ifdef DAT_PROF
+    if (const char *e = getenv("DAT_FUSED_WINDOW_MB")) f->window_bytes = (int64_t)atoi(e) << 20;
+    if (const char *e = getenv("DAT_FUSED_SLACK")) f->slack = atoi(e);
+    if (const char *e = getenv("DAT_FUSED_NLEAD")) f->nlead = atoi(e);
+#endif
 
     std::vector<uint32_t> items;
     std::vector<int64_t> tile_base(h + 1), slot_base(h + 1);
@@ -1117,47 +1163,67 @@ static int fused_prepare(dat_plan_t *plan)
         const int64_t tile_bytes = (int64_t)FT * 4 * plan->M;
         const int64_t max_lag = std::max<int64_t>(f->window_bytes / tile_bytes, 2 * (int64_t)G);
         items.reserve((size_t)nt * 3);
-        build_items(items, tile_base, h, identity, /*slack=*/2 * (int64_t)G, max_lag);
-        // flush marks: for every CTA the last N and the last Q item of each layer; count them
-        std::vector<int64_t> last_n((size_t)G, -1), last_q((size_t)G, -1);      // item index of the CTA's latest N/Q
-        std::vector<int> lay_n((size_t)G, -1), lay_q((size_t)G, -1);
+        build_items(items, tile_base, h, identity, f->slack, max_lag);
+        // Records, grouped by CTA (item i belongs to CTA i mod G).  For N and Q items the record
+        // names the slot of the CTA's running sums: layers with at most G tiles use one slot per
+        // tile and flush at once; in larger layers a CTA accumulates over its tiles of the layer
+        // and flushes with its last one (slot = the CTA's index).  expect[] counts the flushes.
         auto layer_of = [&](int64_t tile) {
             return (int64_t)(std::upper_bound(tile_base.begin(), tile_base.end(), tile) - tile_base.begin()) - 1;
         };
-        for (int64_t i = 0; i < (int64_t)items.size(); ++i) {
+        const int64_t n_items = (int64_t)items.size();
+        std::vector<int64_t> cta_first((size_t)G + 1, 0);
+        for (int c = 0; c < G; ++c) cta_first[c + 1] = cta_first[c] + (n_items > c ? (n_items - 1 - c) / G + 1 : 0);
+        std::vector<uint4> recs((size_t)n_items);
+        std::vector<int64_t> last_rec[2] = {std::vector<int64_t>((size_t)G, -1), std::vector<int64_t>((size_t)G, -1)};
+        std::vector<int> last_layer[2] = {std::vector<int>((size_t)G, -1), std::vector<int>((size_t)G, -1)};
+        for (int64_t i = 0; i < n_items; ++i) {
             const uint32_t type = items[i] >> 30;
-            if (type == ITEM_U) continue;
+            const int64_t tile = items[i] & ITEM_TILE_MASK;
             const int cta = (int)(i % G);
-            const int l = (int)layer_of(items[i] & ITEM_TILE_MASK);
-            std::vector<int64_t> &last = (type == ITEM_N) ? last_n : last_q;
-            std::vector<int> &lay = (type == ITEM_N) ? lay_n : lay_q;
-            const int64_t ntl = tile_base[l + 1] - tile_base[l];
-            if (last[cta] >= 0 && (lay[cta] != l)) {           // the CTA moved on to another layer
-                items[last[cta]] |= ITEM_FLUSH;
-                expect[(type == ITEM_N ? 0 : h) + lay[cta]]++;
+            const int64_t r = cta_first[cta] + i / G;
+            const int l = (int)layer_of(tile);
+            const int64_t lo = plan->offsets[l], hi = plan->offsets[l + 1];
+            const int64_t begin = (lo & ~(int64_t)3) + (tile - tile_base[l]) * FT;
+            const bool fast = begin >= lo && begin + FT <= hi;
+            uint32_t info = type | (fast ? REC_FAST : 0u) | ((uint32_t)l << 8);
+            uint32_t slot = 0;
+            if (type != ITEM_U) {
+                const int k = (type == ITEM_N) ? 0 : 1;
+                const int64_t ntl = tile_base[l + 1] - tile_base[l];
+                if (last_rec[k][cta] >= 0 && last_layer[k][cta] != l) {     // the CTA moved on to another layer
+                    recs[last_rec[k][cta]].x |= REC_FLUSH;
+                    expect[k * h + last_layer[k][cta]]++;
+                    last_rec[k][cta] = -1;
+                }
+                if (ntl <= G) {
+                    slot = (uint32_t)(slot_base[l] + (tile - tile_base[l]));
+                    info |= REC_FLUSH;
+                    expect[k * h + l]++;
+                } else {
+                    slot = (uint32_t)(slot_base[l] + cta);
+                    last_rec[k][cta] = r;
+                    last_layer[k][cta] = l;
+                }
             }
-            last[cta] = i;
-            lay[cta] = l;
-            if (ntl <= G) {                                     // small layers: one slot per tile, flush at once
-                items[i] |= ITEM_FLUSH;
-                expect[(type == ITEM_N ? 0 : h) + l]++;
-                last[cta] = -1;
-            }
+            recs[r] = make_uint4(info, slot, (uint32_t)begin, (uint32_t)((uint64_t)begin >> 32));
         }
-        for (int c = 0; c < G; ++c) {
-            if (last_n[c] >= 0) { items[last_n[c]] |= ITEM_FLUSH; expect[lay_n[c]]++; }
-            if (last_q[c] >= 0) { items[last_q[c]] |= ITEM_FLUSH; expect[h + lay_q[c]]++; }
-        }
-        f->n_items = (int64_t)items.size();
-        f->sync_words = (size_t)h * 4 + 64;
-        cudaError_t e = upload(&f->d_items, items);
-        if (e == cudaSuccess) e = upload(&f->d_tile_base, tile_base);
+        for (int k = 0; k < 2; ++k)
+            for (int c = 0; c < G; ++c)
+                if (last_rec[k][c] >= 0) { recs[last_rec[k][c]].x |= REC_FLUSH; expect[k * h + last_layer[k][c]]++; }
+        if (ns > 0xFFFFFFFFll || h >= (1 << 24)) return DAT_ERR_UNSUPPORTED;
+        f->n_items = n_items;
+        f->sync_words = (size_t)h * 2 + 64;
+        cudaError_t e = upload(&f->d_recs, recs);
+        if (e == cudaSuccess) e = upload(&f->d_cta_first, cta_first);
         if (e == cudaSuccess) e = upload(&f->d_slot_base, slot_base);
         if (e == cudaSuccess) e = upload(&f->d_expect, expect);
         if (e == cudaSuccess) e = cudaMalloc((void **)&f->d_sync, f->sync_words * 4);
+        if (e == cudaSuccess) e = cudaMalloc((void **)&f->d_flags, (size_t)h * 3 * 8);
         if (e == cudaSuccess) e = cudaMalloc((void **)&f->d_npart, (size_t)ns * plan->M * 8);
         if (e == cudaSuccess) e = cudaMalloc((void **)&f->d_qpart, (size_t)ns * 16);
         if (e == cudaSuccess) e = cudaMemset(f->d_sync, 0, f->sync_words * 4);
+        if (e == cudaSuccess) e = cudaMemset(f->d_flags, 0, (size_t)h * 3 * 8);
         if (e == cudaSuccess) e = cudaMemset(f->d_npart, 0, (size_t)ns * plan->M * 8);
         if (e == cudaSuccess) e = cudaMemset(f->d_qpart, 0, (size_t)ns * 16);
         if (e != cudaSuccess) { plan->last_cuda = (int)e; (void)cudaGetLastError(); return DAT_ERR_NOMEM; }
@@ -1195,30 +1261,26 @@ extern "C" int dat_step(dat_plan_t *plan, float *theta, float *mom, const float 
     a.theta = theta;
     a.mom = mom;
     a.off = plan->d_offsets;
-    a.tile_base = f->d_tile_base;
     a.slot_base = f->d_slot_base;
-    a.items = f->d_items;
+    a.cta_first = f->d_cta_first;
+    a.recs = f->d_recs;
     a.expect = f->d_expect;
-    a.n_items = f->n_items;
     a.npart = f->d_npart;
     a.qpart = f->d_qpart;
     const size_t h = (size_t)plan->h;
     a.cnt_n = f->d_sync;
     a.cnt_q = f->d_sync + h;
-    a.flag_n = f->d_sync + 2 * h;
-    a.flag_q = f->d_sync + 3 * h;
-    a.done = f->d_sync + 4 * h;
+    a.done = f->d_sync + 2 * h;
+    a.flags = f->d_flags;
     a.status = plan->d_status;
     a.worker_norms = plan->d_worker_norms;
     a.scales = plan->d_scales;
-    a.qmul = plan->d_qmul;
-    a.dq = plan->d_dq;
-    a.step_a = plan->d_step_a;
     a.code_sum = identity ? nullptr : code_sum_out;
     a.norms_out = layer_norms_out;
     a.scales_out = identity ? nullptr : scales_out;
     a.h = (int)plan->h;
     a.M = plan->M;
+    a.nlead = f->nlead;
     a.epoch = f->epoch;
     a.S_f = (float)plan->S;
     a.SM_f = (float)((uint64_t)plan->S * (uint64_t)plan->M);
