@@ -127,10 +127,12 @@ struct RedDesc {
 #ifdef DAT_PROF
 // counters: 0 c.wait_full 1 n.wait 2 c.Q 3 c.U 4 n.work 5 r.work 6 p.wait_empty 7 p.wait_flag 8 p.issue 9 total
 #define PROF_T0() const long long prof_t0 = clock64()
-#define PROF_ADD(k) do { if (a.prof && (threadIdx.x & 31) == 0 && (threadIdx.x == 0 || threadIdx.x == F_CT || threadIdx.x >= F_CT + F_NT)) a.prof[blockIdx.x * 16 + (k)] += (unsigned long long)(clock64() - prof_t0); } while (0)
+#define PROF_ADD(k) do { if (a.prof && (threadIdx.x & 31) == 0 && (threadIdx.x == 0 || threadIdx.x == F_CT || threadIdx.x >= F_CT + F_NT)) sh.prof[(k)] += (unsigned long long)(clock64() - prof_t0); } while (0)
+#define PROF_LAYER(layer, col) do { if (a.prof) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); a.prof[296 * 16 + 2 * 4096 * 8 + (layer) * 4 + (col)] = t_; } } while (0)
 #define PROF_TRACE(role, idx, col, val) do { if (a.prof && blockIdx.x == 0 && (threadIdx.x & 31) == 0 && (idx) < 4096) a.prof[296 * 16 + ((role) * 4096 + (idx)) * 8 + (col)] = (unsigned long long)(val); } while (0)
 #else
 #define PROF_TRACE(role, idx, col, val) do {} while (0)
+#define PROF_LAYER(layer, col) do {} while (0)
 #define PROF_T0() do {} while (0)
 #define PROF_ADD(k) do {} while (0)
 #endif
@@ -173,6 +175,9 @@ struct Shared {
     double red_q[F_RED][F_CW][2];                // per-warp sums of theta^2 and m'^2 of one Q item
     double acc_n[DAT_MAX_WORKERS];               // the CTA's running sums for its current layer (reducer)
     double acc_q[2];
+#ifdef DAT_PROF
+    unsigned long long prof[16];
+#endif
     int q_pos;                                   // list position of the producer (throttles the norm warps)
     int n_issued;                                // passes the norm warps have started
     int abort_flag;
@@ -381,6 +386,7 @@ enum { NORM_ISSUED = 0, NORM_END = 1, NORM_LATER = 2, NORM_FAIL = 3 };
 __device__ __forceinline__ int norm_issue(const FusedArgs &a, Shared &sh, float *nbuf, NormWalk &w, uint32_t seq, int lane)
 {
     const uint32_t b = seq % F_NBUF, use = seq / F_NBUF;
+    PROF_T0();
     if (w.row0 < 0) {                            // next N item
         while (!w.have_item && w.pos < w.n) {
             if ((w.pos & ~31) != w.batch_base) {
@@ -403,10 +409,15 @@ __device__ __forceinline__ int norm_issue(const FusedArgs &a, Shared &sh, float 
         w.row0 = 0;
         w.have_item = false;
     }
+    PROF_ADD(10);
     const int rows = min(F_ROWS, a.M - w.row0);
     const bool last = (w.row0 + F_ROWS >= a.M);
     const bool fast = (w.item.flags & REC_FAST) != 0;
+    { PROF_T0();
     if (!wait_mbar(sh, &sh.nempty[b], (use & 1u) ^ 1u, a.status)) return NORM_FAIL;
+    PROF_ADD(12); }
+    {
+    PROF_T0();
     if (fast) {
         if (lane == 0) mbar_expect_tx(&sh.nfull[b], (uint32_t)rows * (FT * 4));
         __syncwarp();
@@ -426,6 +437,8 @@ __device__ __forceinline__ int norm_issue(const FusedArgs &a, Shared &sh, float 
     __syncwarp();
     if (lane == 0) mbar_arrive(&sh.nfull[b]);
     w.row0 = last ? -1 : w.row0 + F_ROWS;
+    PROF_ADD(11);
+    }
     return NORM_ISSUED;
 }
 
@@ -438,14 +451,15 @@ __device__ __forceinline__ void norm_rows(const float *buf, int rows, int nt, do
         acc[r] = 0.0;
         if (FULL || r < rows) {
             const float4 *g = reinterpret_cast<const float4 *>(buf + r * FT) + nt;
+            double part[FT / 4 / F_NT];                      // one short chain per 16-byte group
 #pragma unroll
             for (int k = 0; k < FT / 4 / F_NT; ++k) {
                 const float4 v = g[F_NT * k];
-                acc[r] = fma((double)v.x, (double)v.x, acc[r]);
-                acc[r] = fma((double)v.y, (double)v.y, acc[r]);
-                acc[r] = fma((double)v.z, (double)v.z, acc[r]);
-                acc[r] = fma((double)v.w, (double)v.w, acc[r]);
+                const double x = (double)v.x, y = (double)v.y, z = (double)v.z, w = (double)v.w;
+                part[k] = fma(w, w, fma(z, z, fma(y, y, x * x)));
             }
+            static_assert(FT / 4 / F_NT == 4, "four groups per thread and row");
+            acc[r] = (part[0] + part[1]) + (part[2] + part[3]);
         }
     }
 }
@@ -514,6 +528,7 @@ __device__ __forceinline__ void norm_warps(const FusedArgs &a, Shared &sh, float
     static_assert(F_ROWS == 4, "the cross-lane sum is written for four rows");
     const int nt = threadIdx.x - F_CT, lane = nt & 31, nw = nt >> 5;
     uint32_t nred = 0, consumed = 0;
+    PROF_T0();
     if (nw != 0) {
         // the second warp only takes the passes in order
         while (norm_consume(a, sh, nbuf, consumed, nred, nt)) ++consumed;
@@ -529,7 +544,9 @@ __device__ __forceinline__ void norm_warps(const FusedArgs &a, Shared &sh, float
             // throttle while a started pass has not been taken (its item may be what the
             // producer is waiting for)
             while (!ended && issued < consumed + F_NBUF) {
+                PROF_T0();
                 const int r = norm_issue(a, sh, nbuf, w, issued, lane);
+                PROF_ADD(14);
                 if (r == NORM_FAIL) return;
                 if (r == NORM_LATER) break;
                 issued++;
@@ -550,6 +567,7 @@ __device__ __forceinline__ void norm_warps(const FusedArgs &a, Shared &sh, float
             }
         }
     }
+    PROF_ADD(15);
     if (*(volatile int *)&sh.abort_flag) return;
     const uint32_t rb = nred % F_RED, ruse = nred / F_RED;
     if (!wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
@@ -586,6 +604,7 @@ __device__ __forceinline__ uint32_t producer(const FusedArgs &a, Shared &sh, flo
         item_bounds(a, item, lo, hi);
         if (type == ITEM_U && u_layer != item.layer) {
             // m' of this tile was written by the tile's Q item: the layer's result word orders it
+            if (blockIdx.x == 0 && lane == 0) PROF_LAYER(item.layer, 3);
             { PROF_T0();
             if (!wait_words(sh, a.flags + 3 * (long long)item.layer + 2, 1, a.epoch, a.status, u_f)) return issued;
             PROF_ADD(7); }
@@ -618,6 +637,7 @@ __device__ __forceinline__ uint32_t producer(const FusedArgs &a, Shared &sh, flo
             if (type == ITEM_Q && !IDENTITY && q_layer != item.layer) {
                 // every copy announced above has been started, so the stage completes even if
                 // this wait gives up
+                if (blockIdx.x == 0 && lane == 0) PROF_LAYER(item.layer, 2);
                 PROF_T0();
                 if (!wait_words(sh, a.flags + 3 * (long long)item.layer, 2, a.epoch, a.status, q_f)) {
                     if (lane == 0) sh.hdr[slot].kind = ITEM_END;      // nothing valid to consume in this stage
@@ -714,6 +734,7 @@ __device__ __forceinline__ void finish_norm(const FusedArgs &a, Shared &sh, int 
         const float dq = (nu == 0.0f) ? 0.0f : nu / a.SM_f;
         if (a.scales_out) a.scales_out[layer] = nu;
         if (bad) atomicOr(a.status, DAT_STATUS_NONFINITE);
+        PROF_LAYER(layer, 0);
         unsigned long long *w = a.flags + 3 * (long long)layer;
         st_release64(w, ((unsigned long long)a.epoch << 32) | __float_as_uint(qmul));
         st_release64(w + 1, ((unsigned long long)a.epoch << 32) | __float_as_uint(dq));
@@ -762,6 +783,7 @@ __device__ __forceinline__ void finish_quant(const FusedArgs &a, Shared &sh, int
         const float neg_a = -(a.lr * ratio);
         if (a.norms_out) { a.norms_out[2 * layer] = n_theta; a.norms_out[2 * layer + 1] = n_u; }
         if (!isfinite(n_theta) || !isfinite(n_u)) atomicOr(a.status, DAT_STATUS_NONFINITE);
+        PROF_LAYER(layer, 1);
         st_release64(a.flags + 3 * (long long)layer + 2, ((unsigned long long)a.epoch << 32) | __float_as_uint(neg_a));
     }
 }
@@ -966,7 +988,9 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
             if (e0 < hi && DAT_CHECK(lo >= 0 && hi <= a.d && e0 >= 0, 5, e0)) dat_store4(a.mom, e0, lo, hi, m);
             ss0 = dat_warp_sum(ss0);
             ss1 = dat_warp_sum(ss1);
+            { PROF_T0();
             if (!wait_mbar(sh, &sh.qred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
+            PROF_ADD(13); }
             if (lane == 0) { sh.red_q[rb][warp][0] = ss0; sh.red_q[rb][warp][1] = ss1; }
             if (ct == 0) {
                 sh.qdesc[rb].kind = ITEM_Q; sh.qdesc[rb].flush = hflush;
@@ -1014,6 +1038,9 @@ k_fused_step(const __grid_constant__ FusedArgs a)
         }
         for (int s = 0; s < F_STAGES; ++s) sh.hdr[s].kind = ITEM_END;
         for (int b = 0; b < F_NBUF; ++b) sh.nhdr[b].kind = ITEM_END;
+#ifdef DAT_PROF
+        for (int k = 0; k < 16; ++k) sh.prof[k] = 0;
+#endif
         sh.abort_flag = 0;
         sh.q_pos = 0;
         sh.n_issued = 0;
@@ -1030,8 +1057,11 @@ k_fused_step(const __grid_constant__ FusedArgs a)
     else if (warp < F_CW + F_NW) { if (!IDENTITY) norm_warps(a, sh, nbuf); }
     else if (warp == F_CW + F_NW) issued = producer<IDENTITY>(a, sh, stages);
     else reducer(a, sh, !IDENTITY);
-    __syncthreads();
     PROF_ADD(9);
+    __syncthreads();
+#ifdef DAT_PROF
+    if (a.prof && threadIdx.x < 16) a.prof[blockIdx.x * 16 + threadIdx.x] += sh.prof[threadIdx.x];
+#endif
 
     if (threadIdx.x == F_CT && !IDENTITY && *(volatile int *)&sh.abort_flag) {
         // after an abort the norm warps' last copies may still be in flight: wait (bounded) for the
