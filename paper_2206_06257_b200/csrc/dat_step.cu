@@ -40,13 +40,15 @@
 #define FT 1024                                  // elements per fused tile
 #define F_CW 8                                   // consumer warps (Q and U items)
 #define F_CT (F_CW * 32)                         // consumer threads; thread t owns elements 4t..4t+3
-#define F_NW 2                                   // norm warps (N items)
+#define F_NW 1                                   // norm issuer warp (walks the N items, starts their copies)
 #define F_NT (F_NW * 32)
 #define F_THREADS (F_CT + F_NT + 64)             // + one producer warp + one reducer warp
 #define F_ROWS 4                                 // worker rows per stage
 #define F_STAGES 3
 #define F_NBUF 2                                 // norm warps' own tile buffers (F_ROWS rows each)
-#define F_RED 2                                  // reduction hand-off buffers per group
+#define F_PREFETCH 6                             // N items whose gradient tiles are requested into L2 ahead of time
+#define F_RED 2                                  // hand-off buffers, consumers -> reducer, Q items
+#define F_REDN 1                                 // the same for N items (M values per warp: kept single to fit two CTAs per SM)
 #define F_NLEAD 6                                // default: list items the norm warps may run ahead of the producer
 #define F_CTAS_PER_SM 2
 #define F_STAGE_FLOATS ((F_ROWS + 2) * FT)       // gradient rows + theta row + momentum row
@@ -166,12 +168,12 @@ __device__ __noinline__ void dat_check_fail(const FusedArgs &a, int site, long l
 struct Shared {
     unsigned long long full[F_STAGES], empty[F_STAGES];
     unsigned long long nfull[F_NBUF], nempty[F_NBUF];         // norm warps' buffers
-    unsigned long long nred_full[F_RED], nred_empty[F_RED];   // norm warps -> reducer
+    unsigned long long nred_full[F_REDN], nred_empty[F_REDN]; // consumers -> reducer, N items
     unsigned long long qred_full[F_RED], qred_empty[F_RED];   // consumer warps -> reducer
     StageHdr hdr[F_STAGES];
     NormHdr nhdr[F_NBUF];
-    RedDesc ndesc[F_RED], qdesc[F_RED];
-    double red_n[F_RED][F_NW][DAT_MAX_WORKERS];  // per-warp sums of squares of one N item
+    RedDesc ndesc[F_REDN], qdesc[F_RED];
+    double red_n[F_REDN][F_CW][DAT_MAX_WORKERS];  // per-warp sums of squares of one N item
     double red_q[F_RED][F_CW][2];                // per-warp sums of theta^2 and m'^2 of one Q item
     double acc_n[DAT_MAX_WORKERS];               // the CTA's running sums for its current layer (reducer)
     double acc_q[2];
@@ -224,6 +226,11 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// Asks for `bytes` at `src` to be brought into L2 (no destination, no completion to wait for).
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
 {
@@ -374,6 +381,9 @@ struct NormWalk {
     int item_pos = 0;
     int row0 = -1;                               // next worker row of the item being cut into passes
     long long lo = 0, hi = 0;
+    int pf_pos = 0, pf_ahead = 0;                // L2 prefetch cursor: list position, N items it is ahead
+    uint4 pf_batch;
+    int pf_base = -1;
 };
 
 enum { NORM_ISSUED = 0, NORM_END = 1, NORM_LATER = 2, NORM_FAIL = 3 };
@@ -408,6 +418,24 @@ __device__ __forceinline__ int norm_issue(const FusedArgs &a, Shared &sh, float 
         item_bounds(a, w.item, w.lo, w.hi);
         w.row0 = 0;
         w.have_item = false;
+        // Hide the HBM latency behind L2: ask for the gradient tiles of the N items a few places
+        // further down the list now, so that their copies into shared memory find them in L2.
+        if (w.pf_pos < w.pos) { w.pf_pos = w.pos; w.pf_ahead = 0; }
+        w.pf_ahead--;
+        while (w.pf_ahead < F_PREFETCH && w.pf_pos < w.n) {
+            if ((w.pf_pos & ~31) != w.pf_base) {
+                w.pf_base = w.pf_pos & ~31;
+                w.pf_batch = (w.pf_base + lane < w.n) ? __ldg(a.recs + w.first + w.pf_base + lane) : make_uint4(ITEM_U, 0, 0, 0);
+            }
+            const uint4 r = shfl_rec(w.pf_batch, w.pf_pos & 31);
+            w.pf_pos++;
+            if ((r.x & 3u) != ITEM_N) continue;
+            w.pf_ahead++;
+            if (r.x & REC_FAST) {
+                const long long begin = (long long)(((unsigned long long)r.w << 32) | r.z);
+                for (int i = lane; i < a.M; i += 32) bulk_prefetch_l2(a.gp.p[i] + begin, FT * 4);
+            }
+        }
     }
     PROF_ADD(10);
     const int rows = min(F_ROWS, a.M - w.row0);
@@ -442,76 +470,71 @@ __device__ __forceinline__ int norm_issue(const FusedArgs &a, Shared &sh, float 
     return NORM_ISSUED;
 }
 
-// F_ROWS rows of a full tile from a norm buffer: thread nt owns the 16-byte groups nt + 64k.
+// F_ROWS rows of a full tile from a norm buffer: consumer thread ct owns the 16-byte group ct.
 template <bool FULL>
-__device__ __forceinline__ void norm_rows(const float *buf, int rows, int nt, double acc[F_ROWS])
+__device__ __forceinline__ void norm_rows(const float *buf, int rows, int ct, double acc[F_ROWS])
 {
 #pragma unroll
     for (int r = 0; r < F_ROWS; ++r) {
         acc[r] = 0.0;
         if (FULL || r < rows) {
-            const float4 *g = reinterpret_cast<const float4 *>(buf + r * FT) + nt;
-            double part[FT / 4 / F_NT];                      // one short chain per 16-byte group
-#pragma unroll
-            for (int k = 0; k < FT / 4 / F_NT; ++k) {
-                const float4 v = g[F_NT * k];
-                const double x = (double)v.x, y = (double)v.y, z = (double)v.z, w = (double)v.w;
-                part[k] = fma(w, w, fma(z, z, fma(y, y, x * x)));
-            }
-            static_assert(FT / 4 / F_NT == 4, "four groups per thread and row");
-            acc[r] = (part[0] + part[1]) + (part[2] + part[3]);
+            const float4 v = *(reinterpret_cast<const float4 *>(buf + r * FT) + ct);
+            const double x = (double)v.x, y = (double)v.y, z = (double)v.z, w = (double)v.w;
+            acc[r] = fma(w, w, fma(z, z, fma(y, y, x * x)));
         }
     }
 }
 
-// The same for a tile at a layer boundary: masked global loads, one group at a time.
+// The same for a tile at a layer boundary: masked global loads.
 __device__ __noinline__ void norm_rows_masked(const FusedArgs &a, int row0, int rows, long long begin, long long lo,
-                                               long long hi, int nt, double acc[F_ROWS])
+                                               long long hi, int ct, double acc[F_ROWS])
 {
 #pragma unroll 1
     for (int r = 0; r < F_ROWS; ++r) {
         double s = 0.0;
         if (r < rows) {
-            const float *__restrict__ g = a.gp.p[row0 + r];
-#pragma unroll 1
-            for (int k = 0; k < FT / 4 / F_NT; ++k) {
-                float v[4];
-                dat_load4(g, begin + 4 * (long long)(nt + F_NT * k), lo, hi, v);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) s = fma((double)v[j], (double)v[j], s);
-            }
+            float v[4];
+            dat_load4(a.gp.p[row0 + r], begin + 4 * (long long)ct, lo, hi, v);
+            s = fma((double)v[3], (double)v[3], fma((double)v[2], (double)v[2], fma((double)v[1], (double)v[1], (double)v[0] * (double)v[0])));
         }
         acc[r] = s;
     }
 }
 
-// One pass: both norm warps.  Returns false at the end marker or when a wait gave up.
-__device__ __forceinline__ bool norm_consume(const FusedArgs &a, Shared &sh, const float *nbuf, uint32_t seq,
-                                             uint32_t &nred, int nt)
+// One pass of the norm ring, taken by every consumer warp.  Returns 1 = pass done, 0 = end
+// marker, -1 = a wait gave up.  The caller has seen nfull[seq % F_NBUF] complete.
+__device__ __forceinline__ int norm_consume(const FusedArgs &a, Shared &sh, const float *nbuf, uint32_t seq,
+                                            uint32_t &nred, int ct)
 {
-    const int lane = nt & 31, nw = nt >> 5;
-    const uint32_t b = seq % F_NBUF, use = seq / F_NBUF;
-    if (!wait_mbar(sh, &sh.nfull[b], use & 1u, a.status)) return false;
+    static_assert(F_ROWS == 4, "the cross-lane sum is written for four rows");
+    const int lane = ct & 31, warp = ct >> 5;
+    const uint32_t b = seq % F_NBUF;
     PROF_T0();
     const NormHdr &H = sh.nhdr[b];
-    if (H.kind != ITEM_N) return false;
+    const uint32_t rb = nred % F_REDN, ruse = nred / F_REDN;
+    if (H.kind != ITEM_N) {
+        if (!wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return -1;
+        if (ct == 0) sh.ndesc[rb].kind = ITEM_END;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.nred_full[rb]);
+        return 0;
+    }
     const uint32_t flags = H.flags;
     const int row0 = H.row0, rows = min(F_ROWS, a.M - row0);
-    const uint32_t rb = nred % F_RED, ruse = nred / F_RED;
     double acc[F_ROWS];
-    if ((flags & HDR_FAST) && rows == F_ROWS) norm_rows<true>(nbuf + (size_t)b * F_NBUF_FLOATS, rows, nt, acc);
-    else if (flags & HDR_FAST) norm_rows<false>(nbuf + (size_t)b * F_NBUF_FLOATS, rows, nt, acc);
-    else norm_rows_masked(a, row0, rows, H.begin, H.lo, H.hi, nt, acc);
+    if ((flags & HDR_FAST) && rows == F_ROWS) norm_rows<true>(nbuf + (size_t)b * F_NBUF_FLOATS, rows, ct, acc);
+    else if (flags & HDR_FAST) norm_rows<false>(nbuf + (size_t)b * F_NBUF_FLOATS, rows, ct, acc);
+    else norm_rows_masked(a, row0, rows, H.begin, H.lo, H.hi, ct, acc);
     const int layer = H.layer;
     const long long slot = H.slot;
     __syncwarp();
     if (lane == 0) mbar_arrive(&sh.nempty[b]);
     // the item's first pass claims a hand-off buffer
-    if (row0 == 0 && !wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return false;
+    if (row0 == 0 && !wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return -1;
     const double s = warp_sum4(acc, lane);
-    if ((lane & 7) == 0 && (lane >> 3) < rows) sh.red_n[rb][nw][row0 + (lane >> 3)] = s;
+    if ((lane & 7) == 0 && (lane >> 3) < rows) sh.red_n[rb][warp][row0 + (lane >> 3)] = s;
     if (flags & HDR_LAST_CHUNK) {
-        if (nt == 0) {
+        if (ct == 0) {
             sh.ndesc[rb].kind = ITEM_N; sh.ndesc[rb].flush = flags & HDR_FLUSH;
             sh.ndesc[rb].layer = layer; sh.ndesc[rb].slot = slot;
         }
@@ -519,61 +542,31 @@ __device__ __forceinline__ bool norm_consume(const FusedArgs &a, Shared &sh, con
         if (lane == 0) mbar_arrive(&sh.nred_full[rb]);
         nred++;
     }
-    PROF_ADD(4);
-    return true;
+    PROF_ADD(1);
+    return 1;
 }
 
-__device__ __forceinline__ void norm_warps(const FusedArgs &a, Shared &sh, float *nbuf)
+// The norm issuer warp: walks the CTA's N items and keeps the norm buffers filled, staying
+// within `nlead` list items of the producer.
+__device__ __forceinline__ void norm_issuer(const FusedArgs &a, Shared &sh, float *nbuf)
 {
-    static_assert(F_ROWS == 4, "the cross-lane sum is written for four rows");
-    const int nt = threadIdx.x - F_CT, lane = nt & 31, nw = nt >> 5;
-    uint32_t nred = 0, consumed = 0;
-    PROF_T0();
-    if (nw != 0) {
-        // the second warp only takes the passes in order
-        while (norm_consume(a, sh, nbuf, consumed, nred, nt)) ++consumed;
-    } else {
-        NormWalk w;
-        w.first = __ldg(a.cta_first + blockIdx.x);
-        w.n = __ldg(a.cta_first + blockIdx.x + 1) - w.first;
-        uint32_t issued = 0;
-        bool ended = false;
-        long long t_idle = 0;
-        for (;;) {
-            // start as many passes as the buffers and the throttle allow; never wait for the
-            // throttle while a started pass has not been taken (its item may be what the
-            // producer is waiting for)
-            while (!ended && issued < consumed + F_NBUF) {
-                PROF_T0();
-                const int r = norm_issue(a, sh, nbuf, w, issued, lane);
-                PROF_ADD(14);
-                if (r == NORM_FAIL) return;
-                if (r == NORM_LATER) break;
-                issued++;
-                ended = (r == NORM_END);
-            }
-            if (consumed < issued) {
-                if (!norm_consume(a, sh, nbuf, consumed, nred, nt)) break;
-                ++consumed;
-                t_idle = 0;
-            } else {
-                // nothing in flight and the next item is still ahead of the producer
-                PROF_T0();
-                if (t_idle == 0) t_idle = clock64();
-                __nanosleep(64);
-                if (*(volatile int *)&sh.abort_flag) return;
-                if (clock64() - t_idle > F_WAIT_CYCLES) { raise_timeout(sh, a.status); return; }
-                PROF_ADD(1);
-            }
-        }
+    const int lane = threadIdx.x & 31;
+    NormWalk w;
+    w.first = __ldg(a.cta_first + blockIdx.x);
+    w.n = __ldg(a.cta_first + blockIdx.x + 1) - w.first;
+    long long t_idle = 0;
+    for (uint32_t seq = 0;;) {
+        const int r = norm_issue(a, sh, nbuf, w, seq, lane);
+        if (r == NORM_FAIL || r == NORM_END) return;
+        if (r == NORM_ISSUED) { ++seq; t_idle = 0; continue; }
+        // the next item is still too far ahead of the producer
+        PROF_T0();
+        if (t_idle == 0) t_idle = clock64();
+        __nanosleep(64);
+        if (*(volatile int *)&sh.abort_flag) return;
+        if (clock64() - t_idle > F_WAIT_CYCLES) { raise_timeout(sh, a.status); return; }
+        PROF_ADD(4);
     }
-    PROF_ADD(15);
-    if (*(volatile int *)&sh.abort_flag) return;
-    const uint32_t rb = nred % F_RED, ruse = nred / F_RED;
-    if (!wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
-    if (nt == 0) sh.ndesc[rb].kind = ITEM_END;
-    __syncwarp();
-    if (lane == 0) mbar_arrive(&sh.nred_full[rb]);
 }
 
 // ---- producer warp -------------------------------------------------------------------------------
@@ -684,7 +677,7 @@ __device__ __forceinline__ void finish_norm(const FusedArgs &a, Shared &sh, int 
     for (int i = lane; i < a.M; i += 32) {
         double s = sh.acc_n[i];
 #pragma unroll
-        for (int w = 0; w < F_NW; ++w) s += sh.red_n[buf][w][i];
+        for (int w = 0; w < F_CW; ++w) s += sh.red_n[buf][w][i];
         sh.acc_n[i] = s;
     }
     __syncwarp();
@@ -798,8 +791,8 @@ __device__ __forceinline__ void reducer(const FusedArgs &a, Shared &sh, bool hav
     while (!(done_n && done_q)) {
         bool progress = false;
         if (!done_n) {
-            const uint32_t b = kn % F_RED;
-            if (mbar_test_wait(&sh.nred_full[b], (kn / F_RED) & 1u)) {
+            const uint32_t b = kn % F_REDN;
+            if (mbar_test_wait(&sh.nred_full[b], (kn / F_REDN) & 1u)) {
                 PROF_T0();
                 if (sh.ndesc[b].kind == ITEM_END) done_n = true;
                 else {
@@ -904,19 +897,39 @@ __device__ __noinline__ void rows_quant_masked(const FusedArgs &a, int chunk, in
 // needs to know comes from its header, so the consumers touch global memory only for the
 // results (and for the masked loads of boundary tiles).
 template <bool IDENTITY>
-__device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const float *stages)
+__device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const float *stages, const float *nbuf)
 {
     const int ct = threadIdx.x, lane = ct & 31, warp = ct >> 5;
-    uint32_t taken = 0, nred = 0;
+    uint32_t taken = 0, nred = 0;                // stage ring, its hand-offs
+    uint32_t nseq = 0, nred_n = 0;               // norm ring, its hand-offs
+    bool n_done = IDENTITY, q_done = false;
     int sum[4] = {0, 0, 0, 0};
     float facc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     const float Mf = (float)a.M;
     for (;;) {
         const uint32_t slot = taken % F_STAGES, use = taken / F_STAGES;
         if (threadIdx.x == 0) PROF_TRACE(0, taken, 0, clock64());
+        // take whatever is ready, a norm pass first (other CTAs' flags wait for those)
+        int pick = -1;
         { PROF_T0();
-        if (!wait_mbar(sh, &sh.full[slot], use & 1u, a.status)) return;
+        long long t0 = 0;
+        for (uint32_t spins = 1;; ++spins) {
+            if (!n_done && mbar_test_wait(&sh.nfull[nseq % F_NBUF], (nseq / F_NBUF) & 1u)) { pick = 0; break; }
+            if (!q_done && mbar_test_wait(&sh.full[slot], use & 1u)) { pick = 1; break; }
+            if (n_done && q_done) return;
+            if ((spins & 63u) == 0u) {
+                if (*(volatile int *)&sh.abort_flag) return;
+                if (t0 == 0) t0 = clock64();
+                else if (clock64() - t0 > F_WAIT_CYCLES) { raise_timeout(sh, a.status); return; }
+            }
+        }
         PROF_ADD(0); }
+        if (pick == 0) {
+            const int r = norm_consume(a, sh, nbuf, nseq, nred_n, ct);
+            if (r < 0) return;
+            if (r == 0) n_done = true; else ++nseq;
+            continue;
+        }
         PROF_T0();
         const StageHdr &H = sh.hdr[slot];
         const uint32_t kind = H.kind;
@@ -928,7 +941,8 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
             if (ct == 0) sh.qdesc[rb].kind = ITEM_END;
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.qred_full[rb]);
-            return;
+            q_done = true;
+            continue;
         }
         const uint32_t flags = H.flags;
         const bool fast = flags & HDR_FAST, last_chunk = flags & HDR_LAST_CHUNK;
@@ -1031,11 +1045,9 @@ k_fused_step(const __grid_constant__ FusedArgs a)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < F_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], F_CW); }
-        for (int b = 0; b < F_NBUF; ++b) { mbar_init(&sh.nfull[b], 1); mbar_init(&sh.nempty[b], F_NW); }
-        for (int b = 0; b < F_RED; ++b) {
-            mbar_init(&sh.nred_full[b], F_NW); mbar_init(&sh.nred_empty[b], 1);
-            mbar_init(&sh.qred_full[b], F_CW); mbar_init(&sh.qred_empty[b], 1);
-        }
+        for (int b = 0; b < F_NBUF; ++b) { mbar_init(&sh.nfull[b], 1); mbar_init(&sh.nempty[b], F_CW); }
+        for (int b = 0; b < F_REDN; ++b) { mbar_init(&sh.nred_full[b], F_CW); mbar_init(&sh.nred_empty[b], 1); }
+        for (int b = 0; b < F_RED; ++b) { mbar_init(&sh.qred_full[b], F_CW); mbar_init(&sh.qred_empty[b], 1); }
         for (int s = 0; s < F_STAGES; ++s) sh.hdr[s].kind = ITEM_END;
         for (int b = 0; b < F_NBUF; ++b) sh.nhdr[b].kind = ITEM_END;
 #ifdef DAT_PROF
@@ -1053,8 +1065,8 @@ k_fused_step(const __grid_constant__ FusedArgs a)
     PROF_T0();
     uint32_t issued = 0;
     const int warp = threadIdx.x >> 5;
-    if (warp < F_CW) consumer<IDENTITY>(a, sh, stages);
-    else if (warp < F_CW + F_NW) { if (!IDENTITY) norm_warps(a, sh, nbuf); }
+    if (warp < F_CW) consumer<IDENTITY>(a, sh, stages, nbuf);
+    else if (warp < F_CW + F_NW) { if (!IDENTITY) norm_issuer(a, sh, nbuf); }
     else if (warp == F_CW + F_NW) issued = producer<IDENTITY>(a, sh, stages);
     else reducer(a, sh, !IDENTITY);
     PROF_ADD(9);
