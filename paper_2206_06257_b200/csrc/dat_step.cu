@@ -44,9 +44,8 @@
 #define F_NT (F_NW * 32)
 #define F_THREADS (F_CT + F_NT + 64)             // + one producer warp + one reducer warp
 #define F_ROWS 4                                 // worker rows per stage
-#define F_STAGES 3
-#define F_NBUF 2                                 // norm warps' own tile buffers (F_ROWS rows each)
-#define F_PREFETCH 6                             // N items whose gradient tiles are requested into L2 ahead of time
+#define F_STAGES 2
+#define F_NBUF 3                                 // norm warps' own tile buffers (F_ROWS rows each)
 #define F_RED 2                                  // hand-off buffers, consumers -> reducer, Q items
 #define F_REDN 1                                 // the same for N items (M values per warp: kept single to fit two CTAs per SM)
 #define F_NLEAD 6                                // default: list items the norm warps may run ahead of the producer
@@ -227,11 +226,6 @@ __device__ __forceinline__ void bulk_g2s(void *dst, const void *src, uint32_t by
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
-// Asks for `bytes` at `src` to be brought into L2 (no destination, no completion to wait for).
-__device__ __forceinline__ void bulk_prefetch_l2(const void *src, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
 {
     uint32_t v;
@@ -381,9 +375,6 @@ struct NormWalk {
     int item_pos = 0;
     int row0 = -1;                               // next worker row of the item being cut into passes
     long long lo = 0, hi = 0;
-    int pf_pos = 0, pf_ahead = 0;                // L2 prefetch cursor: list position, N items it is ahead
-    uint4 pf_batch;
-    int pf_base = -1;
 };
 
 enum { NORM_ISSUED = 0, NORM_END = 1, NORM_LATER = 2, NORM_FAIL = 3 };
@@ -418,24 +409,6 @@ __device__ __forceinline__ int norm_issue(const FusedArgs &a, Shared &sh, float 
         item_bounds(a, w.item, w.lo, w.hi);
         w.row0 = 0;
         w.have_item = false;
-        // Hide the HBM latency behind L2: ask for the gradient tiles of the N items a few places
-        // further down the list now, so that their copies into shared memory find them in L2.
-        if (w.pf_pos < w.pos) { w.pf_pos = w.pos; w.pf_ahead = 0; }
-        w.pf_ahead--;
-        while (w.pf_ahead < F_PREFETCH && w.pf_pos < w.n) {
-            if ((w.pf_pos & ~31) != w.pf_base) {
-                w.pf_base = w.pf_pos & ~31;
-                w.pf_batch = (w.pf_base + lane < w.n) ? __ldg(a.recs + w.first + w.pf_base + lane) : make_uint4(ITEM_U, 0, 0, 0);
-            }
-            const uint4 r = shfl_rec(w.pf_batch, w.pf_pos & 31);
-            w.pf_pos++;
-            if ((r.x & 3u) != ITEM_N) continue;
-            w.pf_ahead++;
-            if (r.x & REC_FAST) {
-                const long long begin = (long long)(((unsigned long long)r.w << 32) | r.z);
-                for (int i = lane; i < a.M; i += 32) bulk_prefetch_l2(a.gp.p[i] + begin, FT * 4);
-            }
-        }
     }
     PROF_ADD(10);
     const int rows = min(F_ROWS, a.M - w.row0);
@@ -917,6 +890,7 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
             if (!n_done && mbar_test_wait(&sh.nfull[nseq % F_NBUF], (nseq / F_NBUF) & 1u)) { pick = 0; break; }
             if (!q_done && mbar_test_wait(&sh.full[slot], use & 1u)) { pick = 1; break; }
             if (n_done && q_done) return;
+            __nanosleep(32);
             if ((spins & 63u) == 0u) {
                 if (*(volatile int *)&sh.abort_flag) return;
                 if (t0 == 0) t0 = clock64();
