@@ -232,6 +232,10 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+__device__ __forceinline__ void red_add(uint32_t *p)
+{
+    asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
+}
 __device__ __forceinline__ void st_release(uint32_t *p, uint32_t v)
 {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -659,14 +663,14 @@ __device__ __forceinline__ void finish_norm(const FusedArgs &a, Shared &sh, int 
     for (int i = lane; i < a.M; i += 32) { a.npart[slot * a.M + i] = sh.acc_n[i]; sh.acc_n[i] = 0.0; }
     __threadfence();
     __syncwarp();
-    uint32_t last = 0;
-    if (lane == 0) {
-        const uint32_t old = atomicAdd(a.cnt_n + layer, 1u);
-        last = (old == __ldg(a.expect + layer) - 1u);
-        if (last) { a.cnt_n[layer] = 0u; __threadfence(); }
-    }
-    last = __shfl_sync(0xFFFFFFFFu, last, 0);
-    if (!last) return;
+    if (lane == 0) red_add(a.cnt_n + layer);      // no answer needed: the layer's owner watches the count
+}
+
+// The owner of a layer (CTA layer mod G) finalises it once every contribution has arrived:
+// all contributions are reduced in a fixed order and the layer's scale is published.
+__device__ __forceinline__ void finalize_norm(const FusedArgs &a, int layer, int lane)
+{
+    if (lane == 0) a.cnt_n[layer] = 0u;           // ready for the next call
     const long long s0 = __ldg(a.slot_base + layer);
     const int ns = (int)(__ldg(a.slot_base + layer + 1) - s0);
     // Every lane sums its slots (lane, lane+32, ...) in order, eight workers at a time so that many
@@ -723,14 +727,12 @@ __device__ __forceinline__ void finish_quant(const FusedArgs &a, Shared &sh, int
     if (lane < 2) { a.qpart[slot * 2 + lane] = sh.acc_q[lane]; sh.acc_q[lane] = 0.0; }
     __threadfence();
     __syncwarp();
-    uint32_t last = 0;
-    if (lane == 0) {
-        const uint32_t old = atomicAdd(a.cnt_q + layer, 1u);
-        last = (old == __ldg(a.expect + a.h + layer) - 1u);
-        if (last) { a.cnt_q[layer] = 0u; __threadfence(); }
-    }
-    last = __shfl_sync(0xFFFFFFFFu, last, 0);
-    if (!last) return;
+    if (lane == 0) red_add(a.cnt_q + layer);
+}
+
+__device__ __forceinline__ void finalize_quant(const FusedArgs &a, int layer, int lane)
+{
+    if (lane == 0) a.cnt_q[layer] = 0u;
     const long long s0 = __ldg(a.slot_base + layer);
     const int ns = (int)(__ldg(a.slot_base + layer + 1) - s0);
     double x = 0.0, y = 0.0;
@@ -754,14 +756,20 @@ __device__ __forceinline__ void finish_quant(const FusedArgs &a, Shared &sh, int
     }
 }
 
-// Serves both hand-off rings in turn (non-blocking tests), until both groups have said END.
-__device__ __forceinline__ void reducer(const FusedArgs &a, Shared &sh, bool have_norm_warps)
+// Serves both hand-off rings in turn (non-blocking tests) and finalises the layers this CTA owns
+// (layer mod G == CTA) as their contribution counts fill up, until both rings have said END and
+// every owned layer is done.
+__device__ __forceinline__ void reducer(const FusedArgs &a, Shared &sh, bool have_norm)
 {
     const int lane = threadIdx.x & 31;
     uint32_t kn = 0, kq = 0;
-    bool done_n = !have_norm_warps, done_q = false;
+    bool done_n = !have_norm, done_q = false;
+    int own_n = have_norm ? (int)blockIdx.x : a.h, own_q = (int)blockIdx.x;     // next owned layer to finalise
+    uint32_t want_n = (own_n < a.h) ? __ldg(a.expect + own_n) : 0u;
+    uint32_t want_q = (own_q < a.h) ? __ldg(a.expect + a.h + own_q) : 0u;
     long long t_last = clock64();
-    while (!(done_n && done_q)) {
+    uint32_t round = 0;
+    while (!(done_n && done_q) || own_n < a.h || own_q < a.h) {
         bool progress = false;
         if (!done_n) {
             const uint32_t b = kn % F_REDN;
@@ -793,12 +801,31 @@ __device__ __forceinline__ void reducer(const FusedArgs &a, Shared &sh, bool hav
                 PROF_ADD(5);
             }
         }
+        // owned layers: look at the counts when idle, and every few rounds when busy
+        if (!progress || (++round & 3u) == 0u) {
+            if (own_n < a.h && ld_acquire(a.cnt_n + own_n) == want_n) {
+                PROF_T0();
+                finalize_norm(a, own_n, lane);
+                own_n += (int)gridDim.x;
+                want_n = (own_n < a.h) ? __ldg(a.expect + own_n) : 0u;
+                progress = true;
+                PROF_ADD(5);
+            }
+            if (own_q < a.h && ld_acquire(a.cnt_q + own_q) == want_q) {
+                PROF_T0();
+                finalize_quant(a, own_q, lane);
+                own_q += (int)gridDim.x;
+                want_q = (own_q < a.h) ? __ldg(a.expect + a.h + own_q) : 0u;
+                progress = true;
+                PROF_ADD(5);
+            }
+        }
         if (progress) {
             t_last = clock64();
         } else {
-            if (*(volatile int *)&sh.abort_flag) return;
+            if (*(volatile int *)&sh.abort_flag || (ld_acquire(a.status) & DAT_STATUS_TIMEOUT)) { atomicExch(&sh.abort_flag, 1); return; }
             if (clock64() - t_last > F_WAIT_CYCLES) { raise_timeout(sh, a.status); return; }
-            __nanosleep(20);
+            __nanosleep(40);
         }
     }
 }
