@@ -48,7 +48,7 @@
 #define F_NBUF 3                                 // norm warps' own tile buffers (F_ROWS rows each)
 #define F_RED 2                                  // hand-off buffers, consumers -> reducer, Q items
 #define F_REDN 1                                 // the same for N items (M values per warp: kept single to fit two CTAs per SM)
-#define F_NLEAD 6                                // default: list items the norm warps may run ahead of the producer
+#define F_NLEAD 24                               // default: list items the norm warps may run ahead of the producer
 #define F_CTAS_PER_SM 2
 #define F_STAGE_FLOATS ((F_ROWS + 2) * FT)       // gradient rows + theta row + momentum row
 #define F_STAGE_BYTES (F_STAGE_FLOATS * 4)
@@ -481,7 +481,7 @@ __device__ __noinline__ void norm_rows_masked(const FusedArgs &a, int row0, int 
 // One pass of the norm ring, taken by every consumer warp.  Returns 1 = pass done, 0 = end
 // marker, -1 = a wait gave up.  The caller has seen nfull[seq % F_NBUF] complete.
 __device__ __forceinline__ int norm_consume(const FusedArgs &a, Shared &sh, const float *nbuf, uint32_t seq,
-                                            uint32_t &nred, int ct)
+                                            uint32_t &nred, int ct, double nacc[2 * F_ROWS])
 {
     static_assert(F_ROWS == 4, "the cross-lane sum is written for four rows");
     const int lane = ct & 31, warp = ct >> 5;
@@ -506,18 +506,45 @@ __device__ __forceinline__ int norm_consume(const FusedArgs &a, Shared &sh, cons
     const long long slot = H.slot;
     __syncwarp();
     if (lane == 0) mbar_arrive(&sh.nempty[b]);
-    // the item's first pass claims a hand-off buffer
-    if (row0 == 0 && !wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return -1;
-    const double s = warp_sum4(acc, lane);
-    if ((lane & 7) == 0 && (lane >> 3) < rows) sh.red_n[rb][warp][row0 + (lane >> 3)] = s;
-    if (flags & HDR_LAST_CHUNK) {
-        if (ct == 0) {
-            sh.ndesc[rb].kind = ITEM_N; sh.ndesc[rb].flush = flags & HDR_FLUSH;
-            sh.ndesc[rb].layer = layer; sh.ndesc[rb].slot = slot;
+    const bool last = (flags & HDR_LAST_CHUNK) != 0;
+    if (a.M <= 2 * F_ROWS) {
+        // Few workers: every thread keeps its own running sums over the CTA's tiles of the layer
+        // and they are reduced across lanes only when the CTA's contribution is due.
+        if (row0 == 0) {
+#pragma unroll
+            for (int r = 0; r < F_ROWS; ++r) nacc[r] += acc[r];
+        } else {
+#pragma unroll
+            for (int r = 0; r < F_ROWS; ++r) nacc[F_ROWS + r] += acc[r];
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.nred_full[rb]);
-        nred++;
+        if (last && (flags & HDR_FLUSH)) {
+            if (!wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return -1;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const double s = warp_sum4(nacc + half * F_ROWS, lane);
+                if ((lane & 7) == 0 && half * F_ROWS + (lane >> 3) < a.M) sh.red_n[rb][warp][half * F_ROWS + (lane >> 3)] = s;
+            }
+#pragma unroll
+            for (int r = 0; r < 2 * F_ROWS; ++r) nacc[r] = 0.0;
+            if (ct == 0) { sh.ndesc[rb].kind = ITEM_N; sh.ndesc[rb].flush = 1u; sh.ndesc[rb].layer = layer; sh.ndesc[rb].slot = slot; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.nred_full[rb]);
+            nred++;
+        }
+    } else {
+        // the item's first pass claims a hand-off buffer
+        if (row0 == 0 && !wait_mbar(sh, &sh.nred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return -1;
+        const double s = warp_sum4(acc, lane);
+        if ((lane & 7) == 0 && (lane >> 3) < rows) sh.red_n[rb][warp][row0 + (lane >> 3)] = s;
+        if (last) {
+            if (ct == 0) {
+                sh.ndesc[rb].kind = ITEM_N; sh.ndesc[rb].flush = flags & HDR_FLUSH;
+                sh.ndesc[rb].layer = layer; sh.ndesc[rb].slot = slot;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.nred_full[rb]);
+            nred++;
+        }
     }
     PROF_ADD(1);
     return 1;
@@ -903,6 +930,8 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
     uint32_t taken = 0, nred = 0;                // stage ring, its hand-offs
     uint32_t nseq = 0, nred_n = 0;               // norm ring, its hand-offs
     bool n_done = IDENTITY, q_done = false;
+    double nacc[2 * F_ROWS] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};     // running sums of squares (M <= 8)
+    double qss0 = 0.0, qss1 = 0.0;               // running sums of theta^2 and m'^2 until the next flush
     int sum[4] = {0, 0, 0, 0};
     float facc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     const float Mf = (float)a.M;
@@ -926,7 +955,7 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
         }
         PROF_ADD(0); }
         if (pick == 0) {
-            const int r = norm_consume(a, sh, nbuf, nseq, nred_n, ct);
+            const int r = norm_consume(a, sh, nbuf, nseq, nred_n, ct, nacc);
             if (r < 0) return;
             if (r == 0) n_done = true; else ++nseq;
             continue;
@@ -993,27 +1022,30 @@ __device__ __forceinline__ void consumer(const FusedArgs &a, Shared &sh, const f
 #pragma unroll
                 for (int j = 0; j < 4; ++j) ghat[j] = (float)sum[j] * f1;
             }
-            double ss0 = 0.0, ss1 = 0.0;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 m[j] = __fmaf_rn(a.mu, m[j], __fmaf_rn(a.wd, th[j], ghat[j]));
-                ss0 = fma((double)th[j], (double)th[j], ss0);
-                ss1 = fma((double)m[j], (double)m[j], ss1);
+                qss0 = fma((double)th[j], (double)th[j], qss0);
+                qss1 = fma((double)m[j], (double)m[j], qss1);
             }
             if (e0 < hi && DAT_CHECK(lo >= 0 && hi <= a.d && e0 >= 0, 5, e0)) dat_store4(a.mom, e0, lo, hi, m);
-            ss0 = dat_warp_sum(ss0);
-            ss1 = dat_warp_sum(ss1);
-            { PROF_T0();
-            if (!wait_mbar(sh, &sh.qred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
-            PROF_ADD(13); }
-            if (lane == 0) { sh.red_q[rb][warp][0] = ss0; sh.red_q[rb][warp][1] = ss1; }
-            if (ct == 0) {
-                sh.qdesc[rb].kind = ITEM_Q; sh.qdesc[rb].flush = hflush;
-                sh.qdesc[rb].layer = hlayer; sh.qdesc[rb].slot = hslot;
+            if (hflush) {
+                // the CTA's contribution to the layer is due: reduce across lanes and hand over
+                const double ss0 = dat_warp_sum(qss0), ss1 = dat_warp_sum(qss1);
+                qss0 = 0.0;
+                qss1 = 0.0;
+                { PROF_T0();
+                if (!wait_mbar(sh, &sh.qred_empty[rb], (ruse & 1u) ^ 1u, a.status)) return;
+                PROF_ADD(13); }
+                if (lane == 0) { sh.red_q[rb][warp][0] = ss0; sh.red_q[rb][warp][1] = ss1; }
+                if (ct == 0) {
+                    sh.qdesc[rb].kind = ITEM_Q; sh.qdesc[rb].flush = 1u;
+                    sh.qdesc[rb].layer = hlayer; sh.qdesc[rb].slot = hslot;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.qred_full[rb]);
+                nred++;
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.qred_full[rb]);
-            nred++;
             PROF_ADD(2);
         } else {
             float th[4], m[4];
@@ -1177,7 +1209,7 @@ static int fused_prepare(dat_plan_t *plan)
     int l2 = 0;
     cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, plan->device);
     f->window_bytes = l2 > 0 ? (int64_t)l2 / 10 * 7 : (int64_t)32 << 20;
-    f->slack = 2 * (int64_t)G;
+    f->slack = 8 * (int64_t)G;
 #ifdef DAT_PROF
     if (const char *e = getenv("DAT_FUSED_WINDOW_MB")) f->window_bytes = (int64_t)atoi(e) << 20;
     if (const char *e = getenv("DAT_FUSED_SLACK")) f->slack = atoi(e);
