@@ -48,7 +48,7 @@
 #define F_NBUF 3                                 // norm warps' own tile buffers (F_ROWS rows each)
 #define F_RED 2                                  // hand-off buffers, consumers -> reducer, Q items
 #define F_REDN 1                                 // the same for N items (M values per warp: kept single to fit two CTAs per SM)
-#define F_NLEAD 24                               // default: list items the norm warps may run ahead of the producer
+#define F_NLEAD 12                               // default: list items the norm warps may run ahead of the producer
 #define F_CTAS_PER_SM 2
 #define F_STAGE_FLOATS ((F_ROWS + 2) * FT)       // gradient rows + theta row + momentum row
 #define F_STAGE_BYTES (F_STAGE_FLOATS * 4)
@@ -1209,7 +1209,7 @@ static int fused_prepare(dat_plan_t *plan)
     int l2 = 0;
     cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, plan->device);
     f->window_bytes = l2 > 0 ? (int64_t)l2 / 10 * 7 : (int64_t)32 << 20;
-    f->slack = 8 * (int64_t)G;
+    f->slack = 4 * (int64_t)G;
 #ifdef DAT_PROF
     if (const char *e = getenv("DAT_FUSED_WINDOW_MB")) f->window_bytes = (int64_t)atoi(e) << 20;
     if (const char *e = getenv("DAT_FUSED_SLACK")) f->slack = atoi(e);
