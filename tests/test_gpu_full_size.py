@@ -1,0 +1,92 @@
+"""Parity at the full sizes of the workloads, in the launch configuration bench.py times
+(fused dat_step, inputs generated on the device).  The oracle recomputes sampled layers one by
+one (its window mode keeps the global element index, hence the same random stream); properties
+that hold at any size are checked on everything."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import assert_close_per_layer, hp_tuple, np_of, ulp_diff
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_and_check(oracle, cfg, sample_layers, step=0):
+    from paper_2206_06257_b200 import api, synth
+    dev = "cuda"
+    theta, mom = synth.make_params(cfg, device=dev)
+    grads = synth.make_grads(cfg, step, device=dev)
+    hp = hp_tuple(cfg)
+    th0, mo0 = theta.clone(), mom.clone()
+    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits)
+    try:
+        cs = torch.zeros(cfg.d, dtype=torch.int32, device=dev)
+        sc = torch.zeros(cfg.h, dtype=torch.float32, device=dev)
+        norms = torch.zeros(2 * cfg.h, dtype=torch.float32, device=dev)
+        api.dat_step(plan, theta, mom, grads, cfg.seed, step, hp, cs, norms, sc)
+        torch.cuda.synchronize()
+        assert api.dat_get_status(plan) == 0
+    finally:
+        api.dat_plan_destroy(plan)
+    offs = cfg.offsets
+    S = 2 ** cfg.bits - 1
+    # properties at any size
+    assert torch.isfinite(theta).all() and torch.isfinite(mom).all()
+    assert int(cs.abs().max()) <= cfg.M * S
+    norms_h = np_of(norms).reshape(-1, 2)
+    d64 = (theta.double() - th0.double()) ** 2
+    csum = torch.cat([torch.zeros(1, dtype=torch.float64, device=dev), torch.cumsum(d64, 0)])
+    idx = torch.from_numpy(offs).to(dev)
+    step_len = torch.sqrt((csum[idx[1:]] - csum[idx[:-1]]).clamp_min(0)).cpu().numpy()
+    for l in range(cfg.h):
+        tau = min(max(float(norms_h[l, 0]), cfg.c_l), cfg.c_u)
+        expect = cfg.lr * tau if norms_h[l, 1] != 0 else 0.0
+        # (the prefix-sum difference leaves ~1e-7 of cancellation noise on zero-step layers)
+        assert abs(step_len[l] - expect) <= 1e-4 * expect + 1e-6, (l, step_len[l], expect)
+    # sampled layers, element by element
+    sc_h = np_of(sc)
+    for l in sample_layers:
+        a, b = int(offs[l]), int(offs[l + 1])
+        g_l = [np_of(g[a:b]) for g in grads]
+        ref = oracle.step(offs, np_of(th0[a:b]), np_of(mo0[a:b]), g_l, cfg.bits, cfg.seed, step, *hp,
+                          l0=l, l1=l + 1, window=True)
+        assert ulp_diff(sc_h[l:l + 1], ref["scales"][l:l + 1]).max() <= 1
+        if sc_h[l] != ref["scales"][l]:
+            ref = oracle.step(offs, np_of(th0[a:b]), np_of(mo0[a:b]), g_l, cfg.bits, cfg.seed, step, *hp,
+                              l0=l, l1=l + 1, window=True, scales_in=sc_h)
+        assert np.array_equal(np_of(cs[a:b]), ref["code_sum"]), "layer %d code sums" % l
+        assert np.array_equal(np_of(mom[a:b]).view(np.uint32), ref["mom"].view(np.uint32)), "layer %d momentum" % l
+        assert_close_per_layer(np_of(theta[a:b]), ref["theta"], np.array([0, b - a]), "theta layer %d" % l)
+    return theta, mom
+
+
+def test_resnet50_bench_configuration_every_layer(oracle):
+    from paper_2206_06257_b200 import synth
+    cfg = synth.config("resnet50")
+    _run_and_check(oracle, cfg, range(cfg.h))
+
+
+def test_resnet50_m32_b4_student_t_with_zero_layers(oracle):
+    from paper_2206_06257_b200 import synth
+    cfg = synth.config("resnet50_m32")
+    zg, zp = cfg.zero_grad_layers[0], cfg.zero_param_layers[0]
+    sample = sorted(set(list(range(0, cfg.h, 7)) + [zg, zp, 159, 160]))
+    sample = [l for l in sample if cfg.offsets[l + 1] - cfg.offsets[l] <= 1_100_000]
+    theta, mom = _run_and_check(oracle, cfg, sample)
+    a, b = int(cfg.offsets[zp]), int(cfg.offsets[zp + 1])
+    assert not theta[a:b].any() and mom[a:b].any()          # all-zero tensor does not move (c_l = 0)
+
+
+@pytest.mark.parametrize("bits", [2, 8])
+def test_flat_1b_sampled_layers(oracle, bits):
+    from paper_2206_06257_b200 import synth
+    if torch.cuda.get_device_properties(0).total_memory < 80e9:
+        pytest.skip("needs about 60 GB of device memory")
+    cfg = synth.config("flat1b", bits=bits)
+    sizes = np.diff(cfg.offsets)
+    order = np.argsort(sizes)
+    sample = sorted(set([int(order[0]), int(order[1]), int(order[len(order) // 2]), int(order[len(order) // 3]),
+                         0, cfg.h - 1, int(np.argmin(np.abs(sizes - 300_000)))]))
+    sample = [l for l in sample if sizes[l] <= 2_000_000]
+    _run_and_check(oracle, cfg, sample)
+    torch.cuda.empty_cache()
