@@ -250,10 +250,28 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    unfused = (args.path == "unfused")
+    if unfused:
+        if cfg.bits == 32:
+            raise SystemExit("--path unfused needs a quantized configuration (bits < 32)")
+        lb, sb, ns, _ = api.dat_plan_sizes(plan)
+        u_levels = torch.empty(cfg.M * lb, dtype=torch.uint8, device=dev)
+        u_signs = torch.empty(cfg.M * sb, dtype=torch.uint8, device=dev)
+        u_scales = torch.empty(ns, dtype=torch.float32, device=dev)
+        u_ghat = torch.empty(cfg.d, dtype=torch.float32, device=dev)
+
+    def one_step(step_index):
+        if unfused:
+            api.dat_quantize(plan, grads, cfg.seed, step_index, u_levels, u_signs, u_scales)
+            api.dat_aggregate(plan, u_levels, u_signs, u_scales, None, u_ghat)
+            api.dat_lalr_step(plan, theta, mom, u_ghat, hp)
+        else:
+            api.dat_step(plan, theta, mom, grads, cfg.seed, step_index, hp)
+
     # ---- warm-up
     step_no = 0
     for _ in range(max(args.warmup, 3)):
-        api.dat_step(plan, theta, mom, grads, cfg.seed, step_no, hp)
+        one_step(step_no)
         step_no += 1
     torch.cuda.synchronize()
     status = api.dat_get_status(plan)
@@ -272,7 +290,7 @@ def run_gpu(args):
         if flush is not None:
             flush.fill_(1.0)
         ev[2 * k].record(stream)
-        api.dat_step(plan, theta, mom, grads, cfg.seed, step_no, hp)
+        one_step(step_no)
         ev[2 * k + 1].record(stream)
         step_no += 1
     sampler.sample()
@@ -291,7 +309,7 @@ def run_gpu(args):
 
     # ---- end to end through the host-buffer entry point (H2D + step + D2H inside the timed region)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not unfused:
         th_h = theta.detach().cpu().pin_memory()
         mo_h = mom.detach().cpu().pin_memory()
         g_h = [g.detach().cpu().pin_memory() for g in grads]
@@ -327,9 +345,13 @@ def run_gpu(args):
     if rank == 0:
         peak, peak_src = measured_peaks()
         kernel_ms = float(step_ms.mean())
-        algo_bytes = (4 * cfg.M + 16) * cfg.d
+        if unfused:     # norm pass + quantize pass over the gradients, planes written and read, g_hat, two LALR passes
+            beta = (cfg.bits + 1) / 8.0
+            algo_bytes = int((8 * cfg.M + 2 * beta * cfg.M + 32) * cfg.d)
+        else:
+            algo_bytes = (4 * cfg.M + 16) * cfg.d
         achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-        traffic = NCU_DRAM_BYTES_PER_LAUNCH.get("%s_b%d" % (cfg.name, cfg.bits))
+        traffic = None if unfused else NCU_DRAM_BYTES_PER_LAUNCH.get("%s_b%d" % (cfg.name, cfg.bits))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": region_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -340,7 +362,8 @@ def run_gpu(args):
             "pct_of_8TBps": 100.0 * achieved / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "algorithmic_bytes_per_launch": algo_bytes,
-                         "kernel": "k_fused_step (one launch per step)", "peak_source": peak_src},
+                         "kernel": ("unfused path: 7 kernels per step (whole step timed)" if unfused else "k_fused_step (one launch per step)"),
+                         "peak_source": peak_src},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "status_word": int(status), "outputs_finite": finite, "wall_s_timed_region": t_wall,
         }
@@ -359,6 +382,8 @@ def main():
                     choices=["tiny_mlp", "resnet18", "resnet50", "resnet50_m32", "flat1b", "flat_small"])
     ap.add_argument("--bits", type=int, default=0, help="override the config's bits")
     ap.add_argument("--impl", default="dat", choices=["dat", "reference"])
+    ap.add_argument("--path", default="fused", choices=["fused", "unfused"],
+                    help="fused: dat_step (the headline); unfused: dat_quantize + dat_aggregate + dat_lalr_step")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
