@@ -19,6 +19,7 @@ import numpy as np
 from . import build as _build
 
 SCALE_SHARED_MAX = 0
+RNG_BITS = (16, 23)      # resolutions of the quantizer's uniform number
 SCALE_PER_WORKER = 1
 
 _lib = None
@@ -47,11 +48,13 @@ def _declare(L):
     L.dat_oracle_random_word.restype = _u32
     L.dat_oracle_uniform12.argtypes = [_u32]
     L.dat_oracle_uniform12.restype = _f32
+    L.dat_oracle_uniform12_at.argtypes = [_u64, _u64, _u32, _u64, _int]
+    L.dat_oracle_uniform12_at.restype = _f32
     L.dat_oracle_worker_norms.argtypes = [_i64, _p, _i64, _i64, _int, _p, _p]
     L.dat_oracle_worker_norms.restype = None
     L.dat_oracle_scales.argtypes = [_i64, _i64, _i64, _int, _int, _p, _p]
     L.dat_oracle_scales.restype = None
-    L.dat_oracle_quantize.argtypes = [_i64, _p, _i64, _i64, _int, _int, _int, _p, _u64, _u64, _p, _p, _p]
+    L.dat_oracle_quantize.argtypes = [_i64, _p, _i64, _i64, _int, _int, _int, _p, _u64, _u64, _int, _p, _p, _p]
     L.dat_oracle_quantize.restype = None
     L.dat_oracle_level_plane_bytes.argtypes = [_i64, _int]
     L.dat_oracle_level_plane_bytes.restype = _i64
@@ -67,7 +70,7 @@ def _declare(L):
     L.dat_oracle_average.restype = None
     L.dat_oracle_lalr.argtypes = [_p, _i64, _i64, _p, _p, _p, _f32, _f32, _f32, _f32, _f32, _p]
     L.dat_oracle_lalr.restype = None
-    L.dat_oracle_step.argtypes = [_i64, _p, _i64, _i64, _int, _int, _int, _p, _p, _p, _u64, _u64, _p,
+    L.dat_oracle_step.argtypes = [_i64, _p, _i64, _i64, _int, _int, _int, _p, _p, _p, _u64, _u64, _int, _p,
                                   _f32, _f32, _f32, _f32, _f32, _p, _p, _p]
     L.dat_oracle_step.restype = _int
 
@@ -130,6 +133,13 @@ def uniform12(w):
     return float(lib().dat_oracle_uniform12(int(w) & 0xFFFFFFFF))
 
 
+def uniform12_at(seed, step, worker, e, rng_bits):
+    """The quantizer's 1 + u of element e: u has 23 bits (one Philox block per 4 elements) or
+    16 bits (one block per 8 elements)."""
+    assert rng_bits in RNG_BITS
+    return float(lib().dat_oracle_uniform12_at(int(seed), int(step), int(worker), int(e), int(rng_bits)))
+
+
 # ---------------------------------------------------------------- S1
 
 def worker_norms(offsets, grads, l0=None, l1=None, window=False):
@@ -156,11 +166,11 @@ def scales(norms, scale_mode=SCALE_SHARED_MAX, l0=None, l1=None):
 # ---------------------------------------------------------------- S2
 
 def quantize(offsets, grads, bits, seed, step, scales_, scale_mode=SCALE_SHARED_MAX,
-             l0=None, l1=None, window=False):
+             l0=None, l1=None, window=False, rng_bits=16):
     """Returns (level uint32 [M, n], neg uint8 [M, n])."""
     o = _offsets(offsets)
     h, l0, l1, n, shift = _range(o, l0, l1, window)
-    assert bits in (1, 2, 4, 8, 16)
+    assert bits in (1, 2, 4, 8, 16) and rng_bits in RNG_BITS
     grads = [_check(g, np.float32, n) for g in grads]
     M = len(grads)
     sc = _check(np.ascontiguousarray(scales_, dtype=np.float32), np.float32,
@@ -168,7 +178,7 @@ def quantize(offsets, grads, bits, seed, step, scales_, scale_mode=SCALE_SHARED_
     level = np.zeros((M, n), dtype=np.uint32)
     neg = np.zeros((M, n), dtype=np.uint8)
     lib().dat_oracle_quantize(h, _addr(o), l0, l1, M, bits, scale_mode, _ptr_array(grads, shift),
-                              int(seed), int(step), _addr(sc),
+                              int(seed), int(step), int(rng_bits), _addr(sc),
                               _ptr_array(list(level), shift), _ptr_array(list(neg), shift))
     return level, neg
 
@@ -252,12 +262,12 @@ def lalr(offsets, theta, mom, g_hat, lr, momentum, weight_decay, c_l=0.0, c_u=10
 
 def step(offsets, theta, mom, grads, bits, seed, step_, lr, momentum, weight_decay,
          c_l=0.0, c_u=10.0, scale_mode=SCALE_SHARED_MAX, scales_in=None,
-         l0=None, l1=None, window=False, want_code_sum=True):
+         l0=None, l1=None, window=False, want_code_sum=True, rng_bits=16):
     """One DAT outer-minimisation step.  Returns a dict with theta, mom (new arrays),
     code_sum (int32 or None), layer_norms [h, 2], scales."""
     o = _offsets(offsets)
     h, l0, l1, n, shift = _range(o, l0, l1, window)
-    assert bits in (1, 2, 4, 8, 16, 32)
+    assert bits in (1, 2, 4, 8, 16, 32) and rng_bits in RNG_BITS
     th = _check(theta, np.float32, n).copy()
     mo = _check(mom, np.float32, n).copy()
     grads = [_check(g, np.float32, n) for g in grads]
@@ -272,7 +282,7 @@ def step(offsets, theta, mom, grads, bits, seed, step_, lr, momentum, weight_dec
     sout = np.zeros(n_scales, dtype=np.float32)
     rc = lib().dat_oracle_step(h, _addr(o), l0, l1, M, bits, scale_mode,
                                _addr(th, shift), _addr(mo, shift), _ptr_array(grads, shift),
-                               int(seed), int(step_), _addr(sin), lr, momentum, weight_decay, c_l, c_u,
+                               int(seed), int(step_), int(rng_bits), _addr(sin), lr, momentum, weight_decay, c_l, c_u,
                                _addr(code_sum, shift), _addr(norms), _addr(sout))
     if rc != 0:
         raise MemoryError("dat_oracle_step")

@@ -103,6 +103,29 @@ float dat_oracle_uniform12(uint32_t w)
     return f;
 }
 
+/* The quantizer's random number 1 + u of element e of `worker` at (seed, step), for the two
+ * resolutions of u the method is run with (the paper fixes neither generator nor resolution):
+ *   rng_bits = 23: u = (low 23 bits of dat_oracle_random_word) / 2^23 -- one Philox block per
+ *                  four consecutive elements;
+ *   rng_bits = 16: one Philox block per EIGHT consecutive elements: counter
+ *                  (lo(e/8), hi(e/8), worker, hi(seed)), same key; element e takes word
+ *                  (e/2) mod 4, its low half if e is even and its high half if e is odd;
+ *                  u = half / 2^16 (exact in a float).
+ * P(level rounds up) then matches the fractional part of x to within 2^-23 resp. 2^-16.      */
+float dat_oracle_uniform12_at(uint64_t seed, uint64_t step, uint32_t worker, uint64_t e, int rng_bits)
+{
+    if (rng_bits != 16)
+        return dat_oracle_uniform12(dat_oracle_random_word(seed, step, worker, e));
+    uint64_t q = e >> 3;
+    uint32_t ctr[4] = { (uint32_t)q, (uint32_t)(q >> 32), worker, (uint32_t)(seed >> 32) };
+    uint32_t key[2] = { (uint32_t)seed, (uint32_t)step };
+    uint32_t out[4];
+    dat_oracle_philox4x32_10(ctr, key, out);
+    uint32_t w = out[(e >> 1) & 3u];
+    uint32_t half = (e & 1u) ? (w >> 16) : (w & 0xFFFFu);
+    return 1.0f + (float)half * (1.0f / 65536.0f);
+}
+
 /* ------------------------------------------------------------------------- */
 /* S1: quantizer norms.  ||g||_2 of Eq. rand_q, one per (worker, layer).       */
 /* ------------------------------------------------------------------------- */
@@ -161,7 +184,7 @@ static float scale_of(const float *scales, int scale_mode, int64_t h, int i, int
  * level[i][e] in {0..S}; neg[i][e] = 1 iff g < 0 (so -0.0 and NaN give 0).       */
 void dat_oracle_quantize(int64_t h, const int64_t *offsets, int64_t l0, int64_t l1,
                          int M, int bits, int scale_mode,
-                         const float *const *grads, uint64_t seed, uint64_t step,
+                         const float *const *grads, uint64_t seed, uint64_t step, int rng_bits,
                          const float *scales,
                          uint32_t *const *level, uint8_t *const *neg)
 {
@@ -173,7 +196,7 @@ void dat_oracle_quantize(int64_t h, const int64_t *offsets, int64_t l0, int64_t 
             float t = (nu == 0.0f) ? 0.0f : S_f / nu;
             for (int64_t e = offsets[l]; e < offsets[l + 1]; ++e) {
                 float g = grads[i][e];
-                float u1 = dat_oracle_uniform12(dat_oracle_random_word(seed, step, (uint32_t)i, (uint64_t)e));
+                float u1 = dat_oracle_uniform12_at(seed, step, (uint32_t)i, (uint64_t)e, rng_bits);
                 float y = fminf(fmaf(fabsf(g), t, u1), S_f + 1.0f);
                 level[i][e] = (uint32_t)floorf(y) - 1u;
                 neg[i][e] = (uint8_t)(g < 0.0f);
@@ -328,7 +351,7 @@ void dat_oracle_lalr(const int64_t *offsets, int64_t l0, int64_t l1,
 int dat_oracle_step(int64_t h, const int64_t *offsets, int64_t l0, int64_t l1,
                     int M, int bits, int scale_mode,
                     float *theta, float *mom, const float *const *grads,
-                    uint64_t seed, uint64_t step, const float *scales_in,
+                    uint64_t seed, uint64_t step, int rng_bits, const float *scales_in,
                     float lr, float mu, float wd, float c_l, float c_u,
                     int32_t *code_sum, float *layer_norms, float *scales_out)
 {
@@ -370,7 +393,7 @@ int dat_oracle_step(int64_t h, const int64_t *offsets, int64_t l0, int64_t l1,
                 dat_oracle_worker_norms(h, offsets, l, l + 1, M, grads, norms);
                 dat_oracle_scales(h, l, l + 1, M, scale_mode, norms, scales);
             }
-            dat_oracle_quantize(h, offsets, l, l + 1, M, bits, scale_mode, grads, seed, step, scales,
+            dat_oracle_quantize(h, offsets, l, l + 1, M, bits, scale_mode, grads, seed, step, rng_bits, scales,
                                 (uint32_t *const *)level, (uint8_t *const *)neg);
             dat_oracle_aggregate(h, offsets, l, l + 1, M, bits, scale_mode,
                                  (const uint32_t *const *)level, (const uint8_t *const *)neg,

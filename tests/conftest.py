@@ -18,3 +18,9 @@ def oracle():
     import oracle as _oracle
     _oracle.lib()
     return _oracle
+
+
+@pytest.fixture(params=[16, 23], ids=["rng16", "rng23"])
+def rng_bits(request):
+    """Resolution of the quantizer's uniform number: both supported values."""
+    return request.param

@@ -67,3 +67,39 @@ def test_uniform_moments(oracle):
     for bit in range(32):
         frac = ((w >> np.uint64(bit)) & np.uint64(1)).mean()
         assert abs(frac - 0.5) < 5 * 0.5 / 4096 ** 0.5
+
+
+def test_uniform_at_23_bits_is_the_word_uniform(oracle):
+    for e in (0, 1, 5, 1023, (1 << 33) + 3):
+        assert oracle.uniform12_at(9, 4, 2, e, 23) == oracle.uniform12(oracle.random_word(9, 4, 2, e))
+
+
+def test_uniform_at_16_bits_keying(oracle):
+    """16-bit resolution: one block per eight elements, counter (lo(e/8), hi(e/8), worker, hi(seed)),
+    key (lo(seed), step); element e takes word (e/2) mod 4, low half if e is even, high half if
+    odd; 1 + half / 2^16.  Checked against the block function, which the known-answer vectors pin."""
+    seed = 0x0123456789ABCDEF
+    for e in (0, 1, 2, 3, 6, 7, 8, 9, 15, 16, (1 << 20) + 5, (1 << 35) + 6):
+        for worker in (0, 3):
+            for step in (0, 9):
+                q = e >> 3
+                blk = oracle.philox4x32_10([q & 0xFFFFFFFF, q >> 32, worker, seed >> 32],
+                                           [seed & 0xFFFFFFFF, step])
+                w = int(blk[(e >> 1) & 3])
+                half = (w >> 16) if (e & 1) else (w & 0xFFFF)
+                got = oracle.uniform12_at(seed, step, worker, e, 16)
+                assert got == 1.0 + half / 65536.0
+                assert 1.0 <= got < 2.0
+
+
+def test_uniform_at_16_bits_moments(oracle):
+    n = 40000
+    u = np.array([oracle.uniform12_at(7, 3, 1, e, 16) for e in range(n)]) - 1.0
+    assert u.min() >= 0.0 and u.max() < 1.0
+    assert np.all(u * 65536 == np.round(u * 65536))          # on the 2^-16 grid
+    assert abs(u.mean() - 0.5) < 5 * (1 / 12 ** 0.5) / n ** 0.5
+    assert abs(u.var() - 1 / 12) < 0.003
+    # neighbours (the two halves of a word, the words of a block) are uncorrelated
+    for lag in (1, 2, 8):
+        c = np.corrcoef(u[:-lag], u[lag:])[0, 1]
+        assert abs(c) < 5 / n ** 0.5

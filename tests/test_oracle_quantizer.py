@@ -30,7 +30,7 @@ def test_worker_norms_match_float64_norm(oracle):
     assert np.array_equal(oracle.scales(nrm, oracle.SCALE_PER_WORKER), nrm)
 
 
-def test_hand_case_b2(oracle):
+def test_hand_case_b2(oracle, rng_bits):
     rows = [list(map(float, l.split())) for l in open(GOLDEN) if l.strip() and not l.startswith("#")]
     g = np.array([r[0] for r in rows], dtype=np.float32)
     offs = _offs(len(g))
@@ -40,7 +40,7 @@ def test_hand_case_b2(oracle):
     n_seeds = 4000
     acc = np.zeros(len(g))
     for seed in range(n_seeds):
-        level, neg = oracle.quantize(offs, [g], 2, seed, 0, sc)
+        level, neg = oracle.quantize(offs, [g], 2, seed, 0, sc, rng_bits=rng_bits)
         for k, r in enumerate(rows):
             fl = int(r[3])
             assert level[0, k] in ((fl, fl + 1) if r[4] > 0 else (fl,))
@@ -55,13 +55,13 @@ def test_hand_case_b2(oracle):
 
 
 @pytest.mark.parametrize("bits", [1, 2, 4, 8, 16])
-def test_level_is_a_neighbouring_grid_point(oracle, bits):
+def test_level_is_a_neighbouring_grid_point(oracle, bits, rng_bits):
     """xi takes one of the two grid points around |g|/||g|| (Eq. xi); levels fit in b bits."""
     rng = np.random.RandomState(bits)
     offs = _offs(257, 64, 1023)
     grads = [(rng.standard_t(3, offs[-1]) * 0.01).astype(np.float32) for _ in range(2)]
     nrm, sc = _norms_scales(oracle, offs, grads)
-    level, neg = oracle.quantize(offs, grads, bits, 11, 5, sc)
+    level, neg = oracle.quantize(offs, grads, bits, 11, 5, sc, rng_bits=rng_bits)
     S = 2 ** bits - 1
     assert level.max() <= S
     for i in range(2):
@@ -77,7 +77,7 @@ def test_level_is_a_neighbouring_grid_point(oracle, bits):
 
 
 @pytest.mark.parametrize("bits", [2, 4, 8])
-def test_exact_cases(oracle, bits):
+def test_exact_cases(oracle, bits, rng_bits):
     S = 2 ** bits - 1
     # (a) one non-zero element, a power of two: x = S exactly, Q(g) = g for every seed
     g = np.zeros(37, dtype=np.float32)
@@ -86,7 +86,7 @@ def test_exact_cases(oracle, bits):
     nrm, sc = _norms_scales(oracle, offs, [g])
     assert sc[0] == np.float32(0.125)
     for seed in range(20):
-        level, neg = oracle.quantize(offs, [g], bits, seed, 0, sc)
+        level, neg = oracle.quantize(offs, [g], bits, seed, 0, sc, rng_bits=rng_bits)
         assert level[0, 5] == S and neg[0, 5] == 1 and level[0].sum() == S
     # (b) S^2 elements all +-c, c a power of two: ||g|| = S*c, x = 1 exactly, every level is 1
     n = S * S
@@ -96,13 +96,13 @@ def test_exact_cases(oracle, bits):
     nrm, sc = _norms_scales(oracle, offs, [g])
     assert sc[0] == np.float32(S * 0.25)
     for seed in range(3):
-        level, neg = oracle.quantize(offs, [g], bits, seed, 1, sc)
+        level, neg = oracle.quantize(offs, [g], bits, seed, 1, sc, rng_bits=rng_bits)
         assert (level[0] == 1).all()
         q = np.where(neg[0] == 1, -1.0, 1.0) * level[0] * (float(sc[0]) / S)
         assert np.array_equal(q.astype(np.float32), g)
 
 
-def test_unbiased_and_variance_bound(oracle):
+def test_unbiased_and_variance_bound(oracle, rng_bits):
     """E[Q(g)] = g and E||Q(g)-g||^2 <= min{n/S^2, sqrt(n)/S} ||g||^2 (QSGD Lemma 3.1, cited
     under assumption A4), by Monte Carlo over seeds."""
     rng = np.random.RandomState(3)
@@ -115,7 +115,7 @@ def test_unbiased_and_variance_bound(oracle):
     mean = np.zeros(n)
     err2 = 0.0
     for seed in range(n_seeds):
-        level, neg = oracle.quantize(offs, [g], bits, seed, 0, sc)
+        level, neg = oracle.quantize(offs, [g], bits, seed, 0, sc, rng_bits=rng_bits)
         q = np.where(neg[0] == 1, -1.0, 1.0) * level[0] * (nu / S)
         mean += q
         err2 += np.sum((q - g) ** 2)
@@ -128,7 +128,7 @@ def test_unbiased_and_variance_bound(oracle):
     assert err2 > 0.01 * min(n / S ** 2, np.sqrt(n) / S) * nu ** 2
 
 
-def test_up_probability_is_fraction(oracle):
+def test_up_probability_is_fraction(oracle, rng_bits):
     """P(level = floor(x)+1) = x - floor(x) for a fixed x, across element positions."""
     n, bits = 40000, 8
     S = 255
@@ -137,40 +137,40 @@ def test_up_probability_is_fraction(oracle):
     offs = _offs(n)
     nrm, sc = _norms_scales(oracle, offs, [g])
     x = 0.3 * S / float(sc[0])
-    level, _ = oracle.quantize(offs, [g], bits, 5, 2, sc)
+    level, _ = oracle.quantize(offs, [g], bits, 5, 2, sc, rng_bits=rng_bits)
     p = (level[0, 1:] == np.floor(x) + 1).mean()
     frac = x - np.floor(x)
     assert abs(p - frac) < 5 * np.sqrt(frac * (1 - frac) / n)
 
 
-def test_scale_invariance_power_of_two(oracle):
+def test_scale_invariance_power_of_two(oracle, rng_bits):
     rng = np.random.RandomState(4)
     offs = _offs(100, 333)
     grads = [(rng.randn(offs[-1]) * 1e-3).astype(np.float32) for _ in range(3)]
     nrm, sc = _norms_scales(oracle, offs, grads)
-    l1, n1 = oracle.quantize(offs, grads, 8, 1, 1, sc)
+    l1, n1 = oracle.quantize(offs, grads, 8, 1, 1, sc, rng_bits=rng_bits)
     grads2 = [g * np.float32(2.0 ** 7) for g in grads]
     nrm2, sc2 = _norms_scales(oracle, offs, grads2)
     assert np.array_equal(sc2, sc * np.float32(128.0))
-    l2, n2 = oracle.quantize(offs, grads2, 8, 1, 1, sc2)
+    l2, n2 = oracle.quantize(offs, grads2, 8, 1, 1, sc2, rng_bits=rng_bits)
     assert np.array_equal(l1, l2) and np.array_equal(n1, n2)
 
 
-def test_zero_norm_layer_gives_zero_levels(oracle):
+def test_zero_norm_layer_gives_zero_levels(oracle, rng_bits):
     offs = _offs(10, 20)
     g = np.zeros(30, dtype=np.float32)
     g[10:] = 1.0
     nrm, sc = _norms_scales(oracle, offs, [g])
     assert sc[0] == 0.0
-    level, neg = oracle.quantize(offs, [g], 8, 0, 0, sc)
+    level, neg = oracle.quantize(offs, [g], 8, 0, 0, sc, rng_bits=rng_bits)
     assert (level[0, :10] == 0).all() and (neg == 0).all()
 
 
-def test_random_stream_independent_of_layer_partition(oracle):
+def test_random_stream_independent_of_layer_partition(oracle, rng_bits):
     rng = np.random.RandomState(5)
     g = rng.randn(64).astype(np.float32)
-    a = oracle.quantize(_offs(64), [g], 8, 3, 3, np.array([10.0], np.float32))
-    b = oracle.quantize(_offs(10, 54), [g], 8, 3, 3, np.array([10.0, 10.0], np.float32))
+    a = oracle.quantize(_offs(64), [g], 8, 3, 3, np.array([10.0], np.float32), rng_bits=rng_bits)
+    b = oracle.quantize(_offs(10, 54), [g], 8, 3, 3, np.array([10.0, 10.0], np.float32), rng_bits=rng_bits)
     assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
 
 

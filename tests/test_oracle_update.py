@@ -22,7 +22,7 @@ def _problem(rng, sizes, M, sigma=1e-2):
 
 # ------------------------------------------------------------------ aggregation
 
-def test_aggregate_is_mean_of_dequantized_messages(oracle):
+def test_aggregate_is_mean_of_dequantized_messages(oracle, rng_bits):
     """g_hat = (1/M) sum_i ||g||*sign*level/S, evaluated independently in float64."""
     rng = np.random.RandomState(0)
     offs, grads, _, _ = _problem(rng, [100, 7, 300], 5)
@@ -30,7 +30,7 @@ def test_aggregate_is_mean_of_dequantized_messages(oracle):
     nrm = oracle.worker_norms(offs, grads)
     for mode in (oracle.SCALE_SHARED_MAX, oracle.SCALE_PER_WORKER):
         sc = oracle.scales(nrm, mode)
-        level, neg = oracle.quantize(offs, grads, bits, 2, 0, sc, mode)
+        level, neg = oracle.quantize(offs, grads, bits, 2, 0, sc, mode, rng_bits=rng_bits)
         code_sum, g_hat = oracle.aggregate(offs, level, neg, sc, bits, mode)
         signed = np.where(neg == 1, -1.0, 1.0) * level.astype(np.float64)
         ref = np.zeros(offs[-1])
@@ -49,24 +49,24 @@ def test_aggregate_is_mean_of_dequantized_messages(oracle):
             assert code_sum is None
 
 
-def test_per_worker_formula_with_equal_scales_matches_shared(oracle):
+def test_per_worker_formula_with_equal_scales_matches_shared(oracle, rng_bits):
     rng = np.random.RandomState(1)
     offs, grads, _, _ = _problem(rng, [64, 200], 4)
     nrm = oracle.worker_norms(offs, grads)
     sc = oracle.scales(nrm, oracle.SCALE_SHARED_MAX)
-    level, neg = oracle.quantize(offs, grads, 8, 0, 0, sc)
+    level, neg = oracle.quantize(offs, grads, 8, 0, 0, sc, rng_bits=rng_bits)
     _, g_shared = oracle.aggregate(offs, level, neg, sc, 8)
     sc_pw = np.tile(sc, (4, 1))
     _, g_pw = oracle.aggregate(offs, level, neg, sc_pw, 8, oracle.SCALE_PER_WORKER)
     assert np.allclose(g_shared, g_pw, rtol=1e-6, atol=4 * 6e-8 * float(sc.max()))
 
 
-def test_m1_aggregate_is_the_signed_code(oracle):
+def test_m1_aggregate_is_the_signed_code(oracle, rng_bits):
     rng = np.random.RandomState(2)
     offs, grads, _, _ = _problem(rng, [50, 50], 1)
     nrm = oracle.worker_norms(offs, grads)
     sc = oracle.scales(nrm)
-    level, neg = oracle.quantize(offs, grads, 8, 0, 0, sc)
+    level, neg = oracle.quantize(offs, grads, 8, 0, 0, sc, rng_bits=rng_bits)
     code_sum, g_hat = oracle.aggregate(offs, level, neg, sc, 8)
     assert np.array_equal(code_sum, np.where(neg[0] == 1, -1, 1) * level[0].astype(np.int64))
 
@@ -169,15 +169,15 @@ def test_zero_norm_conventions(oracle):
 
 # ------------------------------------------------------------------ whole step
 
-def test_step_equals_composition(oracle):
+def test_step_equals_composition(oracle, rng_bits):
     rng = np.random.RandomState(6)
     offs, grads, theta, mom = _problem(rng, [40, 1000, 9, 513], 3)
     hp = dict(lr=0.1, momentum=0.9, weight_decay=5e-4)
     for mode in (oracle.SCALE_SHARED_MAX, oracle.SCALE_PER_WORKER):
-        out = oracle.step(offs, theta, mom, grads, 8, 42, 7, scale_mode=mode, **hp)
+        out = oracle.step(offs, theta, mom, grads, 8, 42, 7, scale_mode=mode, **hp, rng_bits=rng_bits)
         nrm = oracle.worker_norms(offs, grads)
         sc = oracle.scales(nrm, mode)
-        level, neg = oracle.quantize(offs, grads, 8, 42, 7, sc, mode)
+        level, neg = oracle.quantize(offs, grads, 8, 42, 7, sc, mode, rng_bits=rng_bits)
         cs, g_hat = oracle.aggregate(offs, level, neg, sc, 8, mode)
         th, mo, norms = oracle.lalr(offs, theta, mom, g_hat, hp["lr"], hp["momentum"], hp["weight_decay"])
         assert np.array_equal(out["theta"], th) and np.array_equal(out["mom"], mo)
@@ -187,43 +187,43 @@ def test_step_equals_composition(oracle):
             assert np.array_equal(out["code_sum"], cs)
 
 
-def test_step_window_equals_full(oracle):
+def test_step_window_equals_full(oracle, rng_bits):
     rng = np.random.RandomState(7)
     offs, grads, theta, mom = _problem(rng, [40, 1000, 9, 513], 2)
     hp = dict(lr=0.1, momentum=0.9, weight_decay=5e-4)
-    full = oracle.step(offs, theta, mom, grads, 4, 1, 2, **hp)
+    full = oracle.step(offs, theta, mom, grads, 4, 1, 2, **hp, rng_bits=rng_bits)
     a, b = int(offs[1]), int(offs[3])
     win = oracle.step(offs, theta[a:b].copy(), mom[a:b].copy(), [g[a:b].copy() for g in grads], 4, 1, 2,
-                      l0=1, l1=3, window=True, **hp)
+                      l0=1, l1=3, window=True, **hp, rng_bits=rng_bits)
     assert np.array_equal(win["theta"], full["theta"][a:b])
     assert np.array_equal(win["mom"], full["mom"][a:b])
     assert np.array_equal(win["code_sum"], full["code_sum"][a:b])
 
 
-def test_m1_b32_step_is_plain_lalr(oracle):
+def test_m1_b32_step_is_plain_lalr(oracle, rng_bits):
     """M = 1 reduces DAT to AT (Sec. 3); with b = 32 nothing is quantized."""
     rng = np.random.RandomState(8)
     offs, grads, theta, mom = _problem(rng, [100, 50], 1)
-    out = oracle.step(offs, theta, mom, grads, 32, 0, 0, 0.1, 0.9, 1e-4)
+    out = oracle.step(offs, theta, mom, grads, 32, 0, 0, 0.1, 0.9, 1e-4, rng_bits=rng_bits)
     th, mo, _ = oracle.lalr(offs, theta, mom, grads[0], 0.1, 0.9, 1e-4)
     assert np.array_equal(out["theta"], th) and np.array_equal(out["mom"], mo)
 
 
-def test_step_with_many_bits_approaches_unquantized_step(oracle):
+def test_step_with_many_bits_approaches_unquantized_step(oracle, rng_bits):
     """As b grows Q -> identity: the 16-bit step is close to the 32-bit (exact average) step."""
     rng = np.random.RandomState(9)
     offs, grads, theta, mom = _problem(rng, [300, 700], 4)
     hp = dict(lr=0.1, momentum=0.9, weight_decay=5e-4)
-    exact = oracle.step(offs, theta, mom, grads, 32, 0, 0, **hp)
-    q16 = oracle.step(offs, theta, mom, grads, 16, 0, 0, **hp)
-    q2 = oracle.step(offs, theta, mom, grads, 2, 0, 0, **hp)
+    exact = oracle.step(offs, theta, mom, grads, 32, 0, 0, **hp, rng_bits=rng_bits)
+    q16 = oracle.step(offs, theta, mom, grads, 16, 0, 0, **hp, rng_bits=rng_bits)
+    q2 = oracle.step(offs, theta, mom, grads, 2, 0, 0, **hp, rng_bits=rng_bits)
     e16 = np.abs(q16["mom"] - exact["mom"]).max()
     e2 = np.abs(q2["mom"] - exact["mom"]).max()
     nu = oracle.scales(oracle.worker_norms(offs, grads)).max()
     assert e16 <= nu / 65535 + 1e-9 and e2 > 50 * e16
 
 
-def test_resume_is_exact(oracle):
+def test_resume_is_exact(oracle, rng_bits):
     """The random stream is a pure function of (seed, step, worker, element): 4 straight
     steps equal 2 steps + copy of (theta, m) + 2 steps, bit for bit."""
     rng = np.random.RandomState(10)
@@ -232,30 +232,30 @@ def test_resume_is_exact(oracle):
     hp = dict(lr=0.05, momentum=0.9, weight_decay=1e-4)
     th, mo = theta, mom
     for t in range(4):
-        o = oracle.step(offs, th, mo, gs[t], 8, 5, t, **hp)
+        o = oracle.step(offs, th, mo, gs[t], 8, 5, t, **hp, rng_bits=rng_bits)
         th, mo = o["theta"], o["mom"]
     th2, mo2 = theta, mom
     for t in range(2):
-        o = oracle.step(offs, th2, mo2, gs[t], 8, 5, t, **hp)
+        o = oracle.step(offs, th2, mo2, gs[t], 8, 5, t, **hp, rng_bits=rng_bits)
         th2, mo2 = o["theta"], o["mom"]
     th2, mo2 = th2.copy(), mo2.copy()
     for t in range(2, 4):
-        o = oracle.step(offs, th2, mo2, gs[t], 8, 5, t, **hp)
+        o = oracle.step(offs, th2, mo2, gs[t], 8, 5, t, **hp, rng_bits=rng_bits)
         th2, mo2 = o["theta"], o["mom"]
     assert np.array_equal(th, th2) and np.array_equal(mo, mo2)
     # and the step index matters
-    o_same = oracle.step(offs, theta, mom, gs[0], 8, 5, 0, **hp)
-    o_other = oracle.step(offs, theta, mom, gs[0], 8, 5, 1, **hp)
+    o_same = oracle.step(offs, theta, mom, gs[0], 8, 5, 0, **hp, rng_bits=rng_bits)
+    o_other = oracle.step(offs, theta, mom, gs[0], 8, 5, 1, **hp, rng_bits=rng_bits)
     assert not np.array_equal(o_same["code_sum"], o_other["code_sum"])
 
 
-def test_tiny_mlp_config_runs(oracle):
+def test_tiny_mlp_config_runs(oracle, rng_bits):
     from paper_2206_06257_b200 import synth
     cfg = synth.config("tiny_mlp")
     theta, mom = synth.make_params(cfg)
     grads = synth.make_grads(cfg, 0)
     out = oracle.step(cfg.offsets, theta.numpy(), mom.numpy(), [g.numpy() for g in grads], cfg.bits, 0, 0,
-                      cfg.lr, cfg.momentum, cfg.weight_decay, cfg.c_l, cfg.c_u)
+                      cfg.lr, cfg.momentum, cfg.weight_decay, cfg.c_l, cfg.c_u, rng_bits=rng_bits)
     assert np.isfinite(out["theta"]).all() and np.abs(out["code_sum"]).max() <= cfg.M * 255
     for l in range(cfg.h):
         sl = slice(cfg.offsets[l], cfg.offsets[l + 1])
