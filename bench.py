@@ -135,7 +135,7 @@ def time_oracle(cfg, theta, mom, grads, layers, threads, step=0):
     def run(l):
         a, b = int(offs[l]), int(offs[l + 1])
         oracle.step(offs, theta[a:b], mom[a:b], [g[a:b] for g in grads], cfg.bits, cfg.seed, step, *hp,
-                    l0=l, l1=l + 1, window=True, want_code_sum=False)
+                    l0=l, l1=l + 1, window=True, want_code_sum=False, rng_bits=cfg.rng_bits)
         return (b - a) * cfg.M
     order = sorted(layers, key=lambda l: -(offs[l + 1] - offs[l]))     # big layers first
     t0 = time.perf_counter()
@@ -207,7 +207,7 @@ def job_value(world, elems_per_step, steps, seconds):
 
 
 def workload_config(cfg, l2_note):
-    return {"workload": cfg.name, "d": cfg.d, "layers": cfg.h, "workers_M": cfg.M, "bits": cfg.bits,
+    return {"workload": cfg.name, "d": cfg.d, "layers": cfg.h, "workers_M": cfg.M, "bits": cfg.bits, "rng_bits": cfg.rng_bits,
             "lr": cfg.lr, "momentum": cfg.momentum, "weight_decay": cfg.weight_decay,
             "grad_dist": cfg.grad_dist, "parallelism": "replicas", "l2": l2_note}
 
@@ -231,10 +231,12 @@ def run_gpu(args):
     cfg = synth.config(args.config)
     if args.bits:
         cfg.bits = args.bits
+    if args.rng_bits:
+        cfg.rng_bits = args.rng_bits
     theta, mom = synth.make_params(cfg, device=dev)
     grads = synth.make_grads(cfg, 0, device=dev)
     hp = (cfg.lr, cfg.momentum, cfg.weight_decay, cfg.c_l, cfg.c_u)
-    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits)
+    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits, rng_bits=cfg.rng_bits)
     stream = torch.cuda.current_stream()
     working_set = (cfg.M + 2) * cfg.d * 4
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
@@ -381,6 +383,8 @@ def main():
     ap.add_argument("--config", default="resnet50",
                     choices=["tiny_mlp", "resnet18", "resnet50", "resnet50_m32", "flat1b", "flat_small"])
     ap.add_argument("--bits", type=int, default=0, help="override the config's bits")
+    ap.add_argument("--rng-bits", type=int, default=0, choices=[0, 16, 23],
+                    help="override the resolution of the quantizer's uniform number (0: the config's)")
     ap.add_argument("--impl", default="dat", choices=["dat", "reference"])
     ap.add_argument("--path", default="fused", choices=["fused", "unfused"],
                     help="fused: dat_step (the headline); unfused: dat_quantize + dat_aggregate + dat_lalr_step")

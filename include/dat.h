@@ -64,6 +64,9 @@ typedef struct dat_hparams {
  *             followed by one scaling.  (Q stays unbiased for any nu >= max|g|.)              */
 enum { DAT_SCALE_SHARED_MAX = 0 };
 
+/* Resolution of the quantizer's uniform number (see dat_plan_create). */
+enum { DAT_RNG_BITS_16 = 16, DAT_RNG_BITS_23 = 23 };
+
 enum {
     DAT_OK = 0,
     DAT_ERR_ARG = -1,          /* null pointer, negative size, value out of range              */
@@ -94,10 +97,21 @@ enum {
  *   bits           b in {1,2,4,8,16}, or 32 = no quantisation (Q is the identity and the
  *                  aggregate is the plain worker average).
  *   scale_mode     DAT_SCALE_SHARED_MAX.
+ *   rng_bits       resolution of the uniform number u of the stochastic rounding (Eq. xi; the
+ *                  paper fixes neither generator nor resolution).  Randomness is Philox4x32-10
+ *                  keyed on (seed, step, worker, element):
+ *                  DAT_RNG_BITS_23: one block per four consecutive elements (counter
+ *                    (lo(e/4), hi(e/4), worker, hi(seed)), key (lo(seed), step)), element e takes
+ *                    word e mod 4, u = (low 23 bits) / 2^23;
+ *                  DAT_RNG_BITS_16: one block per eight consecutive elements (counter e/8),
+ *                    element e takes word (e/2) mod 4, low half if e is even, high half if odd,
+ *                    u = half / 2^16.  Half the generator work per element; the rounding
+ *                    probability matches frac(x) to 2^-16 of a level.
+ *                  Ignored for bits = 32.
  * Allocates the plan's device workspace (synchronous).  Errors: ARG, BITS, LAYOUT, NOMEM, CUDA.
  * ------------------------------------------------------------------------------------------- */
 int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64_t *layer_offsets,
-                    int num_workers, int bits, int scale_mode);
+                    int num_workers, int bits, int scale_mode, int rng_bits);
 
 /* Frees the plan and its workspace (synchronises the device).  NULL is accepted. */
 int dat_plan_destroy(dat_plan_t *plan);

@@ -22,6 +22,7 @@ _lib = C.CDLL(LIB_PATH)
 
 DAT_MAX_WORKERS = 64
 DAT_SCALE_SHARED_MAX = 0
+DAT_RNG_BITS_16, DAT_RNG_BITS_23 = 16, 23
 DAT_OK, DAT_ERR_ARG, DAT_ERR_ALIGN, DAT_ERR_BITS = 0, -1, -2, -3
 DAT_ERR_LAYOUT, DAT_ERR_CUDA, DAT_ERR_NOMEM, DAT_ERR_UNSUPPORTED, DAT_ERR_TOO_LARGE = -4, -5, -6, -7, -8
 DAT_STATIC_MAX_LAYERS, DAT_STATIC_MAX_TILES = 4096, 32768
@@ -39,7 +40,7 @@ class dat_hparams_t(C.Structure):
 
 
 _p, _i64, _u64, _int = C.c_void_p, C.c_int64, C.c_uint64, C.c_int
-_lib.dat_plan_create.argtypes = [C.POINTER(_p), _i64, _p, _int, _int, _int]
+_lib.dat_plan_create.argtypes = [C.POINTER(_p), _i64, _p, _int, _int, _int, _int]
 _lib.dat_plan_destroy.argtypes = [_p]
 _lib.dat_plan_sizes.argtypes = [_p, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]
 _lib.dat_quantize.argtypes = [_p, _p, _u64, _u64, _p, _p, _p, _p, _p]
@@ -107,12 +108,12 @@ def dat_strerror(code):
     return _lib.dat_strerror(int(code)).decode()
 
 
-def dat_plan_create(layer_offsets, num_workers, bits, scale_mode=DAT_SCALE_SHARED_MAX):
+def dat_plan_create(layer_offsets, num_workers, bits, scale_mode=DAT_SCALE_SHARED_MAX, rng_bits=DAT_RNG_BITS_16):
     """Returns the plan handle (an int).  layer_offsets: h+1 int64 values (any sequence)."""
     offs = np.ascontiguousarray(layer_offsets, dtype=np.int64)
     out = _p()
     _ok(_lib.dat_plan_create(C.byref(out), offs.size - 1, _ptr(offs), int(num_workers), int(bits),
-                             int(scale_mode)), "dat_plan_create")
+                             int(scale_mode), int(rng_bits)), "dat_plan_create")
     return out.value
 
 

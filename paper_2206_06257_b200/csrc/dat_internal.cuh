@@ -29,7 +29,7 @@ struct FusedSchedule;   // dat_step.cu
 struct dat_plan {
     int device = 0;
     int64_t h = 0, d = 0;
-    int M = 0, bits = 0, scale_mode = 0;
+    int M = 0, bits = 0, scale_mode = 0, rng_bits = 16;
     uint32_t S = 0;
     std::vector<int64_t> offsets;      // host copy, h+1
     std::vector<int64_t> tile_base;    // host copy, h+1: first per-layer tile of each layer
@@ -110,21 +110,52 @@ __device__ __forceinline__ void dat_random_words(uint64_t q, uint32_t worker, co
     dat_philox((uint32_t)q, (uint32_t)(q >> 32), worker, k.seed_hi, k, out);
 }
 
-// Stochastic level of one element (Eq. xi): level = min(floor(|g|*qmul + u), S) with u uniform
-// on [0,1).  The low 23 bits of the random word w are the mantissa of u1 = 1 + u in [1,2), so
-// y = fma(|g|, qmul, u1) is clamped to S+1 and level = floor(y) - 1.  y lies in [1, 65537):
-// adding 2^23 - 1 with rounding toward -inf leaves floor(y) - 1 in the low mantissa bits.
-// Returns those float bits, 0x4B000000 + level.
-__device__ __forceinline__ uint32_t dat_level_bits(float g, float qmul, float S1_f, uint32_t w)
+// The quantizer's random number u1 = 1 + u in [1, 2), u uniform on a 2^-23 grid: the low 23 bits
+// of a random word become the mantissa.
+__device__ __forceinline__ float dat_u1_from_word(uint32_t w)
 {
-    const float u1 = __uint_as_float(0x3F800000u | (w & 0x007FFFFFu));
+    return __uint_as_float(0x3F800000u | (w & 0x007FFFFFu));
+}
+
+// The same on a 2^-16 grid, from a 16-bit half word: 1 + half / 2^16.
+__device__ __forceinline__ float dat_u1_from_half(uint32_t half)
+{
+    return __uint_as_float(0x3F800000u | (half << 7));
+}
+
+// u1 of the four elements e0 .. e0+3 (e0 a multiple of 4) of `worker`.  rng16 = false: one
+// Philox block per four elements, word j for element e0+j.  rng16 = true: one block per EIGHT
+// elements (counter e/8); element e takes word (e/2) mod 4, low half if e is even, high if odd.
+__device__ __forceinline__ void dat_u1x4(uint64_t e0, uint32_t worker, const PhiloxKeys &k, bool rng16, float u1[4])
+{
+    uint32_t w[4];
+    if (!rng16) {
+        dat_random_words(e0 >> 2, worker, k, w);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) u1[j] = dat_u1_from_word(w[j]);
+    } else {
+        dat_random_words(e0 >> 3, worker, k, w);
+        const uint32_t wa = (e0 & 4u) ? w[2] : w[0], wb = (e0 & 4u) ? w[3] : w[1];
+        u1[0] = dat_u1_from_half(wa & 0xFFFFu);
+        u1[1] = dat_u1_from_half(wa >> 16);
+        u1[2] = dat_u1_from_half(wb & 0xFFFFu);
+        u1[3] = dat_u1_from_half(wb >> 16);
+    }
+}
+
+// Stochastic level of one element (Eq. xi): level = min(floor(|g|*qmul + u), S) with u uniform
+// on [0,1).  With u1 = 1 + u in [1,2), y = fma(|g|, qmul, u1) is clamped to S+1 and
+// level = floor(y) - 1.  y lies in [1, 65537): adding 2^23 - 1 with rounding toward -inf leaves
+// floor(y) - 1 in the low mantissa bits.  Returns those float bits, 0x4B000000 + level.
+__device__ __forceinline__ uint32_t dat_level_bits_u1(float g, float qmul, float S1_f, float u1)
+{
     const float y = fminf(__fmaf_rn(fabsf(g), qmul, u1), S1_f);
     return __float_as_uint(__fadd_rd(y, 8388607.0f));
 }
 
-__device__ __forceinline__ uint32_t dat_level(float g, float qmul, float S1_f, uint32_t w)
+__device__ __forceinline__ uint32_t dat_level_u1(float g, float qmul, float S1_f, float u1)
 {
-    return dat_level_bits(g, qmul, S1_f, w) & 0x007FFFFFu;
+    return dat_level_bits_u1(g, qmul, S1_f, u1) & 0x007FFFFFu;
 }
 
 // sum += sign(g) * level, from the bits of dat_level_bits: with sm = 0 or -1 (all ones) for

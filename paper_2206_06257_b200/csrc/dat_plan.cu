@@ -51,7 +51,7 @@ PhiloxKeys dat_make_keys(uint64_t seed, uint64_t step)
 }
 
 extern "C" int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64_t *layer_offsets,
-                               int num_workers, int bits, int scale_mode)
+                               int num_workers, int bits, int scale_mode, int rng_bits)
 {
     if (!out) return DAT_ERR_ARG;
     *out = nullptr;
@@ -59,6 +59,7 @@ extern "C" int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64
     if (num_workers < 1 || num_workers > DAT_MAX_WORKERS) return DAT_ERR_ARG;
     if (!(bits == 1 || bits == 2 || bits == 4 || bits == 8 || bits == 16 || bits == 32)) return DAT_ERR_BITS;
     if (scale_mode != DAT_SCALE_SHARED_MAX) return DAT_ERR_UNSUPPORTED;
+    if (rng_bits != DAT_RNG_BITS_16 && rng_bits != DAT_RNG_BITS_23) return DAT_ERR_ARG;
     if (layer_offsets[0] != 0) return DAT_ERR_LAYOUT;
     for (int64_t l = 0; l < num_layers; ++l)
         if (layer_offsets[l + 1] <= layer_offsets[l]) return DAT_ERR_LAYOUT;
@@ -76,6 +77,7 @@ extern "C" int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64
     p->M = num_workers;
     p->bits = bits;
     p->scale_mode = scale_mode;
+    p->rng_bits = rng_bits;
     p->S = (bits == 32) ? 0u : (uint32_t)((1ull << bits) - 1ull);
     try {
         p->offsets.assign(layer_offsets, layer_offsets + num_layers + 1);

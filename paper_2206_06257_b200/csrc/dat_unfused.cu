@@ -87,7 +87,7 @@ template <int BITS>
 __global__ void __launch_bounds__(DAT_THREADS)
 k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h, int64_t d,
            const float *__restrict__ qmul, uint8_t *__restrict__ levels, uint8_t *__restrict__ signs,
-           int64_t level_bytes, int64_t sign_bytes)
+           int64_t level_bytes, int64_t sign_bytes, bool rng16)
 {
     constexpr int GROUPS = DAT_TILE / 4;                     // aligned groups per tile
     constexpr int LEVEL_TILE_BYTES = DAT_TILE * BITS / 8;
@@ -114,8 +114,8 @@ k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h,
         const int64_t e0 = e_tile + 4 * (int64_t)v;
         float gv[4];
         dat_load4(g, e0, 0, d, gv);
-        uint32_t w[4];
-        dat_random_words((uint64_t)e0 >> 2, (uint32_t)worker, keys, w);
+        float u1[4];
+        dat_u1x4((uint64_t)e0, (uint32_t)worker, keys, rng16, u1);
         uint32_t lev[4], neg = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -125,7 +125,7 @@ k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h,
                 l_hi = __ldg(off + l + 1);
                 t = __ldg(qmul + l);
             }
-            lev[j] = (e < d) ? dat_level(gv[j], t, S1_f, w[j]) : 0u;
+            lev[j] = (e < d) ? dat_level_u1(gv[j], t, S1_f, u1[j]) : 0u;
             neg |= (uint32_t)(gv[j] < 0.0f) << j;
         }
         // pack the group's level bits
@@ -201,7 +201,7 @@ extern "C" int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_
     dim3 grid((unsigned)flat_tiles, (unsigned)plan->M);
 #define DAT_Q(B)                                                                                           \
     k_quantize<B><<<grid, DAT_THREADS, 0, s>>>(gp, keys, plan->d_offsets, h, plan->d, plan->d_qmul, levels, \
-                                               signs, plan->level_bytes, plan->sign_bytes)
+                                               signs, plan->level_bytes, plan->sign_bytes, plan->rng_bits == 16)
     switch (plan->bits) {
     case 1: DAT_Q(1); break;
     case 2: DAT_Q(2); break;

@@ -122,6 +122,7 @@ class Config:
     zero_grad_layers: Tuple[int, ...] = ()
     zero_param_layers: Tuple[int, ...] = ()
     seed: int = 0
+    rng_bits: int = 16                      # resolution of the quantizer's uniform number (16 or 23)
     offsets: np.ndarray = field(init=False)
 
     def __post_init__(self):

@@ -18,7 +18,7 @@ def _run_and_check(oracle, cfg, sample_layers, step=0):
     grads = synth.make_grads(cfg, step, device=dev)
     hp = hp_tuple(cfg)
     th0, mo0 = theta.clone(), mom.clone()
-    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits)
+    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits, rng_bits=cfg.rng_bits)
     try:
         cs = torch.zeros(cfg.d, dtype=torch.int32, device=dev)
         sc = torch.zeros(cfg.h, dtype=torch.float32, device=dev)
@@ -49,11 +49,11 @@ def _run_and_check(oracle, cfg, sample_layers, step=0):
         a, b = int(offs[l]), int(offs[l + 1])
         g_l = [np_of(g[a:b]) for g in grads]
         ref = oracle.step(offs, np_of(th0[a:b]), np_of(mo0[a:b]), g_l, cfg.bits, cfg.seed, step, *hp,
-                          l0=l, l1=l + 1, window=True)
+                          l0=l, l1=l + 1, window=True, rng_bits=cfg.rng_bits)
         assert ulp_diff(sc_h[l:l + 1], ref["scales"][l:l + 1]).max() <= 1
         if sc_h[l] != ref["scales"][l]:
             ref = oracle.step(offs, np_of(th0[a:b]), np_of(mo0[a:b]), g_l, cfg.bits, cfg.seed, step, *hp,
-                              l0=l, l1=l + 1, window=True, scales_in=sc_h)
+                              l0=l, l1=l + 1, window=True, scales_in=sc_h, rng_bits=cfg.rng_bits)
         assert np.array_equal(np_of(cs[a:b]), ref["code_sum"]), "layer %d code sums" % l
         assert np.array_equal(np_of(mom[a:b]).view(np.uint32), ref["mom"].view(np.uint32)), "layer %d momentum" % l
         assert_close_per_layer(np_of(theta[a:b]), ref["theta"], np.array([0, b - a]), "theta layer %d" % l)

@@ -40,11 +40,11 @@ def _random_problem(seed, sizes, M, sigma_lo=-5, sigma_hi=-1, dist="normal"):
     return offs, grads, theta, mom
 
 
-def _check_unfused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5):
+def _check_unfused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5, rng_bits=16):
     M = len(grads)
     d = int(offs[-1])
     g_dev = [torch.from_numpy(g).cuda() for g in grads]
-    with GpuPlan(api, offs, M, bits) as P:
+    with GpuPlan(api, offs, M, bits, rng_bits) as P:
         lv, sg, sc = P.alloc_message()
         api.dat_quantize(P.plan, g_dev, seed, step, lv, sg, sc)
         torch.cuda.synchronize()
@@ -54,7 +54,7 @@ def _check_unfused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=
         assert ulp_diff(sc_gpu, sc_ref).max() <= 1
         n_scale_mismatch = int((sc_gpu != sc_ref).sum())
         # S2+S3: planes bit-exact given the GPU's scales
-        level, neg = oracle.quantize(offs, grads, bits, seed, step, sc_gpu)
+        level, neg = oracle.quantize(offs, grads, bits, seed, step, sc_gpu, rng_bits=rng_bits)
         lp_ref, sp_ref = oracle_planes(oracle, level, neg, bits)
         assert np.array_equal(np_of(lv).reshape(M, -1), lp_ref)
         assert np.array_equal(np_of(sg).reshape(M, -1), sp_ref)
@@ -77,11 +77,11 @@ def _check_unfused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=
         return n_scale_mismatch
 
 
-def _check_fused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5):
+def _check_fused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5, rng_bits=16):
     M = len(grads)
     d = int(offs[-1])
     g_dev = [torch.from_numpy(g).cuda() for g in grads]
-    with GpuPlan(api, offs, M, bits) as P:
+    with GpuPlan(api, offs, M, bits, rng_bits) as P:
         th_d, mo_d = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
         cs = torch.full((d,), 777, dtype=torch.int32, device="cuda")
         norms = torch.zeros(2 * P.h, dtype=torch.float32, device="cuda")
@@ -89,12 +89,12 @@ def _check_fused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5)
         api.dat_step(P.plan, th_d, mo_d, g_dev, seed, step, hp, cs, norms, sc)
         torch.cuda.synchronize()
         assert P.status() == 0
-        ref = oracle.step(offs, theta, mom, grads, bits, seed, step, *hp)
+        ref = oracle.step(offs, theta, mom, grads, bits, seed, step, *hp, rng_bits=rng_bits)
         if bits != 32:
             sc_gpu = np_of(sc)
             assert ulp_diff(sc_gpu, ref["scales"]).max() <= 1
             if not np.array_equal(sc_gpu, ref["scales"]):        # conditional protocol: same scale bits
-                ref = oracle.step(offs, theta, mom, grads, bits, seed, step, *hp, scales_in=sc_gpu)
+                ref = oracle.step(offs, theta, mom, grads, bits, seed, step, *hp, scales_in=sc_gpu, rng_bits=rng_bits)
             assert np.array_equal(np_of(cs), ref["code_sum"])
         assert np.array_equal(np_of(mo_d).view(np.uint32), ref["mom"].view(np.uint32))
         assert ulp_diff(np_of(norms).reshape(-1, 2), ref["layer_norms"]).max() <= 1
@@ -115,28 +115,49 @@ SIZES_RAGGED = [1, 2, 3, 5, 31, 32, 33, 4096, 4097, 10, 12289, 7, 20001, 64, 819
 
 
 @pytest.mark.parametrize("bits", [1, 2, 4, 8, 16])
-def test_unfused_parity_ragged(api, oracle, bits):
+def test_unfused_parity_ragged(api, oracle, bits, rng_bits):
     offs, grads, theta, mom = _random_problem(bits, SIZES_RAGGED, 3)
-    _check_unfused(api, oracle, offs, grads, theta, mom, bits, HP)
+    _check_unfused(api, oracle, offs, grads, theta, mom, bits, HP, rng_bits=rng_bits)
 
 
 @pytest.mark.parametrize("bits", [1, 2, 4, 8, 16, 32])
-def test_fused_parity_ragged(api, oracle, bits):
+def test_fused_parity_ragged(api, oracle, bits, rng_bits):
     offs, grads, theta, mom = _random_problem(100 + bits, SIZES_RAGGED, 3)
-    _check_fused(api, oracle, offs, grads, theta, mom, bits, HP)
+    _check_fused(api, oracle, offs, grads, theta, mom, bits, HP, rng_bits=rng_bits)
 
 
 @pytest.mark.parametrize("M", [1, 2, 5, 8, 13, 32, 64])
-def test_fused_parity_worker_counts(api, oracle, M):
+def test_fused_parity_worker_counts(api, oracle, M, rng_bits):
     offs, grads, theta, mom = _random_problem(M, [1000, 5000, 3, 9000], M, dist="t3")
-    _check_fused(api, oracle, offs, grads, theta, mom, 4, HP)
+    _check_fused(api, oracle, offs, grads, theta, mom, 4, HP, rng_bits=rng_bits)
 
 
-def test_fused_equals_unfused_on_gpu(api, oracle):
+@pytest.mark.parametrize("bits", [2, 8, 16])
+def test_fused_parity_extreme_scales(api, oracle, bits, rng_bits):
+    """Layers whose norms sit at the ends of the fp32 range (the scaled form of the level
+    computation does not apply there), a layer with a single non-zero element (|g| = nu: the
+    clamp of the level is live), subnormal gradients, and ordinary layers around them."""
+    sizes = [3000, 2500, 4099, 2048, 2600, 777]
+    offs, grads, theta, mom = _random_problem(7 + bits, sizes, 3)
+    o = offs
+    def rescale(x, norm):
+        x64 = x.astype(np.float64)
+        return (x64 / np.sqrt(np.sum(x64 * x64)) * norm).astype(np.float32)
+    for i, g in enumerate(grads):
+        g[o[0]:o[1]] = rescale(g[o[0]:o[1]], 2e38 if i == 1 else 3e37)      # S / nu * 2^-b is subnormal
+        g[o[1]:o[2]] = rescale(g[o[1]:o[2]], 3e-40)                         # subnormal gradients and norm
+        g[o[2]:o[3]] = 0.0
+        g[o[2] + 1234 + i] = np.float32(-0.37 if i else 0.37)               # one element: |g| = nu
+        g[o[4]:o[5]] = rescale(g[o[4]:o[5]], 1e-29)                         # tiny but normal
+    _check_fused(api, oracle, offs, grads, theta, mom, bits, HP, rng_bits=rng_bits)
+    _check_unfused(api, oracle, offs, grads, theta, mom, bits, HP, rng_bits=rng_bits)
+
+
+def test_fused_equals_unfused_on_gpu(api, oracle, rng_bits):
     offs, grads, theta, mom = _random_problem(7, SIZES_RAGGED, 4)
     M, d = 4, int(offs[-1])
     g_dev = [torch.from_numpy(g).cuda() for g in grads]
-    with GpuPlan(api, offs, M, 8) as P:
+    with GpuPlan(api, offs, M, 8, rng_bits) as P:
         lv, sg, sc = P.alloc_message()
         gh = torch.zeros(d, dtype=torch.float32, device="cuda")
         th1, mo1 = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
