@@ -58,6 +58,17 @@ static_assert(F_NSLOT == 2, "the compute warps' loop keeps exactly two batch des
 #define F_KQ 4                                   // hand-off buffers, compute warps -> reducer, Q sums
 #define F_KN_MAX 4                               // the same for N sums (M values per warp; as many as fit)
 #define F_CTAS_PER_SM 1
+#ifndef F_Q_UNROLL
+#define F_Q_UNROLL 2                             // rows of a Q batch whose Philox chains the compiler may interleave
+#endif
+#ifndef F_N_UNROLL
+#define F_N_UNROLL 8                             // 16-byte reads of an N batch in flight per lane
+#endif
+#define F_PRAGMA(x) _Pragma(#x)
+#define F_UNROLL(n) F_PRAGMA(unroll n)
+#ifndef F_L2_HINTS
+#define F_L2_HINTS 1                             // L2 eviction policies on the asynchronous copies
+#endif
 #define F_WAIT_CYCLES (1ll << 31)                // bound of every device-side wait (about a second)
 
 enum { ITEM_N = 0u, ITEM_Q = 1u, ITEM_U = 2u, ITEM_END = 3u };
@@ -115,8 +126,8 @@ struct Batch {
     uint32_t x = 0;                              // the record's word, with the slice's mode in bits 4-5
     uint32_t aux = 0;                            // rows | chunk << 8 | last << 16
     int pos = 0;                                 // the record's index in the CTA's list (names the slot on a flush)
-    float f0 = 0.0f;                             // U: -a_l
     long long begin = 0;                         // first element of the warp's slice
+    unsigned long long w0 = 0, w1 = 0;           // the layer's result words as they stood when the batch was started
 };
 enum { MODE_EMPTY = 0u, MODE_FAST = 1u, MODE_MASKED = 2u };
 
@@ -204,9 +215,26 @@ __device__ __forceinline__ bool mbar_test_wait(unsigned long long *bar, uint32_t
 }
 // global -> shared asynchronous copy of 16 bytes per lane (both addresses 16-byte aligned);
 // the copies of a batch form one group, and a warp waits for its own groups in order.
-__device__ __forceinline__ void cp_async16(uint32_t dst_shared, const void *src)
+// `policy` is an L2 eviction policy (createpolicy): what is read for the last time should not push
+// out what is still waiting for its second pass.
+__device__ __forceinline__ void cp_async16(uint32_t dst_shared, const void *src, unsigned long long policy)
 {
+#if F_L2_HINTS
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst_shared), "l"(src), "l"(policy) : "memory");
+#else
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_shared), "l"(src) : "memory");
+#endif
+}
+struct L2Policies {
+    unsigned long long keep, normal, stream;     // evict last / normal / first
+};
+__device__ __forceinline__ L2Policies make_policies()
+{
+    L2Policies p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p.keep));
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p.normal));
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p.stream));
+    return p;
 }
 __device__ __forceinline__ void cp_async_commit()
 {
@@ -232,6 +260,12 @@ __device__ __forceinline__ unsigned long long ld_acquire64(const unsigned long l
 {
     unsigned long long v;
     asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned long long ld_relaxed64(const unsigned long long *p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p));
     return v;
 }
 __device__ __forceinline__ void st_release64(unsigned long long *p, unsigned long long v)
@@ -313,23 +347,24 @@ struct Walk {
     int pos = 0, chunk = 0;                      // next batch: record, group of workers
     int win_base = -1;                           // lane j holds record win_base + j
     uint2 win;
-    int u_layer = -1;                            // layer whose step length this warp has seen
-    float u_f = 0.0f;
+    int q_pf_layer = -1, u_pf_layer = -1;        // layers whose result words a started batch already carries
 };
 
-enum { ISSUE_OK = 1, ISSUE_NONE = 0, ISSUE_NOT_YET = -1, ISSUE_ABORT = -2 };
+enum { ISSUE_OK = 1, ISSUE_NONE = 0, ISSUE_DEFER = -1 };
 
 // Starts the warp's next batch in the slot at shared address `dst` (already offset by 16 bytes
 // per lane): every lane copies 16 bytes of each half of each row of the slice (gradient rows of
 // the batch's workers; the theta and m rows with an item's last batch), one group per batch.
-// `gl` holds, for M <= F_RB, the lane's byte pointers into the gradient buffers.  A U batch needs
-// the layer's step length first (m' of the tile was written by the tile's Q item: the result word
-// orders it); with `may_block` false one look is taken and ISSUE_NOT_YET returned when the word
-// is not there.
+// `gl` holds, for M <= F_RB, the lane's byte pointers into the gradient buffers.  Nothing here
+// waits: the first Q (U) batch of a layer takes along a relaxed read of the layer's scale (step
+// length) words, to be looked at when the batch is consumed.  A U batch may be started before its
+// layer's step length exists: the m' it copies was written by this very warp when it consumed the
+// tile's Q item (a tile's three items go to the same CTA, a slice to the same warp) -- unless that
+// Q batch is the one still waiting to be consumed (`pending_q` = its first element, else -1):
+// then ISSUE_DEFER is returned and the U batch is started after it.
 template <int NCH>
-__device__ __forceinline__ int issue_next(const FusedArgs &a, Shared &sh, Walk &w, uint32_t dst, bool may_block,
-                                          int warp_off, int lane, const char *const (&gl)[F_RB], const char *th_l,
-                                          const char *mo_l, Batch &out)
+__device__ __forceinline__ int issue_next(const FusedArgs &a, Walk &w, uint32_t dst, long long pending_q, int warp_off, int lane, const char *const (&gl)[F_RB], const char *th_l,
+                                          const char *mo_l, const L2Policies &pol, Batch &out)
 {
     if (w.pos >= w.n) return ISSUE_NONE;
     if (w.win_base != (w.pos & ~31)) {
@@ -340,20 +375,16 @@ __device__ __forceinline__ int issue_next(const FusedArgs &a, Shared &sh, Walk &
     const uint32_t kind = x & 3u;
     const int layer = (int)(x >> 8);
     const long long s0 = ((long long)y << 3) + warp_off;
-    if (kind == ITEM_U && w.u_layer != layer) {
-        const unsigned long long *p = a.flags + 3 * (long long)layer + 2;
-        if (!may_block) {
-            const unsigned long long v = ld_acquire64(p);
-            if ((uint32_t)(v >> 32) != a.epoch) return ISSUE_NOT_YET;
-            w.u_f = __uint_as_float((uint32_t)v);
-        } else {
-            PROF_T0();
-            float f[2];
-            if (!wait_words(sh, p, 1, a.epoch, a.status, f)) return ISSUE_ABORT;
-            w.u_f = f[0];
-            PROF_ADD(7);
-        }
-        w.u_layer = layer;
+    if (kind == ITEM_U && s0 == pending_q) return ISSUE_DEFER;
+    out.w0 = 0;
+    out.w1 = 0;
+    if (kind == ITEM_Q && w.q_pf_layer != layer) {
+        w.q_pf_layer = layer;
+        out.w0 = ld_relaxed64(a.flags + 3 * (long long)layer);
+        out.w1 = ld_relaxed64(a.flags + 3 * (long long)layer + 1);
+    } else if (kind == ITEM_U && w.u_pf_layer != layer) {
+        w.u_pf_layer = layer;
+        out.w0 = ld_relaxed64(a.flags + 3 * (long long)layer + 2);
     }
     uint32_t mode = MODE_FAST;
     if (!(x & REC_FAST)) {
@@ -371,23 +402,26 @@ __device__ __forceinline__ int issue_next(const FusedArgs &a, Shared &sh, Walk &
     out.x = (x & ~((3u << REC_MODE_SHIFT) | (last ? 0u : REC_FLUSH))) | (mode << REC_MODE_SHIFT);
     out.aux = (uint32_t)nr | ((uint32_t)c << 8) | (last ? 0x10000u : 0u);
     out.pos = w.pos;
-    out.f0 = w.u_f;
     out.begin = s0;
     if (mode == MODE_FAST && DAT_CHECK(s0 >= 0 && s0 + F_SLICE <= a.d && (s0 & 7) == 0 && c * F_RB + nr <= a.M, 2, s0)) {
+        // N reads a gradient tile for the first time (keep it for the Q pass), Q for the last;
+        // theta is read again by the U pass; m (Q) and m' (U) are not read again.
         const long long eb = s0 * 4;
+        const unsigned long long pg = (kind == ITEM_N) ? pol.keep : pol.stream;
 #pragma unroll
         for (int r = 0; r < F_RB; ++r) {
             if (r < nr) {
                 const char *src = (NCH == 1 ? gl[r] : reinterpret_cast<const char *>(a.gp.p[c * F_RB + r]) + lane * 16) + eb;
-                cp_async16(dst + r * F_ROW_BYTES, src);
-                cp_async16(dst + r * F_ROW_BYTES + F_ROW_BYTES / 2, src + F_ROW_BYTES / 2);
+                cp_async16(dst + r * F_ROW_BYTES, src, pg);
+                cp_async16(dst + r * F_ROW_BYTES + F_ROW_BYTES / 2, src + F_ROW_BYTES / 2, pg);
             }
         }
         if (last && kind != ITEM_N) {
-            cp_async16(dst + F_RB * F_ROW_BYTES, th_l + eb);
-            cp_async16(dst + F_RB * F_ROW_BYTES + F_ROW_BYTES / 2, th_l + eb + F_ROW_BYTES / 2);
-            cp_async16(dst + (F_RB + 1) * F_ROW_BYTES, mo_l + eb);
-            cp_async16(dst + (F_RB + 1) * F_ROW_BYTES + F_ROW_BYTES / 2, mo_l + eb + F_ROW_BYTES / 2);
+            const unsigned long long pt = (kind == ITEM_Q) ? pol.normal : pol.stream;
+            cp_async16(dst + F_RB * F_ROW_BYTES, th_l + eb, pt);
+            cp_async16(dst + F_RB * F_ROW_BYTES + F_ROW_BYTES / 2, th_l + eb + F_ROW_BYTES / 2, pt);
+            cp_async16(dst + (F_RB + 1) * F_ROW_BYTES, mo_l + eb, pol.stream);
+            cp_async16(dst + (F_RB + 1) * F_ROW_BYTES + F_ROW_BYTES / 2, mo_l + eb + F_ROW_BYTES / 2, pol.stream);
         }
     }
     cp_async_commit();                           // one group per batch, empty for slices without copies
@@ -405,7 +439,7 @@ __device__ __forceinline__ double norm_fast(const unsigned char *slot, int nr, i
     double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
     if (row < nr) {
         const unsigned char *p = slot + row * F_ROW_BYTES + (lane & 3) * (F_ROW_BYTES / 4);
-#pragma unroll
+        F_UNROLL(F_N_UNROLL)
         for (int i = 0; i < F_ROW_BYTES / 64; ++i) {
             const float4 f = lds128(p + (((i + lane) & (F_ROW_BYTES / 64 - 1)) << 4));
             s0 = fma((double)f.x, (double)f.x, s0);
@@ -452,7 +486,7 @@ template <bool IDENTITY, bool RNG16, bool FULL>
 __device__ __forceinline__ void rows_quant(const FusedArgs &a, const QuantConst &qc, const unsigned char *slot, int chunk,
                                            int nr, long long e0, int lane, float ts, float acc[8])
 {
-#pragma unroll
+    F_UNROLL(F_Q_UNROLL)
     for (int r = 0; r < F_RB; ++r) {
         if (FULL || r < nr) {
             const float4 f0 = lds128(slot + r * F_ROW_BYTES + lane * 32);
@@ -594,28 +628,28 @@ __device__ __forceinline__ void compute_warp(const FusedArgs &a, Shared &sh, uns
     const char *mo_l = reinterpret_cast<const char *>(a.mom) + lane * 16;
     const int warp_off = warp * F_SLICE;
     const uint32_t slot_u32 = smem_u32(slots) + lane * 16;
+    const L2Policies pol = make_policies();
 
     Batch cur, nxt;                              // the batch being consumed, the one in flight behind it
-    bool have_nxt = false;
     uint32_t par = 0;                            // slot of the next batch to start
+    int u_layer = -1;                            // layer whose step length this warp has seen
+    float u_f = 0.0f;
+    bool have_nxt = false;
     for (;;) {
-        // The batch to work on: started in the previous round, or started now (only then may the
-        // warp block on a step length: nothing of its own is pending that the word could need).
-        if (!have_nxt) {
+        if (!have_nxt) {                         // nothing in flight: start the batch to work on
             PROF_T0();
-            const int r = issue_next<NCH>(a, sh, w, slot_u32 + par * F_SLOT_BYTES, true, warp_off, lane, gl, th_l, mo_l, nxt);
+            const int r = issue_next<NCH>(a, w, slot_u32 + par * F_SLOT_BYTES, -1, warp_off, lane, gl, th_l, mo_l, pol, nxt);
             PROF_ADD(4);
-            if (r != ISSUE_OK) break;            // end of the list, or abort
+            if (r != ISSUE_OK) break;            // end of the list
             par ^= 1u;
         }
         cur = nxt;
         {   // start the batch after it, into the slot that the previous round has finished with
             PROF_T0();
-            const int r = issue_next<NCH>(a, sh, w, slot_u32 + par * F_SLOT_BYTES, false, warp_off, lane, gl, th_l, mo_l, nxt);
+            const long long pending_q = ((cur.x & 3u) == ITEM_Q) ? cur.begin : -1;
+            have_nxt = issue_next<NCH>(a, w, slot_u32 + par * F_SLOT_BYTES, pending_q, warp_off, lane, gl, th_l, mo_l, pol, nxt) == ISSUE_OK;
             PROF_ADD(4);
-            have_nxt = (r == ISSUE_OK);
             if (have_nxt) par ^= 1u;
-            if (r == ISSUE_ABORT) break;
         }
         { PROF_T0();
         if (have_nxt) cp_async_wait<1>(); else cp_async_wait<0>();
@@ -669,7 +703,10 @@ __device__ __forceinline__ void compute_warp(const FusedArgs &a, Shared &sh, uns
                 for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
                 if (!IDENTITY && q_layer != layer) {
                     PROF_T0();
-                    if (!wait_words(sh, a.flags + 3 * (long long)layer, 2, a.epoch, a.status, q_f)) break;
+                    if ((uint32_t)(h0.w0 >> 32) == a.epoch && (uint32_t)(h0.w1 >> 32) == a.epoch) {
+                        q_f[0] = __uint_as_float((uint32_t)h0.w0);       // the words were there when the batch was started
+                        q_f[1] = __uint_as_float((uint32_t)h0.w1);
+                    } else if (!wait_words(sh, a.flags + 3 * (long long)layer, 2, a.epoch, a.status, q_f)) break;
                     q_layer = layer;
                     ts = q_f[0] * qc.inv_two_b;
                     plain = (q_f[0] != 0.0f) && !(q_f[0] >= qc.t_min && q_f[0] <= 3.402823466e38f);
@@ -721,8 +758,20 @@ __device__ __forceinline__ void compute_warp(const FusedArgs &a, Shared &sh, uns
             PROF_ADD(2);
         } else {
             PROF_T0();
+            if (u_layer != layer) {
+                PROF_T0();
+                if ((uint32_t)(h0.w0 >> 32) == a.epoch) {
+                    u_f = __uint_as_float((uint32_t)h0.w0);
+                } else {
+                    float f[2];
+                    if (!wait_words(sh, a.flags + 3 * (long long)layer + 2, 1, a.epoch, a.status, f)) break;
+                    u_f = f[0];
+                }
+                u_layer = layer;
+                PROF_ADD(7);
+            }
             if (mode != MODE_EMPTY) {
-                const float na = h0.f0;
+                const float na = u_f;
                 float th[8], m[8];
                 load_params(a, sl, mode == MODE_FAST, e0, lo, hi, lane, th, m);
 #pragma unroll
@@ -1072,7 +1121,7 @@ static int fused_prepare(dat_plan_t *plan)
     int l2 = 0;
     cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, plan->device);
     f->window_bytes = l2 > 0 ? (int64_t)l2 / 10 * 7 : (int64_t)32 << 20;
-    f->slack = 4 * (int64_t)G;
+    f->slack = 8 * (int64_t)G;
 #ifdef DAT_PROF
     if (const char *e = getenv("DAT_FUSED_WINDOW_MB")) f->window_bytes = (int64_t)atoi(e) << 20;
     if (const char *e = getenv("DAT_FUSED_SLACK")) f->slack = atoi(e);
