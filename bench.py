@@ -30,7 +30,7 @@ UNIT = "elems/s"
 NOMINAL_HBM_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_fused_step launch, from the ncu capture
 # summarised under profiles/ (None until taken for the kernel as it stands).
-NCU_DRAM_BYTES_PER_LAUNCH = {"resnet50_b8": 2006303744 + 192066816}
+NCU_DRAM_BYTES_PER_LAUNCH = {"resnet50_b8_rng16": 1930594816 + 157463552}
 
 
 def measured_peaks():
@@ -353,7 +353,7 @@ def run_gpu(args):
         else:
             algo_bytes = (4 * cfg.M + 16) * cfg.d
         achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-        traffic = None if unfused else NCU_DRAM_BYTES_PER_LAUNCH.get("%s_b%d" % (cfg.name, cfg.bits))
+        traffic = None if unfused else NCU_DRAM_BYTES_PER_LAUNCH.get("%s_b%d_rng%d" % (cfg.name, cfg.bits, cfg.rng_bits))
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": region_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
