@@ -341,7 +341,7 @@ def run_gpu(args):
         layers, what = oracle_layer_sample(cfg, int(n_cal / t_cal * 15.0))
         t_or, n_or = time_oracle(cfg, th_c.numpy(), mo_c.numpy(), g_c, layers, threads)
         reps = 1
-        while (reps * t_or * threads) < 20.0 and reps < 50:            # about 20 core-seconds of oracle work
+        while t_or * threads < 20.0 and reps < 50:                      # about 20 core-seconds of oracle work
             t_k, n_k = time_oracle(cfg, th_c.numpy(), mo_c.numpy(), g_c, layers, threads, step=reps)
             t_or, n_or, reps = t_or + t_k, n_or + n_k, reps + 1
         cpu = {"value": n_or / t_or, "unit": UNIT, "cores": threads, "kind": "oracle",

@@ -11,9 +11,11 @@
 //   U  (needs a_l) theta -= a_l * m'                                                    [Eq. 3]
 //
 // The host lays the items out as one list in which N runs ahead of Q and Q ahead of U by just
-// enough for the dependencies.  Within a layer the Q items walk the tiles in the opposite
-// direction of the N items (and the U items in the opposite direction of the Q items), so that a
-// layer larger than L2 still finds its most recently read part there.  A tile's three items go
+// enough for the dependencies; layers are taken largest first, so that the end of the list,
+// where nothing is left to overlap with, belongs to the small ones.  Within a layer the Q items
+// walk the tiles in the opposite direction of the N items (and the U items in the opposite
+// direction of the Q items), so that a layer larger than L2 still finds its most recently read
+// part there.  A tile's three items go
 // to the same CTA (tile index mod G; one CTA per SM); every CTA takes its items in list order.
 //
 // Inside a CTA every COMPUTE warp owns a fixed 256-element slice of each tile and feeds itself:
@@ -24,7 +26,7 @@
 // their running sums (squares per worker; theta^2 and m'^2) stay in registers across the tiles
 // of a layer and are handed to the CTA's REDUCER warp only when the CTA's contribution to the
 // layer is due.  The reducer warp adds the warps' sums in a fixed order, publishes the CTA's
-// contribution and counts it; the reducer of the layer's owner CTA (layer mod G) watches the
+// contribution and counts it; the reducer of the layer's owner CTA (its position in the processing order, mod G) watches the
 // count and, when it is complete, reduces all contributions in a fixed order and releases the
 // layer's result words.  Slices that touch a layer boundary are read with ordinary masked loads.
 //
@@ -66,6 +68,9 @@ static_assert(F_NSLOT == 2, "the compute warps' loop keeps exactly two batch des
 #endif
 #define F_PRAGMA(x) _Pragma(#x)
 #define F_UNROLL(n) F_PRAGMA(unroll n)
+#ifndef F_LARGEST_FIRST
+#define F_LARGEST_FIRST 1                        // process the layers in descending size
+#endif
 #ifndef F_L2_HINTS
 #define F_L2_HINTS 1                             // L2 eviction policies on the asynchronous copies
 #endif
@@ -81,6 +86,7 @@ struct FusedSchedule {
     int64_t n_items = 0;
     int64_t *d_slot_base = nullptr;   // h+1, partial-sum slots per layer
     uint32_t *d_expect = nullptr;     // 2h: contributions expected per layer (N, Q)
+    int *d_order = nullptr;           // h: processing order, position -> layer
     uint32_t *d_sync = nullptr;       // cnt_n[h] cnt_q[h] done[1]
     unsigned long long *d_flags = nullptr;   // per layer: (epoch, S/nu) (epoch, nu/(S*M)) (epoch, -a_l)
     double *d_npart = nullptr;        // slots * M
@@ -103,6 +109,7 @@ struct FusedArgs {
     const uint2 *recs;
     const uint32_t *rec_slots;                   // per record: partial-sum slot (N, Q items)
     const uint32_t *expect;
+    const int *order;                            // processing order: position -> layer
     double *npart, *qpart;
     uint32_t *cnt_n, *cnt_q, *done, *status;
     unsigned long long *flags;                   // 3 words per layer, each (epoch << 32) | float bits
@@ -823,7 +830,7 @@ __device__ __forceinline__ void finish_norm(const FusedArgs &a, const double *re
     if (lane == 0) red_add(a.cnt_n + layer);
 }
 
-// The owner of a layer (CTA layer mod G) finalises it once every contribution has arrived:
+// The owner of a layer (CTA = its position in the processing order mod G) finalises it once every contribution has arrived:
 // all contributions are reduced in a fixed order and the layer's scale is published.
 __device__ __forceinline__ void finalize_norm(const FusedArgs &a, int layer, int lane)
 {
@@ -910,19 +917,22 @@ __device__ __forceinline__ void finalize_quant(const FusedArgs &a, int layer, in
 }
 
 // Serves both hand-off rings in turn (non-blocking tests) and finalises the layers this CTA owns
-// (layer mod G == CTA) as their contribution counts fill up, until both rings have said END and
+// (position mod G == CTA) as their contribution counts fill up, until both rings have said END and
 // every owned layer is done.
 __device__ __forceinline__ void reducer(const FusedArgs &a, Shared &sh, const double *red_n, bool have_norm)
 {
     const int lane = threadIdx.x & 31;
     uint32_t kn = 0, kq = 0;
     bool done_n = !have_norm, done_q = false;
-    int own_n = have_norm ? (int)blockIdx.x : a.h, own_q = (int)blockIdx.x;     // next owned layer to finalise
-    uint32_t want_n = (own_n < a.h) ? __ldg(a.expect + own_n) : 0u;
-    uint32_t want_q = (own_q < a.h) ? __ldg(a.expect + a.h + own_q) : 0u;
+    // Ownership follows the processing order: this CTA owns the layers at positions c, c + G, ...
+    // of that order, so the next one to complete is always the one it looks at.
+    int pos_n = have_norm ? (int)blockIdx.x : a.h, pos_q = (int)blockIdx.x;
+    int own_n = (pos_n < a.h) ? __ldg(a.order + pos_n) : 0, own_q = (pos_q < a.h) ? __ldg(a.order + pos_q) : 0;
+    uint32_t want_n = (pos_n < a.h) ? __ldg(a.expect + own_n) : 0u;
+    uint32_t want_q = (pos_q < a.h) ? __ldg(a.expect + a.h + own_q) : 0u;
     long long t_last = clock64();
     uint32_t round = 0;
-    while (!(done_n && done_q) || own_n < a.h || own_q < a.h) {
+    while (!(done_n && done_q) || pos_n < a.h || pos_q < a.h) {
         bool progress = false;
         if (!done_n) {
             const uint32_t b = kn % (uint32_t)a.kn;
@@ -956,19 +966,21 @@ __device__ __forceinline__ void reducer(const FusedArgs &a, Shared &sh, const do
         }
         // owned layers: look at the counts when idle, and every few rounds when busy
         if (!progress || (++round & 3u) == 0u) {
-            if (own_n < a.h && ld_acquire(a.cnt_n + own_n) == want_n) {
+            if (pos_n < a.h && ld_acquire(a.cnt_n + own_n) == want_n) {
                 PROF_T0();
                 finalize_norm(a, own_n, lane);
-                own_n += (int)gridDim.x;
-                want_n = (own_n < a.h) ? __ldg(a.expect + own_n) : 0u;
+                pos_n += (int)gridDim.x;
+                own_n = (pos_n < a.h) ? __ldg(a.order + pos_n) : 0;
+                want_n = (pos_n < a.h) ? __ldg(a.expect + own_n) : 0u;
                 progress = true;
                 PROF_ADD(5);
             }
-            if (own_q < a.h && ld_acquire(a.cnt_q + own_q) == want_q) {
+            if (pos_q < a.h && ld_acquire(a.cnt_q + own_q) == want_q) {
                 PROF_T0();
                 finalize_quant(a, own_q, lane);
-                own_q += (int)gridDim.x;
-                want_q = (own_q < a.h) ? __ldg(a.expect + a.h + own_q) : 0u;
+                pos_q += (int)gridDim.x;
+                own_q = (pos_q < a.h) ? __ldg(a.order + pos_q) : 0;
+                want_q = (pos_q < a.h) ? __ldg(a.expect + a.h + own_q) : 0u;
                 progress = true;
                 PROF_ADD(5);
             }
@@ -1039,7 +1051,7 @@ void dat_fused_destroy(dat_plan_t *plan)
 {
     FusedSchedule *f = plan->fused;
     if (!f) return;
-    void *ptrs[] = {f->d_recs, f->d_rec_slots, f->d_cta_first, f->d_slot_base, f->d_expect, f->d_sync, f->d_flags, f->d_npart, f->d_qpart};
+    void *ptrs[] = {f->d_recs, f->d_rec_slots, f->d_order, f->d_cta_first, f->d_slot_base, f->d_expect, f->d_sync, f->d_flags, f->d_npart, f->d_qpart};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     delete f;
@@ -1131,14 +1143,23 @@ static int fused_prepare(dat_plan_t *plan)
     std::vector<int64_t> tile_base(h + 1), slot_base(h + 1);
     std::vector<uint32_t> expect(2 * h, 0);
     try {
+        // Layers are processed largest first (results do not depend on the order): the end of the
+        // list, where Q and U have no N left to overlap with, then belongs to the small layers.
+        std::vector<int64_t> ntiles(h), order(h);
         int64_t nt = 0, ns = 0;
         for (int64_t l = 0; l < h; ++l) {
-            tile_base[l] = nt;
             slot_base[l] = ns;
             const int64_t a = plan->offsets[l] & ~(int64_t)7;
-            const int64_t n = (plan->offsets[l + 1] - a + FT - 1) / FT;
-            nt += n;
-            ns += std::min<int64_t>(n, G);
+            ntiles[l] = (plan->offsets[l + 1] - a + FT - 1) / FT;
+            ns += std::min<int64_t>(ntiles[l], G);
+            order[l] = l;
+        }
+#if F_LARGEST_FIRST
+        std::stable_sort(order.begin(), order.end(), [&](int64_t x, int64_t y) { return ntiles[x] > ntiles[y]; });
+#endif
+        for (int64_t k = 0; k < h; ++k) {           // tile_base is indexed by position in the processing order
+            tile_base[k] = nt;
+            nt += ntiles[order[k]];
         }
         tile_base[h] = nt;
         slot_base[h] = ns;
@@ -1172,22 +1193,23 @@ static int fused_prepare(dat_plan_t *plan)
             const int64_t tile = items[i] & ITEM_TILE_MASK;
             const int cta = (int)(tile % G);
             const int64_t r = cta_first[cta] + fill[cta]++;
-            const int l = (int)layer_of(tile);
+            const int64_t k_pos = layer_of(tile);
+            const int l = (int)order[k_pos];
             const int64_t lo = plan->offsets[l], hi = plan->offsets[l + 1];
-            const int64_t begin = (lo & ~(int64_t)7) + (tile - tile_base[l]) * FT;
+            const int64_t begin = (lo & ~(int64_t)7) + (tile - tile_base[k_pos]) * FT;
             const bool fast = begin >= lo && begin + FT <= hi;
             uint32_t info = type | (fast ? REC_FAST : 0u) | ((uint32_t)l << 8);
             uint32_t slot = 0;
             if (type != ITEM_U) {
                 const int k = (type == ITEM_N) ? 0 : 1;
-                const int64_t ntl = tile_base[l + 1] - tile_base[l];
+                const int64_t ntl = ntiles[l];
                 if (last_rec[k][cta] >= 0 && last_layer[k][cta] != l) {     // the CTA moved on to another layer
                     recs[last_rec[k][cta]].x |= REC_FLUSH;
                     expect[k * h + last_layer[k][cta]]++;
                     last_rec[k][cta] = -1;
                 }
                 if (ntl <= G) {
-                    slot = (uint32_t)(slot_base[l] + (tile - tile_base[l]));
+                    slot = (uint32_t)(slot_base[l] + (tile - tile_base[k_pos]));
                     info |= REC_FLUSH;
                     expect[k * h + l]++;
                 } else {
@@ -1210,6 +1232,7 @@ static int fused_prepare(dat_plan_t *plan)
         if (e == cudaSuccess) e = upload(&f->d_cta_first, cta_first);
         if (e == cudaSuccess) e = upload(&f->d_slot_base, slot_base);
         if (e == cudaSuccess) e = upload(&f->d_expect, expect);
+        if (e == cudaSuccess) { std::vector<int> order32(order.begin(), order.end()); e = upload(&f->d_order, order32); }
         if (e == cudaSuccess) e = cudaMalloc((void **)&f->d_sync, f->sync_words * 4);
         if (e == cudaSuccess) e = cudaMalloc((void **)&f->d_flags, (size_t)h * 3 * 8);
         if (e == cudaSuccess) e = cudaMalloc((void **)&f->d_npart, (size_t)ns * plan->M * 8);
@@ -1258,6 +1281,7 @@ extern "C" int dat_step(dat_plan_t *plan, float *theta, float *mom, const float 
     a.recs = f->d_recs;
     a.rec_slots = f->d_rec_slots;
     a.expect = f->d_expect;
+    a.order = f->d_order;
     a.npart = f->d_npart;
     a.qpart = f->d_qpart;
     const size_t h = (size_t)plan->h;
