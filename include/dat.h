@@ -61,8 +61,13 @@ typedef struct dat_hparams {
 /* Which l2 norm scales the quantizer of Eq. rand_q.
  * SHARED_MAX: nu_l = max_i ||g_l^(i)||_2, one value per layer shared by all workers, so that
  *             the workers' integer codes lie on one grid and Eq. grad_agg becomes an integer sum
- *             followed by one scaling.  (Q stays unbiased for any nu >= max|g|.)              */
-enum { DAT_SCALE_SHARED_MAX = 0 };
+ *             followed by one scaling.  (Q stays unbiased for any nu >= max|g|.)
+ * PER_WORKER: nu_{i,l} = ||g_l^(i)||_2, every worker's own norm, as Eq. rand_q and Eq. grad_agg
+ *             are written: g_hat = (1/M) sum_i nu_{i,l} * sign * level / S, summed in fp32.  The
+ *             message then carries M*h norms (index i*h + l), and no integer code sum exists.
+ *             Available in the separate calls (dat_quantize, dat_aggregate); the fused dat_step
+ *             sums integer codes and answers DAT_ERR_UNSUPPORTED for such a plan.              */
+enum { DAT_SCALE_SHARED_MAX = 0, DAT_SCALE_PER_WORKER = 1 };
 
 /* Resolution of the quantizer's uniform number (see dat_plan_create). */
 enum { DAT_RNG_BITS_16 = 16, DAT_RNG_BITS_23 = 23 };
@@ -96,7 +101,7 @@ enum {
  *   num_workers    M in [1, DAT_MAX_WORKERS].
  *   bits           b in {1,2,4,8,16}, or 32 = no quantisation (Q is the identity and the
  *                  aggregate is the plain worker average).
- *   scale_mode     DAT_SCALE_SHARED_MAX.
+ *   scale_mode     DAT_SCALE_SHARED_MAX or DAT_SCALE_PER_WORKER.
  *   rng_bits       resolution of the uniform number u of the stochastic rounding (Eq. xi; the
  *                  paper fixes neither generator nor resolution).  Randomness is Philox4x32-10
  *                  keyed on (seed, step, worker, element):
@@ -119,7 +124,7 @@ int dat_plan_destroy(dat_plan_t *plan);
 /* Sizes of the caller-owned buffers of the unfused calls (any output pointer may be NULL):
  *   level_bytes_per_worker  bytes of one worker's level plane: ceil(d*b/8) rounded up to 16
  *   sign_bytes_per_worker   bytes of one worker's sign plane:  ceil(d/8)   rounded up to 16
- *   num_scales              number of fp32 norms in the message (h)
+ *   num_scales              number of fp32 norms in the message (h; M*h with per-worker scales)
  *   workspace_bytes         device bytes the plan itself holds
  * Together: 32 bits per norm + d sign bits + b*d level bits per worker -- the
  * "(32 + d + b d) bits" message of the paper's quantizer, with one norm per layer.            */
@@ -141,8 +146,8 @@ int dat_plan_sizes(const dat_plan_t *plan, int64_t *level_bytes_per_worker,
  *              (b = 16: a little-endian uint16).  Padding bytes are written as zero.
  *   signs      device, M * sign_bytes_per_worker bytes, written: bit (e mod 8) of byte
  *              floor(e/8), 1 = negative.
- *   scales     device fp32[h], written: nu_l.
- *   scales_in  device fp32[h] or NULL.  If given, these norms are used instead of computing
+ *   scales     device fp32[num_scales], written: nu_l (per-worker scales: nu_{i,l} at i*h + l).
+ *   scales_in  device fp32[num_scales] or NULL.  If given, these norms are used instead of computing
  *              ||g_l^(i)||_2 (and are copied to `scales`); may alias `scales`.
  * Errors: ARG, ALIGN, BITS (b = 32 has no codes), CUDA.
  * ------------------------------------------------------------------------------------------- */
@@ -154,7 +159,9 @@ int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_t seed, uin
  * dat_aggregate -- Algorithm A1 Step 9, Eq. grad_agg, on the packed messages:
  *   sum_e = sum_i (sign ? -level : level)  (exact, int32);  g_hat_e = sum_e * (nu_l / (S*M)).
  *   levels, signs, scales   device, as written by dat_quantize, read-only.
- *   code_sum                device int32[d] or NULL; written if given.
+ *   code_sum                device int32[d] or NULL; written if given.  With per-worker scales
+ *                           g_hat_e = (sum_i fma(nu_{i,l}, signed level_i, .)) / (S*M) in ascending
+ *                           worker order, and code_sum must be NULL (DAT_ERR_ARG).
  *   g_hat                   device fp32[d], written.
  * Errors: ARG, ALIGN, BITS (b = 32), CUDA.
  * ------------------------------------------------------------------------------------------- */

@@ -21,7 +21,7 @@ if not os.path.exists(LIB_PATH):
 _lib = C.CDLL(LIB_PATH)
 
 DAT_MAX_WORKERS = 64
-DAT_SCALE_SHARED_MAX = 0
+DAT_SCALE_SHARED_MAX, DAT_SCALE_PER_WORKER = 0, 1
 DAT_RNG_BITS_16, DAT_RNG_BITS_23 = 16, 23
 DAT_OK, DAT_ERR_ARG, DAT_ERR_ALIGN, DAT_ERR_BITS = 0, -1, -2, -3
 DAT_ERR_LAYOUT, DAT_ERR_CUDA, DAT_ERR_NOMEM, DAT_ERR_UNSUPPORTED, DAT_ERR_TOO_LARGE = -4, -5, -6, -7, -8

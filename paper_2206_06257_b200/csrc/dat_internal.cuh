@@ -44,7 +44,7 @@ struct dat_plan {
     double *d_partials = nullptr;      // n_tiles * max(M,2)
     float *d_worker_norms = nullptr;   // M*h
     float *d_scales = nullptr;         // h     nu_l (fused path / scratch)
-    float *d_qmul = nullptr;           // h     S/nu_l (0 if nu_l = 0)
+    float *d_qmul = nullptr;           // h (shared scale) or M*h (per-worker scales): S/nu (0 if nu = 0)
     float *d_dq = nullptr;             // h     nu_l/(S*M)
     float *d_step_a = nullptr;         // h     lr * tau/||u||
     float *d_norms = nullptr;          // 2h

@@ -58,7 +58,7 @@ extern "C" int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64
     if (!layer_offsets || num_layers < 1 || num_layers > (1 << 24)) return DAT_ERR_ARG;
     if (num_workers < 1 || num_workers > DAT_MAX_WORKERS) return DAT_ERR_ARG;
     if (!(bits == 1 || bits == 2 || bits == 4 || bits == 8 || bits == 16 || bits == 32)) return DAT_ERR_BITS;
-    if (scale_mode != DAT_SCALE_SHARED_MAX) return DAT_ERR_UNSUPPORTED;
+    if (scale_mode != DAT_SCALE_SHARED_MAX && scale_mode != DAT_SCALE_PER_WORKER) return DAT_ERR_ARG;
     if (rng_bits != DAT_RNG_BITS_16 && rng_bits != DAT_RNG_BITS_23) return DAT_ERR_ARG;
     if (layer_offsets[0] != 0) return DAT_ERR_LAYOUT;
     for (int64_t l = 0; l < num_layers; ++l)
@@ -102,7 +102,7 @@ extern "C" int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64
     const size_t o_off = take(h1 * 8), o_tb = take(h1 * 8);
     const size_t o_part = take((size_t)nt * (size_t)(num_workers > 2 ? num_workers : 2) * 8);
     const size_t o_wn = take((size_t)num_workers * h * 4);
-    const size_t o_sc = take(h * 4), o_qm = take(h * 4), o_dq = take(h * 4), o_sa = take(h * 4);
+    const size_t o_sc = take(h * 4), o_qm = take((size_t)num_workers * h * 4), o_dq = take(h * 4), o_sa = take(h * 4);
     const size_t o_nr = take(2 * h * 4), o_st = take(256);
     p->ws_bytes = off;
     e = cudaMalloc((void **)&p->ws, p->ws_bytes);
@@ -154,7 +154,7 @@ extern "C" int dat_plan_sizes(const dat_plan_t *plan, int64_t *level_bytes_per_w
     if (!plan) return DAT_ERR_ARG;
     if (level_bytes_per_worker) *level_bytes_per_worker = plan->level_bytes;
     if (sign_bytes_per_worker) *sign_bytes_per_worker = plan->sign_bytes;
-    if (num_scales) *num_scales = plan->h;
+    if (num_scales) *num_scales = (plan->scale_mode == DAT_SCALE_PER_WORKER) ? plan->h * plan->M : plan->h;
     if (workspace_bytes) *workspace_bytes = (int64_t)plan->ws_bytes;
     return DAT_OK;
 }

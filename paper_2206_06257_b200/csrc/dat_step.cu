@@ -1259,6 +1259,7 @@ extern "C" int dat_step(dat_plan_t *plan, float *theta, float *mom, const float 
     int rc = dat_check_plan(plan);
     if (rc != DAT_OK) return rc;
     if (!theta || !mom || !hp) return DAT_ERR_ARG;
+    if (plan->scale_mode != DAT_SCALE_SHARED_MAX && plan->bits != 32) return DAT_ERR_UNSUPPORTED;   // the fused sweep sums integer codes
     if (step >> 32) return DAT_ERR_ARG;
     if (!dat_aligned16(theta) || !dat_aligned16(mom) || (code_sum_out && !dat_aligned16(code_sum_out)) ||
         (layer_norms_out && !dat_aligned16(layer_norms_out)) || (scales_out && !dat_aligned16(scales_out)))

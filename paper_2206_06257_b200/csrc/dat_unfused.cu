@@ -36,7 +36,7 @@ k_sumsq_partial(GradPtrs gp, const int64_t *__restrict__ off, const int64_t *__r
 __global__ void __launch_bounds__(DAT_THREADS)
 k_scales_finalize(const int64_t *__restrict__ tile_base, int h, int M, float S_f,
                   const double *__restrict__ partials, float *__restrict__ worker_norms,
-                  float *__restrict__ scales, float *__restrict__ qmul, uint32_t *status)
+                  float *__restrict__ scales, float *__restrict__ qmul, uint32_t *status, bool per_worker)
 {
     __shared__ float s_norm[DAT_MAX_WORKERS];
     const int l = blockIdx.x;
@@ -60,8 +60,16 @@ k_scales_finalize(const int64_t *__restrict__ tile_base, int h, int M, float S_f
             bad |= !isfinite(s_norm[i]);
             nu = (s_norm[i] > nu) ? s_norm[i] : nu;
         }
-        scales[l] = nu;
-        qmul[l] = (nu == 0.0f) ? 0.0f : S_f / nu;
+        if (per_worker) {
+            // every worker keeps its own norm (Eq. rand_q as written): index i*h + l
+            for (int i = 0; i < M; ++i) {
+                scales[(int64_t)i * h + l] = s_norm[i];
+                qmul[(int64_t)i * h + l] = (s_norm[i] == 0.0f) ? 0.0f : S_f / s_norm[i];
+            }
+        } else {
+            scales[l] = nu;
+            qmul[l] = (nu == 0.0f) ? 0.0f : S_f / nu;
+        }
         if (bad) atomicOr(status, DAT_STATUS_NONFINITE);
     }
 }
@@ -86,8 +94,8 @@ __global__ void k_qmul_from_scales(int h, float S_f, const float *__restrict__ s
 template <int BITS>
 __global__ void __launch_bounds__(DAT_THREADS)
 k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h, int64_t d,
-           const float *__restrict__ qmul, uint8_t *__restrict__ levels, uint8_t *__restrict__ signs,
-           int64_t level_bytes, int64_t sign_bytes, bool rng16)
+           const float *__restrict__ qmul_all, uint8_t *__restrict__ levels, uint8_t *__restrict__ signs,
+           int64_t level_bytes, int64_t sign_bytes, bool rng16, bool per_worker)
 {
     constexpr int GROUPS = DAT_TILE / 4;                     // aligned groups per tile
     constexpr int LEVEL_TILE_BYTES = DAT_TILE * BITS / 8;
@@ -100,6 +108,7 @@ k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h,
     const int worker = blockIdx.y;
     const int64_t e_tile = tile * DAT_TILE;
     const float *__restrict__ g = gp.p[worker];
+    const float *__restrict__ qmul = qmul_all + (per_worker ? (int64_t)worker * h : 0);
     const float S1_f = (float)(1u << BITS);                  // S + 1
 
     if (threadIdx.x == 0) s_first = dat_find(off, h, e_tile);
@@ -182,10 +191,12 @@ extern "C" int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_
     cudaStream_t s = (cudaStream_t)stream;
     const int h = (int)plan->h;
     const float S_f = (float)plan->S;
+    const bool per_worker = (plan->scale_mode == DAT_SCALE_PER_WORKER);
+    const int n_scales = per_worker ? h * plan->M : h;
     if (scales_in) {
         if (scales_in != scales)
-            DAT_CUDA(plan, cudaMemcpyAsync(scales, scales_in, (size_t)h * 4, cudaMemcpyDeviceToDevice, s));
-        k_qmul_from_scales<<<(h + 255) / 256, 256, 0, s>>>(h, S_f, scales, plan->d_qmul, plan->d_status);
+            DAT_CUDA(plan, cudaMemcpyAsync(scales, scales_in, (size_t)n_scales * 4, cudaMemcpyDeviceToDevice, s));
+        k_qmul_from_scales<<<(n_scales + 255) / 256, 256, 0, s>>>(n_scales, S_f, scales, plan->d_qmul, plan->d_status);
         DAT_LAUNCHED(plan);
     } else {
         dim3 grid((unsigned)plan->n_tiles, (unsigned)plan->M);
@@ -193,7 +204,7 @@ extern "C" int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_
                                                      plan->d_partials);
         DAT_LAUNCHED(plan);
         k_scales_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base, h, plan->M, S_f, plan->d_partials,
-                                                    plan->d_worker_norms, scales, plan->d_qmul, plan->d_status);
+                                                    plan->d_worker_norms, scales, plan->d_qmul, plan->d_status, per_worker);
         DAT_LAUNCHED(plan);
     }
     const PhiloxKeys keys = dat_make_keys(seed, step);
@@ -201,7 +212,7 @@ extern "C" int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_
     dim3 grid((unsigned)flat_tiles, (unsigned)plan->M);
 #define DAT_Q(B)                                                                                           \
     k_quantize<B><<<grid, DAT_THREADS, 0, s>>>(gp, keys, plan->d_offsets, h, plan->d, plan->d_qmul, levels, \
-                                               signs, plan->level_bytes, plan->sign_bytes, plan->rng_bits == 16)
+                                               signs, plan->level_bytes, plan->sign_bytes, plan->rng_bits == 16, per_worker)
     switch (plan->bits) {
     case 1: DAT_Q(1); break;
     case 2: DAT_Q(2); break;
@@ -299,6 +310,62 @@ k_aggregate(const uint8_t *__restrict__ levels, const uint8_t *__restrict__ sign
     }
 }
 
+// The same with one norm per worker (Eq. grad_agg as written): no integer sum exists;
+// g_hat = (sum_i nu_{i,l} * signed level_i) / (S*M), accumulated in fp32 with one fused
+// multiply-add per worker, in ascending worker order.
+template <int BITS>
+__global__ void __launch_bounds__(DAT_THREADS)
+k_aggregate_per_worker(const uint8_t *__restrict__ levels, const uint8_t *__restrict__ signs, int64_t level_bytes,
+                       int64_t sign_bytes, int M, const int64_t *__restrict__ off, int h, int64_t d,
+                       const float *__restrict__ scales, float SM_f, float *__restrict__ g_hat)
+{
+    __shared__ int s_first;
+    const int64_t e_blk = (int64_t)blockIdx.x * (DAT_THREADS * 8);
+    if (threadIdx.x == 0) s_first = dat_find(off, h, e_blk);
+    __syncthreads();
+    const int64_t e0 = e_blk + 8 * (int64_t)threadIdx.x;
+    if (e0 >= d) return;
+    int lidx[8];
+    {
+        int l = s_first;
+        int64_t l_hi = __ldg(off + l + 1);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            while (e0 + j >= l_hi && l + 1 < h) {
+                ++l;
+                l_hi = __ldg(off + l + 1);
+            }
+            lidx[j] = l;
+        }
+    }
+    const bool one_layer = (lidx[0] == lidx[7]);
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+    for (int i = 0; i < M; ++i) {
+        uint32_t lev[8];
+        dat_unpack8<BITS>(levels + (int64_t)i * level_bytes, e0, lev);
+        const uint32_t sg = signs[(int64_t)i * sign_bytes + (e0 >> 3)];
+        const float *__restrict__ nu_i = scales + (int64_t)i * h;
+        const float nu0 = __ldg(nu_i + lidx[0]);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float code = ((sg >> j) & 1u) ? -(float)lev[j] : (float)lev[j];
+            const float nu = one_layer ? nu0 : __ldg(nu_i + lidx[j]);
+            acc[j] = __fmaf_rn(nu, code, acc[j]);
+        }
+    }
+    float out[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) out[j] = acc[j] / SM_f;
+    if (e0 + 8 <= d) {
+        reinterpret_cast<float4 *>(g_hat + e0)[0] = make_float4(out[0], out[1], out[2], out[3]);
+        reinterpret_cast<float4 *>(g_hat + e0)[1] = make_float4(out[4], out[5], out[6], out[7]);
+    } else {
+        for (int j = 0; j < 8 && e0 + j < d; ++j) g_hat[e0 + j] = out[j];
+    }
+}
+
 extern "C" int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint8_t *signs,
                              const float *scales, int32_t *code_sum, float *g_hat, void *stream)
 {
@@ -312,9 +379,25 @@ extern "C" int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint
     cudaStream_t s = (cudaStream_t)stream;
     const int h = (int)plan->h;
     const float SM_f = (float)((uint64_t)plan->S * (uint64_t)plan->M);
+    const unsigned grid = (unsigned)((plan->d + DAT_THREADS * 8 - 1) / (DAT_THREADS * 8));
+    if (plan->scale_mode == DAT_SCALE_PER_WORKER) {
+        if (code_sum) return DAT_ERR_ARG;        // differently scaled codes have no integer sum
+#define DAT_APW(B)                                                                                                  \
+    k_aggregate_per_worker<B><<<grid, DAT_THREADS, 0, s>>>(levels, signs, plan->level_bytes, plan->sign_bytes, plan->M, \
+                                                           plan->d_offsets, h, plan->d, scales, SM_f, g_hat)
+        switch (plan->bits) {
+        case 1: DAT_APW(1); break;
+        case 2: DAT_APW(2); break;
+        case 4: DAT_APW(4); break;
+        case 8: DAT_APW(8); break;
+        default: DAT_APW(16); break;
+        }
+#undef DAT_APW
+        DAT_LAUNCHED(plan);
+        return DAT_OK;
+    }
     k_dq_from_scales<<<(h + 255) / 256, 256, 0, s>>>(h, SM_f, scales, plan->d_dq);
     DAT_LAUNCHED(plan);
-    const unsigned grid = (unsigned)((plan->d + DAT_THREADS * 8 - 1) / (DAT_THREADS * 8));
 #define DAT_A(B)                                                                                         \
     k_aggregate<B><<<grid, DAT_THREADS, 0, s>>>(levels, signs, plan->level_bytes, plan->sign_bytes, plan->M, \
                                                 plan->d_offsets, h, plan->d, plan->d_dq, code_sum, g_hat)

@@ -42,13 +42,13 @@ def np_of(t):
 class GpuPlan:
     """Plan + the caller-owned buffers of the unfused calls."""
 
-    def __init__(self, api, offsets, M, bits, rng_bits=16):
+    def __init__(self, api, offsets, M, bits, rng_bits=16, scale_mode=0):
         self.api = api
         self.offsets = np.asarray(offsets, dtype=np.int64)
         self.M, self.bits = M, bits
         self.h = len(self.offsets) - 1
         self.d = int(self.offsets[-1])
-        self.plan = api.dat_plan_create(self.offsets, M, bits, rng_bits=rng_bits)
+        self.plan = api.dat_plan_create(self.offsets, M, bits, scale_mode=scale_mode, rng_bits=rng_bits)
         self.level_bytes, self.sign_bytes, self.num_scales, self.ws = api.dat_plan_sizes(self.plan)
 
     def close(self):

@@ -120,6 +120,52 @@ def test_unfused_parity_ragged(api, oracle, bits, rng_bits):
     _check_unfused(api, oracle, offs, grads, theta, mom, bits, HP, rng_bits=rng_bits)
 
 
+def _check_unfused_per_worker(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5, rng_bits=16):
+    """The paper-literal quantizer (one norm per worker, Eq. rand_q) and Eq. grad_agg summed in fp32."""
+    M = len(grads)
+    d = int(offs[-1])
+    h = len(offs) - 1
+    g_dev = [torch.from_numpy(g).cuda() for g in grads]
+    with GpuPlan(api, offs, M, bits, rng_bits, scale_mode=api.DAT_SCALE_PER_WORKER) as P:
+        assert P.num_scales == M * h
+        lv, sg, sc = P.alloc_message()
+        api.dat_quantize(P.plan, g_dev, seed, step, lv, sg, sc)
+        torch.cuda.synchronize()
+        sc_gpu = np_of(sc).reshape(M, h)
+        sc_ref = oracle.scales(oracle.worker_norms(offs, grads), oracle.SCALE_PER_WORKER)
+        assert ulp_diff(sc_gpu, sc_ref).max() <= 1
+        level, neg = oracle.quantize(offs, grads, bits, seed, step, sc_gpu, oracle.SCALE_PER_WORKER, rng_bits=rng_bits)
+        lp_ref, sp_ref = oracle_planes(oracle, level, neg, bits)
+        assert np.array_equal(np_of(lv).reshape(M, -1), lp_ref)
+        assert np.array_equal(np_of(sg).reshape(M, -1), sp_ref)
+        gh = torch.zeros(d, dtype=torch.float32, device="cuda")
+        api.dat_aggregate(P.plan, lv, sg, sc, None, gh)
+        _, gh_ref = oracle.aggregate(offs, level, neg, sc_gpu, bits, oracle.SCALE_PER_WORKER)
+        assert np.array_equal(np_of(gh).view(np.uint32), gh_ref.view(np.uint32))
+        th_d, mo_d = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        api.dat_lalr_step(P.plan, th_d, mo_d, gh, hp)
+        th_ref, mo_ref, _ = oracle.lalr(offs, theta, mom, gh_ref, *hp)
+        assert np.array_equal(np_of(mo_d).view(np.uint32), mo_ref.view(np.uint32))
+        assert_close_per_layer(np_of(th_d), th_ref, offs, "theta (per-worker scales)")
+        assert P.status() == 0
+        # what this mode does not offer is refused on the host
+        cs = torch.zeros(d, dtype=torch.int32, device="cuda")
+        with pytest.raises(api.DatError) as e:
+            api.dat_aggregate(P.plan, lv, sg, sc, cs, gh)
+        assert e.value.code == api.DAT_ERR_ARG
+        with pytest.raises(api.DatError) as e:
+            api.dat_step(P.plan, th_d, mo_d, g_dev, seed, step, hp)
+        assert e.value.code == api.DAT_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("bits", [1, 4, 8, 16])
+def test_unfused_parity_per_worker_scales(api, oracle, bits, rng_bits):
+    offs, grads, theta, mom = _random_problem(40 + bits, SIZES_RAGGED, 5)
+    grads[2] *= np.float32(37.0)                 # workers with very different norms
+    grads[4][int(offs[7]):int(offs[8])] = 0.0    # one worker's layer all zero: its norm is 0
+    _check_unfused_per_worker(api, oracle, offs, grads, theta, mom, bits, HP, rng_bits=rng_bits)
+
+
 @pytest.mark.parametrize("bits", [1, 2, 4, 8, 16, 32])
 def test_fused_parity_ragged(api, oracle, bits, rng_bits):
     offs, grads, theta, mom = _random_problem(100 + bits, SIZES_RAGGED, 3)
