@@ -56,6 +56,8 @@ def _declare(L):
     L.dat_oracle_scales.restype = None
     L.dat_oracle_quantize.argtypes = [_i64, _p, _i64, _i64, _int, _int, _int, _p, _u64, _u64, _int, _p, _p, _p]
     L.dat_oracle_quantize.restype = None
+    L.dat_oracle_requantize.argtypes = [_i64, _p, _i64, _i64, _int, _u64, _u64, _int, _u32, _p, _p, _p, _p, _p]
+    L.dat_oracle_requantize.restype = None
     L.dat_oracle_level_plane_bytes.argtypes = [_i64, _int]
     L.dat_oracle_level_plane_bytes.restype = _i64
     L.dat_oracle_sign_plane_bytes.argtypes = [_i64]
@@ -181,6 +183,23 @@ def quantize(offsets, grads, bits, seed, step, scales_, scale_mode=SCALE_SHARED_
                               int(seed), int(step), int(rng_bits), _addr(sc),
                               _ptr_array(list(level), shift), _ptr_array(list(neg), shift))
     return level, neg
+
+
+def requantize(offsets, g_hat, bits, seed, step, stream, rng_bits=16, scales_in=None):
+    """Algorithm A1 Step 10: the server's Q(g_hat).  Returns (g_hat' float32 [d], scales float32 [h],
+    level uint32 [d], neg uint8 [d]); the input is untouched.  `stream` = index of the random
+    stream (M by convention)."""
+    o = _offsets(offsets)
+    h, d = o.size - 1, int(o[-1])
+    assert bits in (1, 2, 4, 8, 16) and rng_bits in RNG_BITS
+    gh = _check(g_hat, np.float32, d).copy()
+    sc_in = None if scales_in is None else _check(np.ascontiguousarray(scales_in, dtype=np.float32), np.float32, h)
+    sc = np.zeros(h, dtype=np.float32)
+    level = np.zeros(d, dtype=np.uint32)
+    neg = np.zeros(d, dtype=np.uint8)
+    lib().dat_oracle_requantize(h, _addr(o), 0, h, bits, int(seed), int(step), int(rng_bits), int(stream),
+                                _addr(sc_in), _addr(gh), _addr(sc), _addr(level), _addr(neg))
+    return gh, sc, level, neg
 
 
 # ---------------------------------------------------------------- S3

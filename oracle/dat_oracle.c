@@ -204,6 +204,46 @@ void dat_oracle_quantize(int64_t h, const int64_t *offsets, int64_t l0, int64_t 
         }
 }
 
+/* Algorithm A1 Step 10 (two-sided quantisation, the parameter-server setting): before the
+ * server sends the aggregate back it quantizes it once more, g_hat <- Q(g_hat).  Q is the same
+ * quantizer applied to ONE vector: the scale of layer l is ||g_hat_l||_2 itself (or scales_in[l]
+ * if given), the random numbers come from the stream of index `stream` (by convention M, the
+ * first index no worker uses; the paper does not say where the server's randomness comes from),
+ * and the receiver's value is nu_l * sign * level / S.
+ * Outputs: scales[l], level[e], neg[e], and g_hat overwritten with the de-quantised value.    */
+void dat_oracle_requantize(int64_t h, const int64_t *offsets, int64_t l0, int64_t l1, int bits,
+                           uint64_t seed, uint64_t step, int rng_bits, uint32_t stream,
+                           const float *scales_in, float *g_hat, float *scales,
+                           uint32_t *level, uint8_t *neg)
+{
+    const uint32_t S = (uint32_t)((1ull << bits) - 1ull);
+    const float S_f = (float)S;
+    (void)h;
+    for (int64_t l = l0; l < l1; ++l) {
+        float nu;
+        if (scales_in) {
+            nu = scales_in[l];
+        } else {
+            double ss = 0.0;
+            for (int64_t e = offsets[l]; e < offsets[l + 1]; ++e)
+                ss += (double)g_hat[e] * (double)g_hat[e];
+            nu = (float)sqrt(ss);
+        }
+        scales[l] = nu;
+        float t = (nu == 0.0f) ? 0.0f : S_f / nu;
+        float factor = (nu == 0.0f) ? 0.0f : nu / S_f;
+        for (int64_t e = offsets[l]; e < offsets[l + 1]; ++e) {
+            float g = g_hat[e];
+            float u1 = dat_oracle_uniform12_at(seed, step, stream, (uint64_t)e, rng_bits);
+            float y = fminf(fmaf(fabsf(g), t, u1), S_f + 1.0f);
+            uint32_t lev = (uint32_t)floorf(y) - 1u;
+            level[e] = lev;
+            neg[e] = (uint8_t)(g < 0.0f);
+            g_hat[e] = (float)(neg[e] ? -(int32_t)lev : (int32_t)lev) * factor;
+        }
+    }
+}
+
 /* ------------------------------------------------------------------------- */
 /* S3: the transmitted message.  32 bits per norm, 1 sign bit and b level bits */
 /* per element ("(32 + d + b d) bits", with one norm per layer).               */
