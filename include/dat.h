@@ -168,6 +168,22 @@ int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_t seed, uin
 int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint8_t *signs,
                   const float *scales, int32_t *code_sum, float *g_hat, void *stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * dat_requantize -- Algorithm A1 Step 10 (two-sided quantisation, the parameter-server setting):
+ * the server quantizes the aggregate once more before sending it back, g_hat <- Q(g_hat).
+ *   Q is the quantizer of dat_quantize applied to ONE vector: nu_l = ||g_hat_l||_2 (or
+ *   scales_in[l]), random stream of index M (the first one no worker uses; the paper does not say
+ *   where the server's random numbers come from), level = min(floor(fma(|g|, S/nu_l, u1)) - 1, S),
+ *   and the receiver's value nu_l * sign * level / S, which overwrites g_hat.
+ *   g_hat      device fp32[d], read and overwritten.
+ *   levels     device, level_bytes_per_worker bytes, written: the server's level plane.
+ *   signs      device, sign_bytes_per_worker bytes, written.
+ *   scales     device fp32[h], written: nu_l.       scales_in  device fp32[h] or NULL, as in dat_quantize.
+ * Valid for any plan with b < 32, whatever its scale mode.  Errors: ARG, ALIGN, BITS, CUDA.
+ * ------------------------------------------------------------------------------------------- */
+int dat_requantize(dat_plan_t *plan, float *g_hat, uint64_t seed, uint64_t step, uint8_t *levels,
+                   uint8_t *signs, float *scales, const float *scales_in, void *stream);
+
 /* dat_average -- Eq. grad_agg when Q is the identity (b = 32): g_hat_e = (sum_i g_e^(i)) / M,
  * accumulated in fp32 in ascending worker order.  Valid for any plan.
  *   grads  host array of M device pointers (fp32[d], read-only);  g_hat  device fp32[d], written. */

@@ -29,7 +29,7 @@ DAT_STATIC_MAX_LAYERS, DAT_STATIC_MAX_TILES = 4096, 32768
 DAT_STATUS_NONFINITE, DAT_STATUS_TIMEOUT, DAT_STATUS_BOUNDS = 1, 2, 4
 
 # every symbol include/dat.h declares
-EXPORTS = ["dat_plan_create", "dat_plan_destroy", "dat_plan_sizes", "dat_quantize", "dat_aggregate",
+EXPORTS = ["dat_plan_create", "dat_plan_destroy", "dat_plan_sizes", "dat_quantize", "dat_aggregate", "dat_requantize",
            "dat_average", "dat_lalr_step", "dat_lalr_step_static", "dat_step", "dat_step_host", "dat_get_status",
            "dat_plan_launch_count", "dat_strerror", "dat_last_cuda_error"]
 
@@ -45,6 +45,7 @@ _lib.dat_plan_destroy.argtypes = [_p]
 _lib.dat_plan_sizes.argtypes = [_p, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]
 _lib.dat_quantize.argtypes = [_p, _p, _u64, _u64, _p, _p, _p, _p, _p]
 _lib.dat_aggregate.argtypes = [_p, _p, _p, _p, _p, _p, _p]
+_lib.dat_requantize.argtypes = [_p, _p, _u64, _u64, _p, _p, _p, _p, _p]
 _lib.dat_average.argtypes = [_p, _p, _p, _p]
 _lib.dat_lalr_step.argtypes = [_p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
 _lib.dat_lalr_step_static.argtypes = [_i64, _p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
@@ -136,6 +137,11 @@ def dat_quantize(plan, grads, seed, step, levels, signs, scales, scales_in=None,
 def dat_aggregate(plan, levels, signs, scales, code_sum, g_hat, stream=None):
     _ok(_lib.dat_aggregate(_p(plan), _ptr(levels), _ptr(signs), _ptr(scales), _ptr(code_sum), _ptr(g_hat),
                            _stream(stream)), "dat_aggregate")
+
+
+def dat_requantize(plan, g_hat, seed, step, levels, signs, scales, scales_in=None, stream=None):
+    _ok(_lib.dat_requantize(_p(plan), _ptr(g_hat), int(seed), int(step), _ptr(levels), _ptr(signs), _ptr(scales),
+                            _ptr(scales_in), _stream(stream)), "dat_requantize")
 
 
 def dat_average(plan, grads, g_hat, stream=None):

@@ -95,7 +95,7 @@ template <int BITS>
 __global__ void __launch_bounds__(DAT_THREADS)
 k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h, int64_t d,
            const float *__restrict__ qmul_all, uint8_t *__restrict__ levels, uint8_t *__restrict__ signs,
-           int64_t level_bytes, int64_t sign_bytes, bool rng16, bool per_worker)
+           int64_t level_bytes, int64_t sign_bytes, bool rng16, bool per_worker, uint32_t stream_base)
 {
     constexpr int GROUPS = DAT_TILE / 4;                     // aligned groups per tile
     constexpr int LEVEL_TILE_BYTES = DAT_TILE * BITS / 8;
@@ -124,7 +124,7 @@ k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h,
         float gv[4];
         dat_load4(g, e0, 0, d, gv);
         float u1[4];
-        dat_u1x4((uint64_t)e0, (uint32_t)worker, keys, rng16, u1);
+        dat_u1x4((uint64_t)e0, stream_base + (uint32_t)worker, keys, rng16, u1);     // the worker's random stream
         uint32_t lev[4], neg = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -212,7 +212,7 @@ extern "C" int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_
     dim3 grid((unsigned)flat_tiles, (unsigned)plan->M);
 #define DAT_Q(B)                                                                                           \
     k_quantize<B><<<grid, DAT_THREADS, 0, s>>>(gp, keys, plan->d_offsets, h, plan->d, plan->d_qmul, levels, \
-                                               signs, plan->level_bytes, plan->sign_bytes, plan->rng_bits == 16, per_worker)
+                                               signs, plan->level_bytes, plan->sign_bytes, plan->rng_bits == 16, per_worker, 0u)
     switch (plan->bits) {
     case 1: DAT_Q(1); break;
     case 2: DAT_Q(2); break;
@@ -364,6 +364,70 @@ k_aggregate_per_worker(const uint8_t *__restrict__ levels, const uint8_t *__rest
     } else {
         for (int j = 0; j < 8 && e0 + j < d; ++j) g_hat[e0 + j] = out[j];
     }
+}
+
+// ------------------------------------------------------------------------------------------
+// Algorithm A1 Step 10 (two-sided quantisation): g_hat <- Q(g_hat) at the server.  The same
+// kernels as Steps 7 and 9 on ONE vector: norm per layer, levels on the random stream of index M
+// (the first one no worker uses), packed message, and the receiver's value nu_l * sign * level / S.
+// ------------------------------------------------------------------------------------------
+extern "C" int dat_requantize(dat_plan_t *plan, float *g_hat, uint64_t seed, uint64_t step,
+                              uint8_t *levels, uint8_t *signs, float *scales, const float *scales_in,
+                              void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (plan->bits == 32) return DAT_ERR_BITS;
+    if (!g_hat || !levels || !signs || !scales) return DAT_ERR_ARG;
+    if (step >> 32) return DAT_ERR_ARG;
+    if (!dat_aligned16(g_hat) || !dat_aligned16(levels) || !dat_aligned16(signs) || !dat_aligned16(scales) ||
+        (scales_in && !dat_aligned16(scales_in)))
+        return DAT_ERR_ALIGN;
+    GradPtrs gp;
+    for (int i = 0; i < DAT_MAX_WORKERS; ++i) gp.p[i] = nullptr;
+    gp.p[0] = g_hat;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    const int h = (int)plan->h;
+    const float S_f = (float)plan->S;
+    if (scales_in) {
+        if (scales_in != scales)
+            DAT_CUDA(plan, cudaMemcpyAsync(scales, scales_in, (size_t)h * 4, cudaMemcpyDeviceToDevice, s));
+        k_qmul_from_scales<<<(h + 255) / 256, 256, 0, s>>>(h, S_f, scales, plan->d_qmul, plan->d_status);
+        DAT_LAUNCHED(plan);
+    } else {
+        dim3 grid((unsigned)plan->n_tiles, 1u);
+        k_sumsq_partial<<<grid, DAT_THREADS, 0, s>>>(gp, plan->d_offsets, plan->d_tile_base, h, 1, plan->d_partials);
+        DAT_LAUNCHED(plan);
+        k_scales_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base, h, 1, S_f, plan->d_partials,
+                                                    plan->d_worker_norms, scales, plan->d_qmul, plan->d_status, false);
+        DAT_LAUNCHED(plan);
+    }
+    const PhiloxKeys keys = dat_make_keys(seed, step);
+    const int64_t flat_tiles = (plan->d + DAT_TILE - 1) / DAT_TILE;
+    dim3 qgrid((unsigned)flat_tiles, 1u);
+    const unsigned agrid = (unsigned)((plan->d + DAT_THREADS * 8 - 1) / (DAT_THREADS * 8));
+    k_dq_from_scales<<<(h + 255) / 256, 256, 0, s>>>(h, S_f, scales, plan->d_dq);      // nu / (S * 1)
+    DAT_LAUNCHED(plan);
+#define DAT_RQ(B)                                                                                                   \
+    do {                                                                                                            \
+        k_quantize<B><<<qgrid, DAT_THREADS, 0, s>>>(gp, keys, plan->d_offsets, h, plan->d, plan->d_qmul, levels,    \
+                                                    signs, plan->level_bytes, plan->sign_bytes,                     \
+                                                    plan->rng_bits == 16, false, (uint32_t)plan->M);                \
+        DAT_LAUNCHED(plan);                                                                                         \
+        k_aggregate<B><<<agrid, DAT_THREADS, 0, s>>>(levels, signs, plan->level_bytes, plan->sign_bytes, 1,          \
+                                                     plan->d_offsets, h, plan->d, plan->d_dq, nullptr, g_hat);      \
+    } while (0)
+    switch (plan->bits) {
+    case 1: DAT_RQ(1); break;
+    case 2: DAT_RQ(2); break;
+    case 4: DAT_RQ(4); break;
+    case 8: DAT_RQ(8); break;
+    default: DAT_RQ(16); break;
+    }
+#undef DAT_RQ
+    DAT_LAUNCHED(plan);
+    return DAT_OK;
 }
 
 extern "C" int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint8_t *signs,

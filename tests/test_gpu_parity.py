@@ -166,6 +166,36 @@ def test_unfused_parity_per_worker_scales(api, oracle, bits, rng_bits):
     _check_unfused_per_worker(api, oracle, offs, grads, theta, mom, bits, HP, rng_bits=rng_bits)
 
 
+@pytest.mark.parametrize("bits", [1, 2, 8, 16])
+def test_two_sided_requantize_parity(api, oracle, bits, rng_bits):
+    """Algorithm A1 Step 10 on the GPU against the oracle: norms within 1 ulp, then (given the GPU's
+    norm bits) the server's packed message and the receiver's value bit for bit."""
+    offs, grads, theta, mom = _random_problem(70 + bits, SIZES_RAGGED, 3)
+    d, M = int(offs[-1]), 3
+    g = grads[0].copy()
+    g[int(offs[9]):int(offs[10])] = 0.0          # a layer whose aggregate is zero
+    with GpuPlan(api, offs, M, bits, rng_bits) as P:
+        gh = torch.from_numpy(g).cuda()
+        lv = torch.full((P.level_bytes,), 0xAB, dtype=torch.uint8, device="cuda")
+        sg = torch.full((P.sign_bytes,), 0xCD, dtype=torch.uint8, device="cuda")
+        sc = torch.zeros(P.h, dtype=torch.float32, device="cuda")
+        api.dat_requantize(P.plan, gh, 5, 2, lv, sg, sc)
+        torch.cuda.synchronize()
+        _, sc_ref, _, _ = oracle.requantize(offs, g, bits, 5, 2, stream=M, rng_bits=rng_bits)
+        sc_gpu = np_of(sc)
+        assert ulp_diff(sc_gpu, sc_ref).max() <= 1
+        out_ref, _, level, neg = oracle.requantize(offs, g, bits, 5, 2, stream=M, rng_bits=rng_bits, scales_in=sc_gpu)
+        lp_ref, sp_ref = oracle.pack(level, neg, bits)
+        assert np.array_equal(np_of(lv), lp_ref) and np.array_equal(np_of(sg), sp_ref)
+        assert np.array_equal(np_of(gh).view(np.uint32), out_ref.view(np.uint32))
+        # caller-supplied norms, in place
+        gh2 = torch.from_numpy(g).cuda()
+        api.dat_requantize(P.plan, gh2, 5, 2, lv, sg, sc, scales_in=sc)
+        torch.cuda.synchronize()
+        assert torch.equal(gh2, gh)
+        assert P.status() == 0
+
+
 @pytest.mark.parametrize("bits", [1, 2, 4, 8, 16, 32])
 def test_fused_parity_ragged(api, oracle, bits, rng_bits):
     offs, grads, theta, mom = _random_problem(100 + bits, SIZES_RAGGED, 3)
