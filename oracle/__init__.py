@@ -72,6 +72,8 @@ def _declare(L):
     L.dat_oracle_average.restype = None
     L.dat_oracle_lalr.argtypes = [_p, _i64, _i64, _p, _p, _p, _f32, _f32, _f32, _f32, _f32, _p]
     L.dat_oracle_lalr.restype = None
+    L.dat_oracle_lamb.argtypes = [_p, _i64, _i64, _p, _p, _p, _p, _f32, _f32, _f32, _f32, _f32, _f32, _f32, _i64, _p]
+    L.dat_oracle_lamb.restype = None
     L.dat_oracle_step.argtypes = [_i64, _p, _i64, _i64, _int, _int, _int, _p, _p, _p, _u64, _u64, _int, _p,
                                   _f32, _f32, _f32, _f32, _f32, _p, _p, _p]
     L.dat_oracle_step.restype = _int
@@ -275,6 +277,23 @@ def lalr(offsets, theta, mom, g_hat, lr, momentum, weight_decay, c_l=0.0, c_u=10
     lib().dat_oracle_lalr(_addr(o), l0, l1, _addr(th, shift), _addr(mo, shift), _addr(gh, shift),
                           lr, momentum, weight_decay, c_l, c_u, _addr(norms))
     return th, mo, norms
+
+
+def lamb(offsets, theta, mom, var, g_hat, t, lr, beta1=0.9, beta2=0.999, zeta=1e-6, weight_decay=0.0,
+         c_l=0.0, c_u=10.0):
+    """Algorithm A2 followed by Eq. upth.  Returns (theta', m', v', norms float32 [h, 2] = (||theta_l||, ||u_l||));
+    inputs untouched.  t >= 1 is the iteration count of the bias corrections."""
+    o = _offsets(offsets)
+    h, d = o.size - 1, int(o[-1])
+    assert t >= 1
+    th = _check(theta, np.float32, d).copy()
+    mo = _check(mom, np.float32, d).copy()
+    va = _check(var, np.float32, d).copy()
+    gh = _check(g_hat, np.float32, d)
+    norms = np.zeros((h, 2), dtype=np.float32)
+    lib().dat_oracle_lamb(_addr(o), 0, h, _addr(th), _addr(mo), _addr(va), _addr(gh),
+                          lr, beta1, beta2, zeta, weight_decay, c_l, c_u, int(t), _addr(norms))
+    return th, mo, va, norms
 
 
 # ---------------------------------------------------------------- whole step

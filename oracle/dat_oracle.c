@@ -383,6 +383,59 @@ void dat_oracle_lalr(const int64_t *offsets, int64_t l0, int64_t l1,
 }
 
 /* ------------------------------------------------------------------------- */
+/* Algorithm A2 (LAMB) as the outer-minimisation oracle: the direction u_t is    */
+/* Adam's, the update is again Eq. upth = Eq. 3, layer by layer.                 */
+/* ------------------------------------------------------------------------- */
+
+/* t = 1, 2, ... is the iteration count of the bias corrections.  Per element (fp32, one rounding
+ * per listed operation):
+ *   m' = fma(beta1, m, (1-beta1) * g)            v' = fma(beta2, v, (1-beta2) * (g*g))
+ *   m^ = m' / (1 - beta1^t)                      v^ = v' / (1 - beta2^t)
+ *   u  = fma(wd, theta, m^ / (sqrt(v^) + zeta))
+ * then theta' = theta - (lr * tau(||theta_l||) / ||u_l||) * u with the norms of the layer in fp64.
+ * Readings: the algorithm as printed overwrites m_t, v_t with their bias-corrected values; they are
+ * taken as temporaries (m^, v^), as in the LAMB paper it cites, and m', v' are the stored moments.
+ * The printed algorithm has no weight decay while the experiments set one; it enters as in the LAMB
+ * paper (added to the ratio), so wd = 0 is the algorithm exactly as printed.
+ * 1 - beta^t is formed in double and rounded to float once.                                       */
+void dat_oracle_lamb(const int64_t *offsets, int64_t l0, int64_t l1,
+                     float *theta, float *mom, float *var, const float *g_hat,
+                     float lr, float beta1, float beta2, float zeta, float wd, float c_l, float c_u,
+                     int64_t t, float *layer_norms)
+{
+    const float om1 = 1.0f - beta1, om2 = 1.0f - beta2;
+    const float bc1 = (float)(1.0 - pow((double)beta1, (double)t));
+    const float bc2 = (float)(1.0 - pow((double)beta2, (double)t));
+    for (int64_t l = l0; l < l1; ++l) {
+        int64_t n = offsets[l + 1] - offsets[l];
+        float *u = (float *)malloc((size_t)n * sizeof(float));
+        double ss_theta = 0.0, ss_u = 0.0;
+        for (int64_t e = offsets[l]; e < offsets[l + 1]; ++e) {
+            float g = g_hat[e];
+            float m_new = fmaf(beta1, mom[e], om1 * g);
+            float v_new = fmaf(beta2, var[e], om2 * (g * g));
+            mom[e] = m_new;
+            var[e] = v_new;
+            float m_hat = m_new / bc1;
+            float v_hat = v_new / bc2;
+            float ue = fmaf(wd, theta[e], m_hat / (sqrtf(v_hat) + zeta));
+            u[e - offsets[l]] = ue;
+            ss_theta += (double)theta[e] * (double)theta[e];
+            ss_u += (double)ue * (double)ue;
+        }
+        float n_theta = (float)sqrt(ss_theta);
+        float n_u = (float)sqrt(ss_u);
+        float tau = fminf(fmaxf(n_theta, c_l), c_u);
+        float ratio = (n_u == 0.0f) ? 0.0f : tau / n_u;
+        float a = lr * ratio;
+        for (int64_t e = offsets[l]; e < offsets[l + 1]; ++e)
+            theta[e] = fmaf(-a, u[e - offsets[l]], theta[e]);
+        if (layer_norms) { layer_norms[2 * l] = n_theta; layer_norms[2 * l + 1] = n_u; }
+        free(u);
+    }
+}
+
+/* ------------------------------------------------------------------------- */
 /* One whole step for layers [l0, l1): S1 -> S2 -> S4/S5 -> S6-S8, one layer   */
 /* at a time (temporary code arrays hold one layer).  scales_in (nullable)      */
 /* replaces the computed scales (same indexing).  code_sum, layer_norms,        */
