@@ -58,6 +58,20 @@ typedef struct dat_hparams {
     float c_u;
 } dat_hparams_t;
 
+/* Hyper-parameters of the LAMB direction (Algorithm A2) and of the update of Eq. upth: beta1, beta2
+ * of the two moments (each in (0,1)), zeta > 0 of the ratio m^/(sqrt(v^) + zeta), weight decay (added
+ * to the ratio as in the LAMB paper; 0 gives the algorithm as printed), and lr, c_l, c_u as above.
+ * The paper's ImageNet runs use beta1 = 0.9, beta2 = 0.999, weight decay 1e-4. */
+typedef struct dat_lamb_hparams {
+    float lr;
+    float beta1;
+    float beta2;
+    float zeta;
+    float weight_decay;
+    float c_l;
+    float c_u;
+} dat_lamb_hparams_t;
+
 /* Which l2 norm scales the quantizer of Eq. rand_q.
  * SHARED_MAX: nu_l = max_i ||g_l^(i)||_2, one value per layer shared by all workers, so that
  *             the workers' integer codes lie on one grid and Eq. grad_agg becomes an integer sum
@@ -203,6 +217,20 @@ int dat_average(dat_plan_t *plan, const float *const *grads, float *g_hat, void 
  * ------------------------------------------------------------------------------------------- */
 int dat_lalr_step(dat_plan_t *plan, float *theta, float *mom, const float *g_hat,
                   const dat_hparams_t *hp, float *layer_norms_out, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * dat_lamb_step -- Algorithm A1 Step 12 with LAMB (Algorithm A2) as the outer-minimisation oracle.
+ * Per element (fp32, one rounding per operation), with t >= 1 the iteration count:
+ *   m' = fma(beta1, m, (1-beta1)*g_hat)     v' = fma(beta2, v, (1-beta2)*(g_hat*g_hat))
+ *   m^ = m'/(1-beta1^t)     v^ = v'/(1-beta2^t)     u = fma(wd, theta, m^/(sqrt(v^) + zeta))
+ * and per layer (Eq. upth): theta' = theta - lr*tau(||theta_l||)/||u_l|| * u, norms in fp64, zero
+ * norms as in dat_lalr_step.  The bias-corrected moments are temporaries; m', v' are what is stored.
+ *   theta, mom, var  device fp32[d], updated in place.     g_hat  device fp32[d], read-only.
+ *   layer_norms_out  device fp32[2h] or NULL: (||theta_l||, ||u_l||).
+ * Errors: ARG (null pointer, t < 1, beta outside (0,1)), ALIGN, CUDA.
+ * ------------------------------------------------------------------------------------------- */
+int dat_lamb_step(dat_plan_t *plan, float *theta, float *mom, float *var, const float *g_hat,
+                  const dat_lamb_hparams_t *hp, int64_t t, float *layer_norms_out, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * dat_lalr_step_static -- the update of dat_lalr_step for callers that must not allocate.

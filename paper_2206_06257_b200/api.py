@@ -30,13 +30,18 @@ DAT_STATUS_NONFINITE, DAT_STATUS_TIMEOUT, DAT_STATUS_BOUNDS = 1, 2, 4
 
 # every symbol include/dat.h declares
 EXPORTS = ["dat_plan_create", "dat_plan_destroy", "dat_plan_sizes", "dat_quantize", "dat_aggregate", "dat_requantize",
-           "dat_average", "dat_lalr_step", "dat_lalr_step_static", "dat_step", "dat_step_host", "dat_get_status",
+           "dat_average", "dat_lalr_step", "dat_lamb_step", "dat_lalr_step_static", "dat_step", "dat_step_host", "dat_get_status",
            "dat_plan_launch_count", "dat_strerror", "dat_last_cuda_error"]
 
 
 class dat_hparams_t(C.Structure):
     _fields_ = [("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
                 ("c_l", C.c_float), ("c_u", C.c_float)]
+
+
+class dat_lamb_hparams_t(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("zeta", C.c_float),
+                ("weight_decay", C.c_float), ("c_l", C.c_float), ("c_u", C.c_float)]
 
 
 _p, _i64, _u64, _int = C.c_void_p, C.c_int64, C.c_uint64, C.c_int
@@ -48,6 +53,7 @@ _lib.dat_aggregate.argtypes = [_p, _p, _p, _p, _p, _p, _p]
 _lib.dat_requantize.argtypes = [_p, _p, _u64, _u64, _p, _p, _p, _p, _p]
 _lib.dat_average.argtypes = [_p, _p, _p, _p]
 _lib.dat_lalr_step.argtypes = [_p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
+_lib.dat_lamb_step.argtypes = [_p, _p, _p, _p, _p, C.POINTER(dat_lamb_hparams_t), _i64, _p, _p]
 _lib.dat_lalr_step_static.argtypes = [_i64, _p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
 _lib.dat_step.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_step_host.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p]
@@ -152,6 +158,13 @@ def dat_lalr_step(plan, theta, mom, g_hat, hp, layer_norms_out=None, stream=None
     h = _hp(hp)
     _ok(_lib.dat_lalr_step(_p(plan), _ptr(theta), _ptr(mom), _ptr(g_hat), C.byref(h), _ptr(layer_norms_out),
                            _stream(stream)), "dat_lalr_step")
+
+
+def dat_lamb_step(plan, theta, mom, var, g_hat, hp, t, layer_norms_out=None, stream=None):
+    """hp: dat_lamb_hparams_t or (lr, beta1, beta2, zeta, weight_decay, c_l, c_u); t >= 1."""
+    h = hp if isinstance(hp, dat_lamb_hparams_t) else dat_lamb_hparams_t(*[float(x) for x in hp])
+    _ok(_lib.dat_lamb_step(_p(plan), _ptr(theta), _ptr(mom), _ptr(var), _ptr(g_hat), C.byref(h), int(t),
+                           _ptr(layer_norms_out), _stream(stream)), "dat_lamb_step")
 
 
 def dat_lalr_step_static(layer_offsets, theta, mom, g_hat, hp, layer_norms_out=None, stream=None):

@@ -1,6 +1,8 @@
 // The three steps as separate calls: dat_quantize (Algorithm A1 Step 7), dat_aggregate /
 // dat_average (Step 9, Eq. grad_agg) and dat_lalr_step (Step 12, Eq. 3).  Codes, scales and
 // g_hat are materialised in device memory between the calls.
+#include <cmath>
+
 #include "dat_internal.cuh"
 
 // ------------------------------------------------------------------------------------------
@@ -609,6 +611,119 @@ extern "C" int dat_lalr_step(dat_plan_t *plan, float *theta, float *mom, const f
     DAT_LAUNCHED(plan);
     k_lalr_pass2<<<(unsigned)plan->n_tiles, DAT_THREADS, 0, s>>>(theta, mom, plan->d_offsets, plan->d_tile_base,
                                                                  h, plan->d_step_a);
+    DAT_LAUNCHED(plan);
+    return DAT_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// LAMB (Algorithm A2) with the update of Eq. upth = Eq. 3.  Pass 1: the moments m', v' are stored,
+// the direction u = m^/(sqrt(v^) + zeta) + wd*theta is formed on the fly for the fp64 partial sums
+// of theta^2 and u^2.  Finalize as for LALR.  Pass 2 forms u again from the stored moments (the same
+// fp32 operations give the same bits) and moves theta.
+// ------------------------------------------------------------------------------------------
+struct LambConst {
+    float beta1, beta2, om1, om2, bc1, bc2, zeta, wd;
+};
+
+__device__ __forceinline__ float dat_lamb_direction(const LambConst &c, float m_new, float v_new, float theta)
+{
+    const float m_hat = m_new / c.bc1;
+    const float v_hat = v_new / c.bc2;
+    return __fmaf_rn(c.wd, theta, m_hat / (sqrtf(v_hat) + c.zeta));
+}
+
+__global__ void __launch_bounds__(DAT_THREADS)
+k_lamb_pass1(const float *__restrict__ theta, float *__restrict__ mom, float *__restrict__ var,
+             const float *__restrict__ g_hat, const int64_t *__restrict__ off,
+             const int64_t *__restrict__ tile_base, int h, LambConst c, double *__restrict__ partials)
+{
+    __shared__ double scratch[DAT_THREADS / 32];
+    const int64_t tile = blockIdx.x;
+    const TileRange r = dat_tile_range(off, tile_base, h, tile);
+    double ss_theta = 0.0, ss_u = 0.0;
+#pragma unroll
+    for (int it = 0; it < DAT_TILE / 4 / DAT_THREADS; ++it) {
+        const int64_t e0 = r.begin + 4 * (int64_t)(it * DAT_THREADS + threadIdx.x);
+        if (e0 < r.end) {
+            float th[4], m[4], v[4], g[4];
+            dat_load4(theta, e0, r.lo, r.hi, th);
+            dat_load4(mom, e0, r.lo, r.hi, m);
+            dat_load4(var, e0, r.lo, r.hi, v);
+            dat_load4(g_hat, e0, r.lo, r.hi, g);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                m[j] = __fmaf_rn(c.beta1, m[j], __fmul_rn(c.om1, g[j]));
+                v[j] = __fmaf_rn(c.beta2, v[j], __fmul_rn(c.om2, __fmul_rn(g[j], g[j])));
+                const bool inside = (e0 + j >= r.lo && e0 + j < r.hi);
+                const float u = inside ? dat_lamb_direction(c, m[j], v[j], th[j]) : 0.0f;
+                ss_theta = fma((double)th[j], (double)th[j], ss_theta);
+                ss_u = fma((double)u, (double)u, ss_u);
+            }
+            dat_store4(mom, e0, r.lo, r.hi, m);
+            dat_store4(var, e0, r.lo, r.hi, v);
+        }
+    }
+    const double a = dat_block_sum(ss_theta, scratch);
+    const double b = dat_block_sum(ss_u, scratch);
+    if (threadIdx.x == 0) { partials[2 * tile] = a; partials[2 * tile + 1] = b; }
+}
+
+__global__ void __launch_bounds__(DAT_THREADS)
+k_lamb_pass2(float *__restrict__ theta, const float *__restrict__ mom, const float *__restrict__ var,
+             const int64_t *__restrict__ off, const int64_t *__restrict__ tile_base, int h, LambConst c,
+             const float *__restrict__ step_a)
+{
+    const int64_t tile = blockIdx.x;
+    const TileRange r = dat_tile_range(off, tile_base, h, tile);
+    const float na = -__ldg(step_a + r.layer);
+#pragma unroll
+    for (int it = 0; it < DAT_TILE / 4 / DAT_THREADS; ++it) {
+        const int64_t e0 = r.begin + 4 * (int64_t)(it * DAT_THREADS + threadIdx.x);
+        if (e0 < r.end) {
+            float th[4], m[4], v[4];
+            dat_load4(theta, e0, r.lo, r.hi, th);
+            dat_load4(mom, e0, r.lo, r.hi, m);
+            dat_load4(var, e0, r.lo, r.hi, v);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const bool inside = (e0 + j >= r.lo && e0 + j < r.hi);
+                const float u = inside ? dat_lamb_direction(c, m[j], v[j], th[j]) : 0.0f;
+                th[j] = __fmaf_rn(na, u, th[j]);
+            }
+            dat_store4(theta, e0, r.lo, r.hi, th);
+        }
+    }
+}
+
+extern "C" int dat_lamb_step(dat_plan_t *plan, float *theta, float *mom, float *var, const float *g_hat,
+                             const dat_lamb_hparams_t *hp, int64_t t, float *layer_norms_out, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (!theta || !mom || !var || !g_hat || !hp || t < 1) return DAT_ERR_ARG;
+    if (!(hp->beta1 > 0.0f && hp->beta1 < 1.0f && hp->beta2 > 0.0f && hp->beta2 < 1.0f)) return DAT_ERR_ARG;
+    if (!dat_aligned16(theta) || !dat_aligned16(mom) || !dat_aligned16(var) || !dat_aligned16(g_hat) ||
+        (layer_norms_out && !dat_aligned16(layer_norms_out)))
+        return DAT_ERR_ALIGN;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int h = (int)plan->h;
+    LambConst c;
+    c.beta1 = hp->beta1;
+    c.beta2 = hp->beta2;
+    c.om1 = 1.0f - hp->beta1;
+    c.om2 = 1.0f - hp->beta2;
+    c.bc1 = (float)(1.0 - pow((double)hp->beta1, (double)t));      // 1 - beta^t in double, rounded once
+    c.bc2 = (float)(1.0 - pow((double)hp->beta2, (double)t));
+    c.zeta = hp->zeta;
+    c.wd = hp->weight_decay;
+    k_lamb_pass1<<<(unsigned)plan->n_tiles, DAT_THREADS, 0, s>>>(theta, mom, var, g_hat, plan->d_offsets,
+                                                                 plan->d_tile_base, h, c, plan->d_partials);
+    DAT_LAUNCHED(plan);
+    k_lalr_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base, plan->d_partials, hp->lr, hp->c_l, hp->c_u,
+                                              plan->d_step_a, layer_norms_out, plan->d_status);
+    DAT_LAUNCHED(plan);
+    k_lamb_pass2<<<(unsigned)plan->n_tiles, DAT_THREADS, 0, s>>>(theta, mom, var, plan->d_offsets,
+                                                                 plan->d_tile_base, h, c, plan->d_step_a);
     DAT_LAUNCHED(plan);
     return DAT_OK;
 }

@@ -196,6 +196,40 @@ def test_two_sided_requantize_parity(api, oracle, bits, rng_bits):
         assert P.status() == 0
 
 
+LAMB_HP = (0.2, 0.9, 0.999, 1e-6, 1e-4, 0.0, 10.0)      # lr, beta1, beta2, zeta, weight decay, c_l, c_u
+
+
+def test_lamb_step_parity_three_steps(api, oracle):
+    """Algorithm A2 + Eq. upth on the GPU against the oracle over t = 1, 2, 3: the moments bit for bit (both
+    sides are fed the same g_hat and the same theta history), theta' within the tolerance, norms within 1 ulp."""
+    offs, grads, theta, mom = _random_problem(91, SIZES_RAGGED + [0 + 50000], 3)
+    d = int(offs[-1])
+    theta[int(offs[4]):int(offs[5])] = 0.0                     # an all-zero parameter tensor
+    var = np.zeros(d, dtype=np.float32)
+    mom = np.zeros(d, dtype=np.float32)
+    with GpuPlan(api, offs, 3, 8) as P:
+        th_d, mo_d, va_d = (torch.from_numpy(x.copy()).cuda() for x in (theta, mom, var))
+        norms = torch.zeros(2 * P.h, dtype=torch.float32, device="cuda")
+        th_ref, mo_ref, va_ref = theta, mom, var
+        for t in (1, 2, 3):
+            g = grads[t - 1]
+            if t == 2:
+                g = g.copy()
+                g[int(offs[10]):int(offs[11])] = 0.0           # a layer with zero gradient
+            th_in = np_of(th_d).copy()                         # the oracle continues from the GPU's theta: moments stay comparable
+            api.dat_lamb_step(P.plan, th_d, mo_d, va_d, torch.from_numpy(g).cuda(), LAMB_HP, t, norms)
+            torch.cuda.synchronize()
+            th_ref, mo_ref, va_ref, n_ref = oracle.lamb(offs, th_in, mo_ref, va_ref, g, t, *LAMB_HP)
+            assert np.array_equal(np_of(mo_d).view(np.uint32), mo_ref.view(np.uint32))
+            assert np.array_equal(np_of(va_d).view(np.uint32), va_ref.view(np.uint32))
+            assert ulp_diff(np_of(norms).reshape(-1, 2), n_ref).max() <= 1
+            assert_close_per_layer(np_of(th_d), th_ref, offs, "theta (LAMB, t = %d)" % t)
+        assert P.status() == 0
+        with pytest.raises(api.DatError) as e:
+            api.dat_lamb_step(P.plan, th_d, mo_d, va_d, th_d, LAMB_HP, 0)
+        assert e.value.code == api.DAT_ERR_ARG
+
+
 @pytest.mark.parametrize("bits", [1, 2, 4, 8, 16, 32])
 def test_fused_parity_ragged(api, oracle, bits, rng_bits):
     offs, grads, theta, mom = _random_problem(100 + bits, SIZES_RAGGED, 3)
