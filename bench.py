@@ -236,7 +236,9 @@ def run_gpu(args):
     theta, mom = synth.make_params(cfg, device=dev)
     grads = synth.make_grads(cfg, 0, device=dev)
     hp = (cfg.lr, cfg.momentum, cfg.weight_decay, cfg.c_l, cfg.c_u)
-    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits, rng_bits=cfg.rng_bits)
+    variant = args.path[len("unfused_"):] if args.path.startswith("unfused_") else ""
+    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits, rng_bits=cfg.rng_bits,
+                               scale_mode=api.DAT_SCALE_PER_WORKER if variant == "per_worker" else api.DAT_SCALE_SHARED_MAX)
     stream = torch.cuda.current_stream()
     working_set = (cfg.M + 2) * cfg.d * 4
     l2_bytes = torch.cuda.get_device_properties(dev).L2_cache_size
@@ -252,7 +254,7 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    unfused = (args.path == "unfused")
+    unfused = args.path.startswith("unfused")
     if unfused:
         if cfg.bits == 32:
             raise SystemExit("--path unfused needs a quantized configuration (bits < 32)")
@@ -261,12 +263,24 @@ def run_gpu(args):
         u_signs = torch.empty(cfg.M * sb, dtype=torch.uint8, device=dev)
         u_scales = torch.empty(ns, dtype=torch.float32, device=dev)
         u_ghat = torch.empty(cfg.d, dtype=torch.float32, device=dev)
+        if variant == "two_sided":      # the server's own message (Algorithm A1 Step 10)
+            s_levels = torch.empty(lb, dtype=torch.uint8, device=dev)
+            s_signs = torch.empty(sb, dtype=torch.uint8, device=dev)
+            s_scales = torch.empty(cfg.h, dtype=torch.float32, device=dev)
+        if variant == "lamb":           # Algorithm A2: second moment, the paper's ImageNet hyper-parameters
+            var = torch.zeros(cfg.d, dtype=torch.float32, device=dev)
+            lamb_hp = (cfg.lr, 0.9, 0.999, 1e-6, 1e-4, cfg.c_l, cfg.c_u)
 
     def one_step(step_index):
         if unfused:
             api.dat_quantize(plan, grads, cfg.seed, step_index, u_levels, u_signs, u_scales)
             api.dat_aggregate(plan, u_levels, u_signs, u_scales, None, u_ghat)
-            api.dat_lalr_step(plan, theta, mom, u_ghat, hp)
+            if variant == "two_sided":
+                api.dat_requantize(plan, u_ghat, cfg.seed, step_index, s_levels, s_signs, s_scales)
+            if variant == "lamb":
+                api.dat_lamb_step(plan, theta, mom, var, u_ghat, lamb_hp, step_index + 1)
+            else:
+                api.dat_lalr_step(plan, theta, mom, u_ghat, hp)
         else:
             api.dat_step(plan, theta, mom, grads, cfg.seed, step_index, hp)
 
@@ -354,6 +368,10 @@ def run_gpu(args):
         if unfused:     # norm pass + quantize pass over the gradients, planes written and read, g_hat, two LALR passes
             beta = (cfg.bits + 1) / 8.0
             algo_bytes = int((8 * cfg.M + 2 * beta * cfg.M + 32) * cfg.d)
+            if variant == "two_sided":  # norm pass and quantize pass over g_hat, the server's planes written and read, g_hat rewritten
+                algo_bytes += int((12 + 2 * beta) * cfg.d)
+            if variant == "lamb":       # pass 1 reads theta, m, v, g_hat and writes m, v; pass 2 reads theta, m, v and writes theta
+                algo_bytes += 12 * cfg.d
         else:
             algo_bytes = (4 * cfg.M + 16) * cfg.d
         achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
@@ -362,13 +380,13 @@ def run_gpu(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": region_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": workload_config(cfg, l2_note),
+            "config": dict(workload_config(cfg, l2_note), path=args.path),
             "step_latency_us": {"median": 1e3 * float(np.median(step_ms)), "min": 1e3 * float(step_ms.min()),
                                 "mean": 1e3 * kernel_ms},
             "pct_of_8TBps": 100.0 * achieved / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "algorithmic_bytes_per_launch": algo_bytes,
-                         "kernel": ("unfused path: 7 kernels per step (whole step timed)" if unfused else "k_fused_step (one launch per step)"),
+                         "kernel": ("%s: %d kernels per step (whole step timed)" % (args.path, launches // K) if unfused else "k_fused_step (one launch per step)"),
                          "peak_source": peak_src},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "status_word": int(status), "outputs_finite": finite, "wall_s_timed_region": t_wall,
@@ -390,8 +408,11 @@ def main():
     ap.add_argument("--rng-bits", type=int, default=0, choices=[0, 16, 23],
                     help="override the resolution of the quantizer's uniform number (0: the config's)")
     ap.add_argument("--impl", default="dat", choices=["dat", "reference"])
-    ap.add_argument("--path", default="fused", choices=["fused", "unfused"],
-                    help="fused: dat_step (the headline); unfused: dat_quantize + dat_aggregate + dat_lalr_step")
+    ap.add_argument("--path", default="fused",
+                    choices=["fused", "unfused", "unfused_per_worker", "unfused_two_sided", "unfused_lamb"],
+                    help="fused: dat_step (the headline); unfused: dat_quantize + dat_aggregate + dat_lalr_step; "
+                         "unfused_per_worker: the same with one quantizer norm per worker; unfused_two_sided: with "
+                         "dat_requantize after the aggregation; unfused_lamb: with dat_lamb_step as the update")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
