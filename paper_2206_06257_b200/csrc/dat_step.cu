@@ -1101,7 +1101,8 @@ static cudaError_t upload(T **dst, const std::vector<T> &src)
 
 static const void *fused_kernel(const dat_plan_t *plan)
 {
-    if (plan->bits == 32) return (const void *)k_fused_step<true, 1, false>;
+    if (plan->bits == 32)       // more than F_RB workers: an item is taken in groups of F_RB rows
+        return plan->M <= F_RB ? (const void *)k_fused_step<true, 1, false> : (const void *)k_fused_step<true, DAT_MAX_WORKERS / F_RB, false>;
     const bool rng16 = (plan->rng_bits == 16);
     if (plan->M <= F_RB) return rng16 ? (const void *)k_fused_step<false, 1, true> : (const void *)k_fused_step<false, 1, false>;
     return rng16 ? (const void *)k_fused_step<false, DAT_MAX_WORKERS / F_RB, true>

@@ -242,6 +242,13 @@ def test_fused_parity_worker_counts(api, oracle, M, rng_bits):
     _check_fused(api, oracle, offs, grads, theta, mom, 4, HP, rng_bits=rng_bits)
 
 
+@pytest.mark.parametrize("M", [9, 13, 64])
+def test_fused_b32_more_than_eight_workers(api, oracle, M):
+    """No quantisation (b = 32) with more gradient rows than one batch holds: the ordered fp32 average of all M."""
+    offs, grads, theta, mom = _random_problem(300 + M, [1000, 5000, 3, 9000], M)
+    _check_fused(api, oracle, offs, grads, theta, mom, 32, HP)
+
+
 @pytest.mark.parametrize("bits", [2, 8, 16])
 def test_fused_parity_extreme_scales(api, oracle, bits, rng_bits):
     """Layers whose norms sit at the ends of the fp32 range (the scaled form of the level
