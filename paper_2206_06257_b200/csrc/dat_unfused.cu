@@ -352,7 +352,9 @@ k_aggregate_per_worker(const uint8_t *__restrict__ levels, const uint8_t *__rest
         const float nu0 = __ldg(nu_i + lidx[0]);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const float code = ((sg >> j) & 1u) ? -(float)lev[j] : (float)lev[j];
+            // (float)level without the conversion unit: 2^23 + level is exact, the sign bit goes on afterwards
+            const float mag = __uint_as_float(0x4B000000u | lev[j]) - 8388608.0f;
+            const float code = __uint_as_float(__float_as_uint(mag) | (((sg >> j) & 1u) << 31));
             const float nu = one_layer ? nu0 : __ldg(nu_i + lidx[j]);
             acc[j] = __fmaf_rn(nu, code, acc[j]);
         }
