@@ -21,15 +21,18 @@ k_sumsq_partial(GradPtrs gp, const int64_t *__restrict__ off, const int64_t *__r
     const TileRange r = dat_tile_range(off, tile_base, h, tile);
     const float *__restrict__ g = gp.p[worker];
     double acc = 0.0;
+    constexpr int ITERS = DAT_TILE / 4 / DAT_THREADS;
+    float v[ITERS][4];
 #pragma unroll
-    for (int it = 0; it < DAT_TILE / 4 / DAT_THREADS; ++it) {
+    for (int it = 0; it < ITERS; ++it) {          // every load of the thread is in flight before the first is used
         const int64_t e0 = r.begin + 4 * (int64_t)(it * DAT_THREADS + threadIdx.x);
-        if (e0 < r.end) {
-            float v[4];
-            dat_load4(g, e0, r.lo, r.hi, v);
+        if (e0 < r.end) dat_load4(g, e0, r.lo, r.hi, v[it]);
+        else v[it][0] = v[it][1] = v[it][2] = v[it][3] = 0.0f;
+    }
 #pragma unroll
-            for (int j = 0; j < 4; ++j) acc = fma((double)v[j], (double)v[j], acc);
-        }
+    for (int it = 0; it < ITERS; ++it) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc = fma((double)v[it][j], (double)v[it][j], acc);
     }
     const double s = dat_block_sum(acc, scratch);
     if (threadIdx.x == 0) partials[tile * M + worker] = s;
@@ -119,12 +122,15 @@ k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h,
     int64_t l_hi = __ldg(off + l + 1);
     float t = __ldg(qmul + l);
 
+    float gall[GROUPS / DAT_THREADS][4];
+#pragma unroll
+    for (int it = 0; it < GROUPS / DAT_THREADS; ++it)      // every load of the thread is in flight before the first is used
+        dat_load4(g, e_tile + 4 * (int64_t)(it * DAT_THREADS + threadIdx.x), 0, d, gall[it]);
 #pragma unroll
     for (int it = 0; it < GROUPS / DAT_THREADS; ++it) {
         const int v = it * DAT_THREADS + threadIdx.x;
         const int64_t e0 = e_tile + 4 * (int64_t)v;
-        float gv[4];
-        dat_load4(g, e0, 0, d, gv);
+        const float *gv = gall[it];
         float u1[4];
         dat_u1x4((uint64_t)e0, stream_base + (uint32_t)worker, keys, rng16, u1);     // the worker's random stream
         uint32_t lev[4], neg = 0;
@@ -276,7 +282,8 @@ k_aggregate(const uint8_t *__restrict__ levels, const uint8_t *__restrict__ sign
     int sum[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) sum[j] = 0;
-    for (int i = 0; i < M; ++i) {
+#pragma unroll 4
+    for (int i = 0; i < M; ++i) {                // four workers' loads in flight at a time
         uint32_t lev[8];
         dat_unpack8<BITS>(levels + (int64_t)i * level_bytes, e0, lev);
         const uint32_t sg = signs[(int64_t)i * sign_bytes + (e0 >> 3)];
@@ -344,6 +351,7 @@ k_aggregate_per_worker(const uint8_t *__restrict__ levels, const uint8_t *__rest
     float acc[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+#pragma unroll 1
     for (int i = 0; i < M; ++i) {
         uint32_t lev[8];
         dat_unpack8<BITS>(levels + (int64_t)i * level_bytes, e0, lev);
