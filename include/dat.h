@@ -285,6 +285,16 @@ int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *gra
              uint64_t seed, uint64_t step, const dat_hparams_t *hp,
              int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream);
 
+/* dat_step_passes -- the same step as dat_step, with the same arguments and the same results bit for
+ * bit up to the norms' last place, computed by three streaming passes in separate launches instead of
+ * one persistent kernel: quantizer norms; then levels, signed sum over the workers, g_hat, m' and the
+ * layer sums in one pass that keeps codes, sums and g_hat in registers; then the theta update.  The
+ * gradients are read twice by construction.  For plans with b < 32 and the shared scale
+ * (DAT_ERR_UNSUPPORTED otherwise).  Its first call on a plan allocates two small tables (synchronous). */
+int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                    uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
+                    float *layer_norms_out, float *scales_out, void *stream);
+
 /* dat_step_host -- dat_step for callers whose data lives in HOST memory: copies theta, mom and
  * the M gradient buffers to plan-owned device staging buffers, runs dat_step, copies theta and
  * mom back, and synchronises `stream` before returning.

@@ -52,6 +52,11 @@ struct dat_plan {
 
     FusedSchedule *fused = nullptr;    // built lazily by dat_step
 
+    // dat_step_passes: per-layer tiles that start on multiples of 8 elements, and their partial sums
+    int64_t *d_tile_base8 = nullptr;   // h+1
+    double *d_partials8 = nullptr;     // 2 per tile
+    int64_t n_tiles8 = 0;
+
     // staging buffers of dat_step_host
     float *stage = nullptr;
 

@@ -140,6 +140,8 @@ extern "C" int dat_plan_destroy(dat_plan_t *plan)
     if (cudaDeviceSynchronize() != cudaSuccess) rc = DAT_ERR_CUDA;
     dat_fused_destroy(plan);
     if (plan->stage) cudaFree(plan->stage);
+    if (plan->d_tile_base8) cudaFree(plan->d_tile_base8);
+    if (plan->d_partials8) cudaFree(plan->d_partials8);
     if (plan->ws) cudaFree(plan->ws);
     if (prev >= 0 && prev != plan->device) cudaSetDevice(prev);
     (void)cudaGetLastError();

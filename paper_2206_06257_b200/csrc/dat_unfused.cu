@@ -807,3 +807,186 @@ extern "C" int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_off
     if (cudaGetLastError() != cudaSuccess) return DAT_ERR_CUDA;
     return DAT_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// dat_step_passes: Steps 7, 9 and 12 of Algorithm A1 as three streaming passes without the
+// packed message -- norms; levels, signed sum over the workers, g_hat, m' and the layer sums
+// in one kernel (codes, sums and g_hat stay in registers); theta update.  The same arithmetic
+// as dat_step, element by element; what differs is that the gradients are read from memory
+// twice by construction and that the passes are separate launches.
+// ------------------------------------------------------------------------------------------
+#define DAT_QU_THREADS 256
+#ifndef DAT_QU_GROUPS
+#define DAT_QU_GROUPS 2                          // groups of 8 elements per thread
+#endif
+#ifndef DAT_QU_UNROLL
+#define DAT_QU_UNROLL 4                          // workers whose loads and Philox blocks are in flight together
+#endif
+#ifndef DAT_QU_MINB
+#define DAT_QU_MINB 4                            // resident CTAs per SM asked for (64 registers per thread): this pass lives on many warps
+#endif
+#define DAT_QU_TILE (DAT_QU_THREADS * 8 * DAT_QU_GROUPS)
+#define DAT_QU_PRAGMA(x) _Pragma(#x)
+#define DAT_QU_UNROLL_N(n) DAT_QU_PRAGMA(unroll n)
+
+template <bool RNG16>
+__global__ void __launch_bounds__(DAT_QU_THREADS, DAT_QU_MINB)
+k_quant_update(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, const int64_t *__restrict__ tile_base8,
+               int h, int M, const float *__restrict__ qmul, const float *__restrict__ dq, const float *__restrict__ theta,
+               float *__restrict__ mom, float S_f, float mu, float wd, double *__restrict__ partials,
+               int32_t *__restrict__ code_sum)
+{
+    __shared__ double scratch[DAT_THREADS / 32];
+    const int64_t tile = blockIdx.x;
+    const int layer = dat_find(tile_base8, h, tile);
+    const int64_t lo = __ldg(off + layer), hi = __ldg(off + layer + 1);
+    const int64_t begin = (lo & ~(int64_t)7) + (tile - __ldg(tile_base8 + layer)) * DAT_QU_TILE;
+    const float t = __ldg(qmul + layer), f = __ldg(dq + layer);
+    const float two_b = S_f + 1.0f, inv_two_b = 1.0f / two_b;
+    // scaled form of Eq. xi (see dat_step.cu): valid while t 2^-b is a normal number
+    const bool plain = (t != 0.0f) && !(t >= 1.17549435e-38f * two_b && t <= 3.402823466e38f);
+    const float ts = t * inv_two_b;
+    const float c0 = inv_two_b * (1.0f / 65536.0f), c1 = -127.0f * inv_two_b;
+    const uint32_t ubits = __float_as_uint(inv_two_b);
+    double ss_theta = 0.0, ss_u = 0.0;
+#pragma unroll 1
+    for (int k = 0; k < DAT_QU_GROUPS; ++k) {
+        const int64_t e0 = begin + 8 * (int64_t)(k * DAT_QU_THREADS + threadIdx.x);
+        if (e0 >= hi) continue;
+        const bool full = (e0 >= lo && e0 + 8 <= hi);
+        float acc[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+        DAT_QU_UNROLL_N(DAT_QU_UNROLL)
+        for (int i = 0; i < M; ++i) {
+            float v[8];
+            if (full) {
+                const float4 a0 = __ldcs(reinterpret_cast<const float4 *>(gp.p[i] + e0)), a1 = __ldcs(reinterpret_cast<const float4 *>(gp.p[i] + e0) + 1);
+                v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+            } else {
+                dat_load4(gp.p[i], e0, lo, hi, v);
+                dat_load4(gp.p[i], e0 + 4, lo, hi, v + 4);
+            }
+            uint32_t w[8];
+            if (RNG16) {
+                dat_random_words((uint64_t)e0 >> 3, (uint32_t)i, keys, w);
+            } else {
+                dat_random_words((uint64_t)e0 >> 2, (uint32_t)i, keys, w);
+                dat_random_words(((uint64_t)e0 >> 2) + 1, (uint32_t)i, keys, w + 4);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (!plain) {
+                    float u1s;
+                    if (RNG16) u1s = __fmaf_rn(__uint_as_float(__byte_perm(w[j >> 1], 0x4B000000u, (j & 1) ? 0x7632 : 0x7610)), c0, c1);
+                    else u1s = __uint_as_float(ubits | (w[j] & 0x007FFFFFu));
+                    const float ys = __saturatef(__fmaf_rn(fabsf(v[j]), ts, u1s));
+                    const float lf = __fmaf_rz(ys, two_b, 8388607.0f) - 8388608.0f;
+                    const float sg = __uint_as_float((__float_as_uint(v[j]) & 0x80000000u) | 0x3F800000u);
+                    acc[j] = __fmaf_rn(lf, sg, acc[j]);
+                } else {
+                    const float u1 = RNG16 ? dat_u1_from_half((j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xFFFFu)) : dat_u1_from_word(w[j]);
+                    const float lf = (float)dat_level_u1(v[j], t, two_b, u1);
+                    acc[j] += (v[j] < 0.0f) ? -lf : lf;
+                }
+            }
+        }
+        // theta and m only now: registers are what limits the number of resident warps here
+        float th[8], m[8];
+        if (full) {
+            const float4 t0 = __ldcg(reinterpret_cast<const float4 *>(theta + e0)), t1 = __ldcg(reinterpret_cast<const float4 *>(theta + e0) + 1);
+            const float4 m0 = __ldcs(reinterpret_cast<const float4 *>(mom + e0)), m1 = __ldcs(reinterpret_cast<const float4 *>(mom + e0) + 1);
+            th[0] = t0.x; th[1] = t0.y; th[2] = t0.z; th[3] = t0.w; th[4] = t1.x; th[5] = t1.y; th[6] = t1.z; th[7] = t1.w;
+            m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
+        } else {
+            dat_load4(theta, e0, lo, hi, th);
+            dat_load4(theta, e0 + 4, lo, hi, th + 4);
+            dat_load4(mom, e0, lo, hi, m);
+            dat_load4(mom, e0 + 4, lo, hi, m + 4);
+        }
+        if (code_sum) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (e0 + j >= lo && e0 + j < hi) code_sum[e0 + j] = (int)acc[j];
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            m[j] = __fmaf_rn(mu, m[j], __fmaf_rn(wd, th[j], acc[j] * f));
+            ss_theta = fma((double)th[j], (double)th[j], ss_theta);
+            ss_u = fma((double)m[j], (double)m[j], ss_u);
+        }
+        dat_store4(mom, e0, lo, hi, m);
+        dat_store4(mom, e0 + 4, lo, hi, m + 4);
+    }
+    const double a = dat_block_sum(ss_theta, scratch);
+    const double b = dat_block_sum(ss_u, scratch);
+    if (threadIdx.x == 0) { partials[2 * tile] = a; partials[2 * tile + 1] = b; }
+}
+
+extern "C" int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                               uint64_t seed, uint64_t step, const dat_hparams_t *hp,
+                               int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (!theta || !mom || !hp) return DAT_ERR_ARG;
+    if (plan->bits == 32 || plan->scale_mode != DAT_SCALE_SHARED_MAX) return DAT_ERR_UNSUPPORTED;
+    if (step >> 32) return DAT_ERR_ARG;
+    if (!dat_aligned16(theta) || !dat_aligned16(mom) || (code_sum_out && !dat_aligned16(code_sum_out)) ||
+        (layer_norms_out && !dat_aligned16(layer_norms_out)) || (scales_out && !dat_aligned16(scales_out)))
+        return DAT_ERR_ALIGN;
+    GradPtrs gp;
+    rc = dat_check_grads(plan, grads, &gp);
+    if (rc != DAT_OK) return rc;
+    const int h = (int)plan->h;
+    if (!plan->d_tile_base8) {      // first call: the tiling of the second pass (synchronous)
+        std::vector<int64_t> tb((size_t)h + 1);
+        int64_t nt = 0;
+        for (int l = 0; l < h; ++l) {
+            tb[l] = nt;
+            nt += (plan->offsets[l + 1] - (plan->offsets[l] & ~(int64_t)7) + DAT_QU_TILE - 1) / DAT_QU_TILE;
+        }
+        tb[h] = nt;
+        cudaError_t e = cudaMalloc((void **)&plan->d_tile_base8, ((size_t)h + 1) * 8);
+        if (e == cudaSuccess) e = cudaMalloc((void **)&plan->d_partials8, (size_t)nt * 16);
+        if (e == cudaSuccess) e = cudaMemcpy(plan->d_tile_base8, tb.data(), ((size_t)h + 1) * 8, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            if (plan->d_tile_base8) cudaFree(plan->d_tile_base8);
+            if (plan->d_partials8) cudaFree(plan->d_partials8);
+            plan->d_tile_base8 = nullptr;
+            plan->d_partials8 = nullptr;
+            plan->last_cuda = (int)e;
+            (void)cudaGetLastError();
+            return DAT_ERR_NOMEM;
+        }
+        plan->n_tiles8 = nt;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    const float S_f = (float)plan->S;
+    const float SM_f = (float)((uint64_t)plan->S * (uint64_t)plan->M);
+    dim3 ngrid((unsigned)plan->n_tiles, (unsigned)plan->M);
+    k_sumsq_partial<<<ngrid, DAT_THREADS, 0, s>>>(gp, plan->d_offsets, plan->d_tile_base, h, plan->M, plan->d_partials);
+    DAT_LAUNCHED(plan);
+    k_scales_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base, h, plan->M, S_f, plan->d_partials, plan->d_worker_norms,
+                                                plan->d_scales, plan->d_qmul, plan->d_status, false);
+    DAT_LAUNCHED(plan);
+    k_dq_from_scales<<<(h + 255) / 256, 256, 0, s>>>(h, SM_f, plan->d_scales, plan->d_dq);
+    DAT_LAUNCHED(plan);
+    if (scales_out) DAT_CUDA(plan, cudaMemcpyAsync(scales_out, plan->d_scales, (size_t)h * 4, cudaMemcpyDeviceToDevice, s));
+    const PhiloxKeys keys = dat_make_keys(seed, step);
+    if (plan->rng_bits == 16)
+        k_quant_update<true><<<(unsigned)plan->n_tiles8, DAT_QU_THREADS, 0, s>>>(gp, keys, plan->d_offsets, plan->d_tile_base8, h, plan->M,
+                                                                                 plan->d_qmul, plan->d_dq, theta, mom, S_f, hp->momentum,
+                                                                                 hp->weight_decay, plan->d_partials8, code_sum_out);
+    else
+        k_quant_update<false><<<(unsigned)plan->n_tiles8, DAT_QU_THREADS, 0, s>>>(gp, keys, plan->d_offsets, plan->d_tile_base8, h, plan->M,
+                                                                                  plan->d_qmul, plan->d_dq, theta, mom, S_f, hp->momentum,
+                                                                                  hp->weight_decay, plan->d_partials8, code_sum_out);
+    DAT_LAUNCHED(plan);
+    k_lalr_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base8, plan->d_partials8, hp->lr, hp->c_l, hp->c_u, plan->d_step_a,
+                                              layer_norms_out, plan->d_status);
+    DAT_LAUNCHED(plan);
+    k_lalr_pass2<<<(unsigned)plan->n_tiles, DAT_THREADS, 0, s>>>(theta, mom, plan->d_offsets, plan->d_tile_base, h, plan->d_step_a);
+    DAT_LAUNCHED(plan);
+    return DAT_OK;
+}

@@ -77,8 +77,9 @@ def _check_unfused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=
         return n_scale_mismatch
 
 
-def _check_fused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5, rng_bits=16):
+def _check_fused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5, rng_bits=16, entry="dat_step"):
     M = len(grads)
+    dat_step = getattr(api, entry)
     d = int(offs[-1])
     g_dev = [torch.from_numpy(g).cuda() for g in grads]
     with GpuPlan(api, offs, M, bits, rng_bits) as P:
@@ -86,7 +87,7 @@ def _check_fused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5,
         cs = torch.full((d,), 777, dtype=torch.int32, device="cuda")
         norms = torch.zeros(2 * P.h, dtype=torch.float32, device="cuda")
         sc = torch.zeros(P.h, dtype=torch.float32, device="cuda")
-        api.dat_step(P.plan, th_d, mo_d, g_dev, seed, step, hp, cs, norms, sc)
+        dat_step(P.plan, th_d, mo_d, g_dev, seed, step, hp, cs, norms, sc)
         torch.cuda.synchronize()
         assert P.status() == 0
         ref = oracle.step(offs, theta, mom, grads, bits, seed, step, *hp, rng_bits=rng_bits)
@@ -102,7 +103,7 @@ def _check_fused(api, oracle, offs, grads, theta, mom, bits, hp, seed=3, step=5,
         assert_close_per_layer(np_of(mo_d), ref["mom"], offs, "mom (fused)")
         # a second call on fresh copies gives bit-identical results (run-to-run determinism)
         th2, mo2 = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
-        api.dat_step(P.plan, th2, mo2, g_dev, seed, step, hp)
+        dat_step(P.plan, th2, mo2, g_dev, seed, step, hp)
         torch.cuda.synchronize()
         assert torch.equal(th2, th_d) and torch.equal(mo2, mo_d)
         return np_of(th_d), np_of(mo_d)
@@ -240,6 +241,49 @@ def test_fused_parity_ragged(api, oracle, bits, rng_bits):
 def test_fused_parity_worker_counts(api, oracle, M, rng_bits):
     offs, grads, theta, mom = _random_problem(M, [1000, 5000, 3, 9000], M, dist="t3")
     _check_fused(api, oracle, offs, grads, theta, mom, 4, HP, rng_bits=rng_bits)
+
+
+@pytest.mark.parametrize("bits", [1, 2, 4, 8, 16])
+def test_step_passes_parity_ragged(api, oracle, bits, rng_bits):
+    """The three-pass form of the step against the oracle, under the same protocol as the fused kernel."""
+    offs, grads, theta, mom = _random_problem(100 + bits, SIZES_RAGGED, 3)
+    _check_fused(api, oracle, offs, grads, theta, mom, bits, HP, rng_bits=rng_bits, entry="dat_step_passes")
+
+
+@pytest.mark.parametrize("M", [1, 5, 13, 64])
+def test_step_passes_worker_counts_and_extreme_scales(api, oracle, M, rng_bits):
+    offs, grads, theta, mom = _random_problem(M, [1000, 5000, 3, 9000], M, dist="t3")
+    grads = [g.copy() for g in grads]
+    for g in grads:
+        g[int(offs[1]):int(offs[2])] *= np.float32(1e30)      # a huge layer norm: the plain form takes over
+        g[int(offs[3]):] *= np.float32(1e-30)                 # a tiny one
+        g[int(offs[2]):int(offs[3])] = 0.0                    # a zero one
+    _check_fused(api, oracle, offs, grads, theta, mom, 8, HP, rng_bits=rng_bits, entry="dat_step_passes")
+
+
+def test_step_passes_equals_fused_on_resnet18(api, oracle):
+    from paper_2206_06257_b200 import synth
+    cfg = synth.config("resnet18")
+    theta, mom = synth.make_params(cfg, "cuda")
+    grads = synth.make_grads(cfg, 0, "cuda")
+    hp = hp_tuple(cfg)
+    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits, rng_bits=cfg.rng_bits)
+    try:
+        th1, mo1, th2, mo2 = theta.clone(), mom.clone(), theta.clone(), mom.clone()
+        cs1 = torch.zeros(cfg.d, dtype=torch.int32, device="cuda")
+        cs2 = torch.zeros(cfg.d, dtype=torch.int32, device="cuda")
+        sc1 = torch.zeros(cfg.h, device="cuda")
+        sc2 = torch.zeros(cfg.h, device="cuda")
+        api.dat_step(plan, th1, mo1, grads, 0, 4, hp, cs1, None, sc1)
+        api.dat_step_passes(plan, th2, mo2, grads, 0, 4, hp, cs2, None, sc2)
+        torch.cuda.synchronize()
+        assert ulp_diff(np_of(sc1), np_of(sc2)).max() <= 1
+        if torch.equal(sc1, sc2):                              # same norm bits: everything downstream is comparable bit for bit
+            assert torch.equal(cs1, cs2) and torch.equal(mo1, mo2)
+        assert_close_per_layer(np_of(th2), np_of(th1), cfg.offsets, "theta (passes vs fused)")
+        assert api.dat_get_status(plan) == 0
+    finally:
+        api.dat_plan_destroy(plan)
 
 
 @pytest.mark.parametrize("M", [9, 13, 64])
