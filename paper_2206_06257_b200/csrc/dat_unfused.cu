@@ -820,7 +820,7 @@ extern "C" int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_off
 #define DAT_QU_GROUPS 2                          // groups of 8 elements per thread
 #endif
 #ifndef DAT_QU_UNROLL
-#define DAT_QU_UNROLL 4                          // workers whose loads and Philox blocks are in flight together
+#define DAT_QU_UNROLL 2                          // workers whose loads and Philox blocks are in flight together
 #endif
 #ifndef DAT_QU_MINB
 #define DAT_QU_MINB 4                            // resident CTAs per SM asked for (64 registers per thread): this pass lives on many warps
