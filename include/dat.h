@@ -269,9 +269,11 @@ int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_offsets, float
                          const float *g_hat, const dat_hparams_t *hp, float *layer_norms_out, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
- * dat_step -- Steps 7, 9 and 12 of Algorithm A1 in one sweep: the result equals
+ * dat_step -- Steps 7, 9 and 12 of Algorithm A1 in one call: the result equals
  * dat_quantize -> dat_aggregate -> dat_lalr_step (or dat_average -> dat_lalr_step when b = 32),
- * but codes, code sums and g_hat are never written to device memory.
+ * but codes, code sums and g_hat are never written to device memory.  Inside, either one
+ * persistent kernel that sweeps the vectors once (dat_step_sweep) or three streaming passes
+ * (dat_step_passes), whichever is faster for the plan's size; both are also exported.
  *   theta, mom        device fp32[d], updated in place.
  *   grads             host array of M device pointers, fp32[d] each, read-only.
  *   seed, step        as in dat_quantize.
@@ -284,6 +286,13 @@ int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_offsets, float
 int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
              uint64_t seed, uint64_t step, const dat_hparams_t *hp,
              int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream);
+
+/* dat_step_sweep -- dat_step by the single persistent kernel, whatever the size (dat_step itself
+ * takes the three passes of dat_step_passes from 2^20 elements on, where they are faster, and this
+ * kernel below that).  Same arguments, results and errors as dat_step. */
+int dat_step_sweep(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                   uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
+                   float *layer_norms_out, float *scales_out, void *stream);
 
 /* dat_step_passes -- the same step as dat_step, with the same arguments and the same results bit for
  * bit up to the norms' last place, computed by three streaming passes in separate launches instead of

@@ -1253,9 +1253,9 @@ static int fused_prepare(dat_plan_t *plan)
     return DAT_OK;
 }
 
-extern "C" int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
-                        uint64_t seed, uint64_t step, const dat_hparams_t *hp,
-                        int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
+extern "C" int dat_step_sweep(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                              uint64_t seed, uint64_t step, const dat_hparams_t *hp,
+                              int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
 {
     int rc = dat_check_plan(plan);
     if (rc != DAT_OK) return rc;

@@ -1022,3 +1022,21 @@ extern "C" int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const
     DAT_LAUNCHED(plan);
     return DAT_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// dat_step: one call for Steps 7, 9 and 12.  Two implementations give the same results (the norms
+// may differ in their last place, everything else follows from them bit for bit): the single
+// persistent sweep (dat_step_sweep) and the three passes above (dat_step_passes).  The passes are
+// the faster of the two from about a million elements on (measured on ResNet-18 .. 1B-parameter
+// shapes, M = 6 .. 32); below that the sweep's single launch wins.
+// ------------------------------------------------------------------------------------------
+#define DAT_STEP_PASSES_FROM ((int64_t)1 << 20)
+
+extern "C" int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                        uint64_t seed, uint64_t step, const dat_hparams_t *hp,
+                        int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
+{
+    if (plan && plan->bits != 32 && plan->scale_mode == DAT_SCALE_SHARED_MAX && plan->d >= DAT_STEP_PASSES_FROM)
+        return dat_step_passes(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
+    return dat_step_sweep(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
+}

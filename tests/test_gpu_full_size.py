@@ -1,5 +1,6 @@
 """Parity at the full sizes of the workloads, in the launch configuration bench.py times
-(fused dat_step, inputs generated on the device).  The oracle recomputes sampled layers one by
+(dat_step, which takes the three passes at these sizes, and the persistent sweep by itself; inputs
+generated on the device).  The oracle recomputes sampled layers one by
 one (its window mode keeps the global element index, hence the same random stream); properties
 that hold at any size are checked on everything."""
 import numpy as np
@@ -11,7 +12,10 @@ from helpers import assert_close_per_layer, hp_tuple, np_of, ulp_diff
 pytestmark = pytest.mark.gpu
 
 
-def _run_and_check(oracle, cfg, sample_layers, step=0):
+ENTRIES = ["dat_step", "dat_step_sweep"]
+
+
+def _run_and_check(oracle, cfg, sample_layers, step=0, entry="dat_step"):
     from paper_2206_06257_b200 import api, synth
     dev = "cuda"
     theta, mom = synth.make_params(cfg, device=dev)
@@ -23,7 +27,7 @@ def _run_and_check(oracle, cfg, sample_layers, step=0):
         cs = torch.zeros(cfg.d, dtype=torch.int32, device=dev)
         sc = torch.zeros(cfg.h, dtype=torch.float32, device=dev)
         norms = torch.zeros(2 * cfg.h, dtype=torch.float32, device=dev)
-        api.dat_step(plan, theta, mom, grads, cfg.seed, step, hp, cs, norms, sc)
+        getattr(api, entry)(plan, theta, mom, grads, cfg.seed, step, hp, cs, norms, sc)
         torch.cuda.synchronize()
         assert api.dat_get_status(plan) == 0
     finally:
@@ -60,25 +64,28 @@ def _run_and_check(oracle, cfg, sample_layers, step=0):
     return theta, mom
 
 
-def test_resnet50_bench_configuration_every_layer(oracle):
+@pytest.mark.parametrize("entry", ENTRIES)
+def test_resnet50_bench_configuration_every_layer(oracle, entry):
     from paper_2206_06257_b200 import synth
     cfg = synth.config("resnet50")
-    _run_and_check(oracle, cfg, range(cfg.h))
+    _run_and_check(oracle, cfg, range(cfg.h), entry=entry)
 
 
-def test_resnet50_m32_b4_student_t_with_zero_layers(oracle):
+@pytest.mark.parametrize("entry", ENTRIES)
+def test_resnet50_m32_b4_student_t_with_zero_layers(oracle, entry):
     from paper_2206_06257_b200 import synth
     cfg = synth.config("resnet50_m32")
     zg, zp = cfg.zero_grad_layers[0], cfg.zero_param_layers[0]
     sample = sorted(set(list(range(0, cfg.h, 7)) + [zg, zp, 159, 160]))
     sample = [l for l in sample if cfg.offsets[l + 1] - cfg.offsets[l] <= 1_100_000]
-    theta, mom = _run_and_check(oracle, cfg, sample)
+    theta, mom = _run_and_check(oracle, cfg, sample, entry=entry)
     a, b = int(cfg.offsets[zp]), int(cfg.offsets[zp + 1])
     assert not theta[a:b].any() and mom[a:b].any()          # all-zero tensor does not move (c_l = 0)
 
 
+@pytest.mark.parametrize("entry", ENTRIES)
 @pytest.mark.parametrize("bits", [2, 8])
-def test_flat_1b_sampled_layers(oracle, bits):
+def test_flat_1b_sampled_layers(oracle, bits, entry):
     from paper_2206_06257_b200 import synth
     if torch.cuda.get_device_properties(0).total_memory < 80e9:
         pytest.skip("needs about 60 GB of device memory")
@@ -88,5 +95,5 @@ def test_flat_1b_sampled_layers(oracle, bits):
     sample = sorted(set([int(order[0]), int(order[1]), int(order[len(order) // 2]), int(order[len(order) // 3]),
                          0, cfg.h - 1, int(np.argmin(np.abs(sizes - 300_000)))]))
     sample = [l for l in sample if sizes[l] <= 2_000_000]
-    _run_and_check(oracle, cfg, sample)
+    _run_and_check(oracle, cfg, sample, entry=entry)
     torch.cuda.empty_cache()
