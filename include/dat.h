@@ -304,6 +304,12 @@ int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const float *con
                     uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
                     float *layer_norms_out, float *scales_out, void *stream);
 
+/* dat_plan_set_probe -- measurement aid: two CUDA events owned by the caller (cudaEvent_t passed as
+ * void*; NULL, NULL switches it off) that later calls of dat_step_passes (and of dat_step where it
+ * takes that path) record on their stream just before and just after k_quant_update, the largest
+ * kernel of the step.  The events must outlive those calls.  Errors: ARG. */
+int dat_plan_set_probe(dat_plan_t *plan, void *event_before, void *event_after);
+
 /* dat_step_host -- dat_step for callers whose data lives in HOST memory: copies theta, mom and
  * the M gradient buffers to plan-owned device staging buffers, runs dat_step, copies theta and
  * mom back, and synchronises `stream` before returning.

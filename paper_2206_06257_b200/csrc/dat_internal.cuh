@@ -57,6 +57,9 @@ struct dat_plan {
     double *d_partials8 = nullptr;     // 2 per tile
     int64_t n_tiles8 = 0;
 
+    // dat_plan_set_probe: events recorded around the second pass of dat_step_passes (measurement aid)
+    void *probe_before = nullptr, *probe_after = nullptr;
+
     // staging buffers of dat_step_host
     float *stage = nullptr;
 

@@ -1006,6 +1006,7 @@ extern "C" int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const
     DAT_LAUNCHED(plan);
     if (scales_out) DAT_CUDA(plan, cudaMemcpyAsync(scales_out, plan->d_scales, (size_t)h * 4, cudaMemcpyDeviceToDevice, s));
     const PhiloxKeys keys = dat_make_keys(seed, step);
+    if (plan->probe_before) DAT_CUDA(plan, cudaEventRecord((cudaEvent_t)plan->probe_before, s));
     if (plan->rng_bits == 16)
         k_quant_update<true><<<(unsigned)plan->n_tiles8, DAT_QU_THREADS, 0, s>>>(gp, keys, plan->d_offsets, plan->d_tile_base8, h, plan->M,
                                                                                  plan->d_qmul, plan->d_dq, theta, mom, S_f, hp->momentum,
@@ -1015,6 +1016,7 @@ extern "C" int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const
                                                                                   plan->d_qmul, plan->d_dq, theta, mom, S_f, hp->momentum,
                                                                                   hp->weight_decay, plan->d_partials8, code_sum_out);
     DAT_LAUNCHED(plan);
+    if (plan->probe_after) DAT_CUDA(plan, cudaEventRecord((cudaEvent_t)plan->probe_after, s));
     k_lalr_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base8, plan->d_partials8, hp->lr, hp->c_l, hp->c_u, plan->d_step_a,
                                               layer_norms_out, plan->d_status);
     DAT_LAUNCHED(plan);
@@ -1039,4 +1041,15 @@ extern "C" int dat_step(dat_plan_t *plan, float *theta, float *mom, const float 
     if (plan && plan->bits != 32 && plan->scale_mode == DAT_SCALE_SHARED_MAX && plan->d >= DAT_STEP_PASSES_FROM)
         return dat_step_passes(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
     return dat_step_sweep(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
+}
+
+// Measurement aid: two CUDA events of the caller's (or NULL, NULL to switch it off) that the next
+// calls of dat_step_passes record on their stream just before and just after k_quant_update, the
+// largest kernel of the step, so that its duration can be read without a profiler.
+extern "C" int dat_plan_set_probe(dat_plan_t *plan, void *event_before, void *event_after)
+{
+    if (!plan || ((event_before == nullptr) != (event_after == nullptr))) return DAT_ERR_ARG;
+    plan->probe_before = event_before;
+    plan->probe_after = event_after;
+    return DAT_OK;
 }
