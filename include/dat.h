@@ -304,6 +304,12 @@ int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const float *con
                     uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
                     float *layer_norms_out, float *scales_out, void *stream);
 
+/* dat_step_pipelined -- the same step as dat_step in one launch that reads every gradient from device
+ * memory once.  Same arguments, results and errors as dat_step. */
+int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                       uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
+                       float *layer_norms_out, float *scales_out, void *stream);
+
 /* dat_plan_set_probe -- measurement aid: two CUDA events owned by the caller (cudaEvent_t passed as
  * void*; NULL, NULL switches it off) that later calls of dat_step_passes (and of dat_step where it
  * takes that path) record on their stream just before and just after k_quant_update, the largest

@@ -12,11 +12,12 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libdat.so")
+# DAT_DEBUG=1 selects the self-checking build (python -m paper_2206_06257_b200.build with the same variable set)
+LIB_PATH = os.path.join(_HERE, "libdat_debug.so" if os.environ.get("DAT_DEBUG") == "1" else "libdat.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
-        "libdat.so is missing: build it with `python -m paper_2206_06257_b200.build` "
+        os.path.basename(LIB_PATH) + " is missing: build it with `python -m paper_2206_06257_b200.build` "
         "(needs nvcc; the CUDA library is the only implementation of this path)")
 _lib = C.CDLL(LIB_PATH)
 
@@ -30,7 +31,7 @@ DAT_STATUS_NONFINITE, DAT_STATUS_TIMEOUT, DAT_STATUS_BOUNDS = 1, 2, 4
 
 # every symbol include/dat.h declares
 EXPORTS = ["dat_plan_create", "dat_plan_destroy", "dat_plan_sizes", "dat_quantize", "dat_aggregate", "dat_requantize",
-           "dat_average", "dat_lalr_step", "dat_lamb_step", "dat_lalr_step_static", "dat_step", "dat_step_sweep", "dat_step_passes", "dat_plan_set_probe", "dat_step_host", "dat_get_status",
+           "dat_average", "dat_lalr_step", "dat_lamb_step", "dat_lalr_step_static", "dat_step", "dat_step_sweep", "dat_step_passes", "dat_step_pipelined", "dat_plan_set_probe", "dat_step_host", "dat_get_status",
            "dat_plan_launch_count", "dat_strerror", "dat_last_cuda_error"]
 
 
@@ -58,6 +59,7 @@ _lib.dat_lalr_step_static.argtypes = [_i64, _p, _p, _p, _p, C.POINTER(dat_hparam
 _lib.dat_step.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_plan_set_probe.argtypes = [_p, _p, _p]
 _lib.dat_step_sweep.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
+_lib.dat_step_pipelined.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_step_passes.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_step_host.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p]
 _lib.dat_get_status.argtypes = [_p, C.POINTER(C.c_uint32), _p]
@@ -207,6 +209,13 @@ def dat_step_passes(plan, theta, mom, grads, seed, step, hp, code_sum_out=None, 
     h = _hp(hp)
     _ok(_lib.dat_step_passes(_p(plan), _ptr(theta), _ptr(mom), _ptr_array(grads), int(seed), int(step), C.byref(h),
                              _ptr(code_sum_out), _ptr(layer_norms_out), _ptr(scales_out), _stream(stream)), "dat_step_passes")
+
+
+def dat_step_pipelined(plan, theta, mom, grads, seed, step, hp, code_sum_out=None, layer_norms_out=None,
+                     scales_out=None, stream=None):
+    h = _hp(hp)
+    _ok(_lib.dat_step_pipelined(_p(plan), _ptr(theta), _ptr(mom), _ptr_array(grads), int(seed), int(step), C.byref(h),
+                              _ptr(code_sum_out), _ptr(layer_norms_out), _ptr(scales_out), _stream(stream)), "dat_step_pipelined")
 
 
 def dat_step_host(plan, theta_host, mom_host, grads_host, seed, step, hp, stream=None):

@@ -10,15 +10,16 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
-LIB = os.path.join(HERE, "libdat.so")
-SOURCES = ["dat_plan.cu", "dat_unfused.cu", "dat_step.cu"]
+DEBUG = os.environ.get("DAT_DEBUG") == "1"        # the self-checking build: libdat_debug.so, with -DDAT_SELFCHECK
+LIB = os.path.join(HERE, "libdat_debug.so" if DEBUG else "libdat.so")
+SOURCES = ["dat_plan.cu", "dat_unfused.cu", "dat_step.cu", "dat_pipeline.cu"]
 HEADERS = [os.path.join(CSRC, "dat_internal.cuh"), os.path.join(ROOT, "include", "dat.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-fmad=false", "-Xcompiler", "-fPIC",
     "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-]
+] + (["-DDAT_SELFCHECK"] if DEBUG else [])
 
 
 def _nvcc():
@@ -34,7 +35,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest:
         return LIB
     objs = []
-    build_dir = os.path.join(HERE, "_build")
+    build_dir = os.path.join(HERE, "_build", "debug" if DEBUG else "release")
     os.makedirs(build_dir, exist_ok=True)
     procs = []
     for s in srcs:

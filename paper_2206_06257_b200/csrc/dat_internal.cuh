@@ -25,6 +25,7 @@ struct PhiloxKeys {
 };
 
 struct FusedSchedule;   // dat_step.cu
+struct PipeSchedule;    // dat_pipeline.cu
 
 struct dat_plan {
     int device = 0;
@@ -50,7 +51,8 @@ struct dat_plan {
     float *d_norms = nullptr;          // 2h
     uint32_t *d_status = nullptr;      // 1
 
-    FusedSchedule *fused = nullptr;    // built lazily by dat_step
+    FusedSchedule *fused = nullptr;    // built lazily by dat_step_sweep
+    PipeSchedule *pipe = nullptr;      // work items and tables of dat_step_pipelined, built with the plan
 
     // dat_step_passes: per-layer tiles that start on multiples of 8 elements, and their partial sums
     int64_t *d_tile_base8 = nullptr;   // h+1
@@ -75,6 +77,9 @@ bool dat_aligned16(const void *p);
 int dat_check_grads(const dat_plan_t *plan, const float *const *grads, GradPtrs *out);
 PhiloxKeys dat_make_keys(uint64_t seed, uint64_t step);
 void dat_fused_destroy(dat_plan_t *plan);                    // dat_step.cu
+int dat_pipe_build(dat_plan_t *plan);                        // dat_pipeline.cu (device current)
+void dat_pipe_destroy(dat_plan_t *plan);
+cudaError_t dat_pipe_reset(dat_plan_t *plan, cudaStream_t s);
 
 #define DAT_CUDA(plan, call)                                              \
     do {                                                                  \
@@ -256,6 +261,120 @@ __device__ __forceinline__ void dat_store4(float *__restrict__ p, int64_t e0, in
         for (int j = 0; j < 4; ++j)
             if (e0 + j >= lo && e0 + j < hi) p[e0 + j] = v[j];
     }
+}
+
+// ------------------------------------------------------------------------------------------
+// 16-byte global loads and stores that stay out of L1 and carry an L2 eviction priority.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t dat_policy_evict_last()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t dat_policy_evict_first()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t dat_policy_evict_normal()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ float4 dat_ld4_hint(const float *p, uint64_t pol)
+{
+    float4 v;
+    asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(pol));
+    return v;
+}
+__device__ __forceinline__ void dat_st4_hint(float *p, float4 v, uint64_t pol)
+{
+    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1,%2,%3,%4}, %5;"
+                 :: "l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(pol) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------
+// Levels and signed sum over the workers for one thread's group of eight consecutive elements
+// (Eq. xi, Eq. grad_agg), shared by the kernels that keep codes and sums in registers.
+// ------------------------------------------------------------------------------------------
+#define DAT_QU_THREADS 256
+#ifndef DAT_QU_GROUPS
+#define DAT_QU_GROUPS 2                          // groups of 8 elements per thread
+#endif
+#ifndef DAT_QU_UNROLL
+#define DAT_QU_UNROLL 2                          // workers whose loads and Philox blocks are in flight together
+#endif
+#ifndef DAT_QU_MINB
+#define DAT_QU_MINB 4                            // resident CTAs per SM asked for (64 registers per thread): this pass lives on many warps
+#endif
+#define DAT_QU_TILE (DAT_QU_THREADS * 8 * DAT_QU_GROUPS)
+#define DAT_QU_PRAGMA(x) _Pragma(#x)
+#define DAT_QU_UNROLL_N(n) DAT_QU_PRAGMA(unroll n)
+
+struct QuConst {
+    float t, ts, two_b, c0, c1;
+    uint32_t ubits;
+};
+
+// The M gradient rows of one group of eight elements: levels and signed sum.  FULL: the group lies
+// inside the layer (16-byte loads); PLAIN: the layer's scale is outside the range of the scaled
+// form.  The common case (FULL, not PLAIN) is inlined, the others are calls.
+template <bool RNG16, bool FULL, bool PLAIN>
+__device__ __forceinline__ void qu_rows_body(const GradPtrs &gp, const PhiloxKeys &keys, const QuConst &qc, int M, int64_t e0,
+                                             int64_t lo, int64_t hi, float acc[8])
+{
+    const uint64_t pol = dat_policy_evict_first();   // a gradient is dead once its level is drawn
+    DAT_QU_UNROLL_N(DAT_QU_UNROLL)
+    for (int i = 0; i < M; ++i) {
+        float v[8];
+        if (FULL) {
+            const float4 a0 = dat_ld4_hint(gp.p[i] + e0, pol), a1 = dat_ld4_hint(gp.p[i] + e0 + 4, pol);
+            v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+        } else {
+            dat_load4(gp.p[i], e0, lo, hi, v);
+            dat_load4(gp.p[i], e0 + 4, lo, hi, v + 4);
+        }
+        uint32_t w[8];
+        if (RNG16) {
+            dat_random_words((uint64_t)e0 >> 3, (uint32_t)i, keys, w);
+        } else {
+            dat_random_words((uint64_t)e0 >> 2, (uint32_t)i, keys, w);
+            dat_random_words(((uint64_t)e0 >> 2) + 1, (uint32_t)i, keys, w + 4);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (!PLAIN) {
+                float u1s;
+                if (RNG16) u1s = __fmaf_rn(__uint_as_float(__byte_perm(w[j >> 1], 0x4B000000u, (j & 1) ? 0x7632 : 0x7610)), qc.c0, qc.c1);
+                else u1s = __uint_as_float(qc.ubits | (w[j] & 0x007FFFFFu));
+                const float ys = __saturatef(__fmaf_rn(fabsf(v[j]), qc.ts, u1s));
+                const float lf = __fmaf_rz(ys, qc.two_b, 8388607.0f) - 8388608.0f;
+                const float sg = __uint_as_float((__float_as_uint(v[j]) & 0x80000000u) | 0x3F800000u);
+                acc[j] = __fmaf_rn(lf, sg, acc[j]);
+            } else {
+                const float u1 = RNG16 ? dat_u1_from_half((j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xFFFFu)) : dat_u1_from_word(w[j]);
+                const float lf = (float)dat_level_u1(v[j], qc.t, qc.two_b, u1);
+                acc[j] += (v[j] < 0.0f) ? -lf : lf;
+            }
+        }
+    }
+}
+template <bool RNG16, bool FULL, bool PLAIN>
+__device__ __noinline__ void qu_rows_call(const GradPtrs &gp, const PhiloxKeys &keys, const QuConst &qc, int M, int64_t e0,
+                                          int64_t lo, int64_t hi, float acc[8])
+{
+    qu_rows_body<RNG16, FULL, PLAIN>(gp, keys, qc, M, e0, lo, hi, acc);
+}
+template <bool RNG16, bool FULL, bool PLAIN>
+__device__ __forceinline__ void qu_rows(const GradPtrs &gp, const PhiloxKeys &keys, const QuConst &qc, int M, int64_t e0,
+                                        int64_t lo, int64_t hi, float acc[8])
+{
+    if (FULL && !PLAIN) qu_rows_body<RNG16, FULL, PLAIN>(gp, keys, qc, M, e0, lo, hi, acc);
+    else qu_rows_call<RNG16, FULL, PLAIN>(gp, keys, qc, M, e0, lo, hi, acc);
 }
 
 #endif  // __CUDACC__

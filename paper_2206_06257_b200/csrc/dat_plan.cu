@@ -126,6 +126,13 @@ extern "C" int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64
         (void)cudaGetLastError();
         return DAT_ERR_CUDA;
     }
+    const int rc = dat_pipe_build(p);
+    if (rc != DAT_OK) {
+        dat_pipe_destroy(p);
+        cudaFree(p->ws);
+        delete p;
+        return rc;
+    }
     *out = p;
     return DAT_OK;
 }
@@ -139,6 +146,7 @@ extern "C" int dat_plan_destroy(dat_plan_t *plan)
     if (prev != plan->device) cudaSetDevice(plan->device);
     if (cudaDeviceSynchronize() != cudaSuccess) rc = DAT_ERR_CUDA;
     dat_fused_destroy(plan);
+    dat_pipe_destroy(plan);
     if (plan->stage) cudaFree(plan->stage);
     if (plan->d_tile_base8) cudaFree(plan->d_tile_base8);
     if (plan->d_partials8) cudaFree(plan->d_partials8);
@@ -171,6 +179,10 @@ extern "C" int dat_get_status(dat_plan_t *plan, uint32_t *flags_out, void *strea
     DAT_CUDA(plan, cudaMemcpyAsync(&v, plan->d_status, sizeof v, cudaMemcpyDeviceToHost, s));
     DAT_CUDA(plan, cudaMemsetAsync(plan->d_status, 0, sizeof v, s));
     DAT_CUDA(plan, cudaStreamSynchronize(s));
+    if (v & DAT_STATUS_TIMEOUT) {       // the call that gave up left its counters mid-way
+        DAT_CUDA(plan, dat_pipe_reset(plan, s));
+        DAT_CUDA(plan, cudaStreamSynchronize(s));
+    }
     *flags_out = v;
     return DAT_OK;
 }

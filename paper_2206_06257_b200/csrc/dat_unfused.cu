@@ -815,81 +815,6 @@ extern "C" int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_off
 // as dat_step, element by element; what differs is that the gradients are read from memory
 // twice by construction and that the passes are separate launches.
 // ------------------------------------------------------------------------------------------
-#define DAT_QU_THREADS 256
-#ifndef DAT_QU_GROUPS
-#define DAT_QU_GROUPS 2                          // groups of 8 elements per thread
-#endif
-#ifndef DAT_QU_UNROLL
-#define DAT_QU_UNROLL 2                          // workers whose loads and Philox blocks are in flight together
-#endif
-#ifndef DAT_QU_MINB
-#define DAT_QU_MINB 4                            // resident CTAs per SM asked for (64 registers per thread): this pass lives on many warps
-#endif
-#define DAT_QU_TILE (DAT_QU_THREADS * 8 * DAT_QU_GROUPS)
-#define DAT_QU_PRAGMA(x) _Pragma(#x)
-#define DAT_QU_UNROLL_N(n) DAT_QU_PRAGMA(unroll n)
-
-struct QuConst {
-    float t, ts, two_b, c0, c1;
-    uint32_t ubits;
-};
-
-// The M gradient rows of one group of eight elements: levels and signed sum.  FULL: the group lies
-// inside the layer (16-byte loads); PLAIN: the layer's scale is outside the range of the scaled
-// form.  The common case (FULL, not PLAIN) is inlined, the others are calls.
-template <bool RNG16, bool FULL, bool PLAIN>
-__device__ __forceinline__ void qu_rows_body(const GradPtrs &gp, const PhiloxKeys &keys, const QuConst &qc, int M, int64_t e0,
-                                             int64_t lo, int64_t hi, float acc[8])
-{
-    DAT_QU_UNROLL_N(DAT_QU_UNROLL)
-    for (int i = 0; i < M; ++i) {
-        float v[8];
-        if (FULL) {
-            const float4 a0 = __ldcs(reinterpret_cast<const float4 *>(gp.p[i] + e0)), a1 = __ldcs(reinterpret_cast<const float4 *>(gp.p[i] + e0) + 1);
-            v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
-        } else {
-            dat_load4(gp.p[i], e0, lo, hi, v);
-            dat_load4(gp.p[i], e0 + 4, lo, hi, v + 4);
-        }
-        uint32_t w[8];
-        if (RNG16) {
-            dat_random_words((uint64_t)e0 >> 3, (uint32_t)i, keys, w);
-        } else {
-            dat_random_words((uint64_t)e0 >> 2, (uint32_t)i, keys, w);
-            dat_random_words(((uint64_t)e0 >> 2) + 1, (uint32_t)i, keys, w + 4);
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            if (!PLAIN) {
-                float u1s;
-                if (RNG16) u1s = __fmaf_rn(__uint_as_float(__byte_perm(w[j >> 1], 0x4B000000u, (j & 1) ? 0x7632 : 0x7610)), qc.c0, qc.c1);
-                else u1s = __uint_as_float(qc.ubits | (w[j] & 0x007FFFFFu));
-                const float ys = __saturatef(__fmaf_rn(fabsf(v[j]), qc.ts, u1s));
-                const float lf = __fmaf_rz(ys, qc.two_b, 8388607.0f) - 8388608.0f;
-                const float sg = __uint_as_float((__float_as_uint(v[j]) & 0x80000000u) | 0x3F800000u);
-                acc[j] = __fmaf_rn(lf, sg, acc[j]);
-            } else {
-                const float u1 = RNG16 ? dat_u1_from_half((j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xFFFFu)) : dat_u1_from_word(w[j]);
-                const float lf = (float)dat_level_u1(v[j], qc.t, qc.two_b, u1);
-                acc[j] += (v[j] < 0.0f) ? -lf : lf;
-            }
-        }
-    }
-}
-template <bool RNG16, bool FULL, bool PLAIN>
-__device__ __noinline__ void qu_rows_call(const GradPtrs &gp, const PhiloxKeys &keys, const QuConst &qc, int M, int64_t e0,
-                                          int64_t lo, int64_t hi, float acc[8])
-{
-    qu_rows_body<RNG16, FULL, PLAIN>(gp, keys, qc, M, e0, lo, hi, acc);
-}
-template <bool RNG16, bool FULL, bool PLAIN>
-__device__ __forceinline__ void qu_rows(const GradPtrs &gp, const PhiloxKeys &keys, const QuConst &qc, int M, int64_t e0,
-                                        int64_t lo, int64_t hi, float acc[8])
-{
-    if (FULL && !PLAIN) qu_rows_body<RNG16, FULL, PLAIN>(gp, keys, qc, M, e0, lo, hi, acc);
-    else qu_rows_call<RNG16, FULL, PLAIN>(gp, keys, qc, M, e0, lo, hi, acc);
-}
-
 template <bool RNG16>
 __global__ void __launch_bounds__(DAT_QU_THREADS, DAT_QU_MINB)
 k_quant_update(const __grid_constant__ GradPtrs gp, const __grid_constant__ PhiloxKeys keys, const int64_t *__restrict__ off, const int64_t *__restrict__ tile_base8,
@@ -1038,8 +963,8 @@ extern "C" int dat_step(dat_plan_t *plan, float *theta, float *mom, const float 
                         uint64_t seed, uint64_t step, const dat_hparams_t *hp,
                         int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
 {
-    if (plan && plan->bits != 32 && plan->scale_mode == DAT_SCALE_SHARED_MAX && plan->d >= DAT_STEP_PASSES_FROM)
-        return dat_step_passes(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
+    if (plan && (plan->bits == 32 || plan->scale_mode == DAT_SCALE_SHARED_MAX))
+        return dat_step_pipelined(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
     return dat_step_sweep(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
 }
 
