@@ -28,10 +28,33 @@ sys.path.insert(0, ROOT)
 METRIC = "worker-grad elems/s through quantize+aggregate+LALR"
 UNIT = "elems/s"
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_fused_step launch, from the ncu capture
-# summarised under profiles/ (None until taken for the kernel as it stands).
-NCU_DRAM_BYTES_PER_LAUNCH = {"resnet50_b8_rng16": 1930594816 + 157463552,                    # k_fused_step
-                             "k_quant_update_resnet50_b8_rng16": 1022409216 + 75441152}
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "traffic.json")
+
+
+def kernel_source_hash():
+    """sha256 over the CUDA sources of the library (what the ncu traffic figures are keyed by)."""
+    import hashlib
+    csrc = os.path.join(ROOT, "paper_2206_06257_b200", "csrc")
+    h = hashlib.sha256()
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            h.update(name.encode())
+            h.update(open(os.path.join(csrc, name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(path, cfg):
+    """DRAM bytes per step from the ncu capture summarised under profiles/ -- or None when no capture
+    exists for this path and workload, or when the kernels have changed since it was taken."""
+    try:
+        table = json.load(open(TRAFFIC_JSON))
+    except Exception:
+        return None, None
+    key = "%s:%s_m%d_b%d_rng%d" % (path, cfg.name, cfg.M, cfg.bits, cfg.rng_bits)
+    rec = table.get(key)
+    if not rec or rec.get("source_hash") != kernel_source_hash():
+        return None, None
+    return int(rec["dram_bytes_per_step"]), rec.get("summary")
 
 
 def measured_peaks():

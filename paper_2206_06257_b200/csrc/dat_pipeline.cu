@@ -24,7 +24,7 @@
 #define DAT_P_THREADS 256
 #define DAT_P_TILE 2048                           // elements per tile (eight per thread), tiles start on multiples of 8
 #ifndef DAT_P_MINB
-#define DAT_P_MINB 3
+#define DAT_P_MINB 4
 #endif
 #ifndef DAT_P_LAG                                 // items between the last N tile of a layer and its first Q tile
 #define DAT_P_LAG 384
@@ -39,8 +39,13 @@
 
 enum { P_MODE_SHARED = 0, P_MODE_IDENTITY = 2 };
 
-struct PipeItem {                                 // layer < 0: the item has no tile for that phase
-    int32_t ln, tn, lq, tq, lu, tu, pad0, pad1;
+struct PipePart {                                 // one tile of one layer; layer < 0: none
+    int64_t lo, hi;                               // the layer's element range
+    int32_t tb, T;                                // first tile of the layer in the partial-sum tables, tiles of the layer
+    int32_t layer, tile;
+};
+struct PipeItem {
+    PipePart n, q, u;
 };
 
 struct PipeSchedule {
@@ -145,12 +150,18 @@ __device__ __forceinline__ bool p_wait(const PArgs &a, const uint32_t *word, int
 }
 
 // ---- staging through shared memory ---------------------------------------------------------------
-// Every thread owns 16 slots of 16 bytes, slot k of thread t at p_stage[k * 256 + t]; it fills them
-// with asynchronous copies and reads back only its own, so the copies need no barrier, only the
-// thread's own wait for its copy groups.  What is in flight costs no registers.
+// Every thread streams its own sequence of 32-byte entries (two 16-byte slots) through a private
+// ring in shared memory: the parts of the N tile it sums, then for its eight elements of the Q tile
+// one entry per worker, theta and m, then theta and m' of its eight elements of the U tile.  Entry j
+// sits in ring position j mod DAT_P_DEPTH; it is fetched by two asynchronous 16-byte copies DEPTH
+// entries ahead of its use, across the borders of the three parts, and read back by the thread that
+// fetched it -- so the copies need no barrier, only the thread's own wait for its copy groups, and
+// what is in flight costs no registers.  Slot k of thread t is p_stage[k * 256 + t].
 extern __shared__ float4 p_stage[];
-#define DAT_P_SLOTS 16
-#define DAT_P_STAGE_BYTES (DAT_P_SLOTS * DAT_P_THREADS * 16)
+#ifndef DAT_P_DEPTH
+#define DAT_P_DEPTH 6
+#endif
+#define DAT_P_STAGE_BYTES (2 * DAT_P_DEPTH * DAT_P_THREADS * 16)
 
 // Self-checking build (-DDAT_SELFCHECK): every address formed from an item is checked before it is used;
 // a violation sets DAT_STATUS_BOUNDS and the access is skipped, nothing faults.
@@ -175,76 +186,77 @@ __device__ __forceinline__ void p_cp_commit() { asm volatile("cp.async.commit_gr
 template <int N>
 __device__ __forceinline__ void p_cp_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 
-// ---- N: sums of squares of one tile, every worker ------------------------------------------------
-// A tile is cut into 4M units (worker, quarter tile of 512 elements); warp w takes the units
-// [w*4M/8, (w+1)*4M/8), a unit being four 16-byte copies per lane.  Two units make a chunk; two chunks
-// are in flight.  Units of the same worker are summed per lane before the warp reduction; the
-// structure depends on M only, so the sums are the same from run to run.
-struct NormTile {
-    int64_t lo, hi, tb, begin;
-    uint32_t T;
-    bool full;
+// What a thread needs to know to fetch entry j of its sequence.
+struct Seq {
+    int nN, nQ, nU;                                // entries of the three parts (0: that part reads global memory itself)
+    int u0;                                        // N: first unit of this warp
+    int64_t eN, eQ, eU;                            // N: tile begin + 4 lane; Q, U: the thread's first element
+    uint64_t pol_last, pol_first, pol_normal;
 };
 
-__device__ __forceinline__ void p_norm_sums(const PArgs &a, const NormTile &nt, double *s_unit)
+__device__ __forceinline__ void p_issue(const PArgs &a, const Seq &q, int j)
 {
-    constexpr int QUARTER = DAT_P_TILE / 4;
-    static_assert(QUARTER == 4 * 128, "a unit is four 16-byte copies per lane");
+    float4 *dst = p_stage + (2 * (j % DAT_P_DEPTH)) * DAT_P_THREADS + threadIdx.x;
+    if (j < q.nN) {
+        // unit u = u0 + j/2 (worker u/4, quarter u%4), its copies 2(j%2) and 2(j%2)+1 of four
+        const int u = q.u0 + (j >> 1);
+        const int64_t e = q.eN + (u & 3) * (DAT_P_TILE / 4) + 256 * (j & 1);
+        p_cp16(a, dst, a.gp.p[u >> 2], e, q.pol_last);
+        p_cp16(a, dst + DAT_P_THREADS, a.gp.p[u >> 2], e + 128, q.pol_last);
+    } else if (j < q.nN + q.nQ) {
+        const int i = j - q.nN;
+        const float *base = (i < a.M) ? a.gp.p[i] : (i == a.M ? a.theta : a.mom);
+        const uint64_t pol = (i < a.M) ? q.pol_first : q.pol_normal;     // a gradient is dead once its level is drawn
+        p_cp16(a, dst, base, q.eQ, pol);
+        p_cp16(a, dst + DAT_P_THREADS, base, q.eQ + 4, pol);
+    } else if (j < q.nN + q.nQ + q.nU) {
+        const float *base = (j == q.nN + q.nQ) ? a.theta : a.mom;
+        p_cp16(a, dst, base, q.eU, q.pol_first);
+        p_cp16(a, dst + DAT_P_THREADS, base, q.eU + 4, q.pol_first);
+    }
+    p_cp_commit();                                 // one group per entry, also past the end: the count stays uniform
+}
+
+// Entry j has arrived (every entry up to j + DEPTH - 1 has been issued): its eight floats.
+__device__ __forceinline__ void p_take(int j, float v[8])
+{
+    p_cp_wait<DAT_P_DEPTH - 1>();
+    const float4 *src = p_stage + (2 * (j % DAT_P_DEPTH)) * DAT_P_THREADS + threadIdx.x;
+    const float4 a0 = src[0], a1 = src[DAT_P_THREADS];
+    v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+}
+
+// ---- N: sums of squares of one tile, every worker ------------------------------------------------
+// A tile is cut into 4M units (worker, quarter tile of 512 elements); warp w takes the units
+// [w*4M/8, (w+1)*4M/8), a unit being two entries per lane.  Units of the same worker are summed per
+// lane before the warp reduction; the structure depends on M only, so the sums are the same from
+// run to run.
+__device__ __forceinline__ void p_norm_sums(const PArgs &a, const PipePart &pt, const Seq &q, double *s_unit)
+{
     const int M = a.M;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int U = 4 * M;
-    for (int u = threadIdx.x; u < U; u += DAT_P_THREADS) s_unit[u] = 0.0;
-    __syncthreads();
     const int u0 = warp * U / 8, u1 = (warp + 1) * U / 8;
     double acc = 0.0;
     int run = u0;
-    float4 *mine = p_stage + threadIdx.x;
-    if (nt.full) {
-        const uint64_t pol = DAT_P_N_POLICY();
-        const int nchunks = (u1 - u0 + 1) >> 1;
-        auto issue = [&](int c) {
-            if (c < nchunks) {
-#pragma unroll
-                for (int uu = 0; uu < 2; ++uu) {
-                    const int u = u0 + 2 * c + uu;
-                    if (u < u1) {
-                        const int64_t e = nt.begin + (u & 3) * QUARTER + 4 * lane;
-#pragma unroll
-                        for (int b = 0; b < 4; ++b) p_cp16(a, mine + ((c & 1) * 8 + uu * 4 + b) * DAT_P_THREADS, a.gp.p[u >> 2], e + 128 * b, pol);
-                    }
-                }
-            }
-            p_cp_commit();
-        };
-        issue(0);
-        issue(1);
+    if (q.nN > 0) {
 #pragma unroll 1
-        for (int c = 0; c < nchunks; ++c) {
-            p_cp_wait<1>();
-#pragma unroll
-            for (int uu = 0; uu < 2; ++uu) {
-                const int u = u0 + 2 * c + uu;
-                if (u < u1) {
-                    if ((u >> 2) != (run >> 2)) {
-                        acc = dat_warp_sum(acc);
-                        if (lane == 0) s_unit[run] = acc;
-                        acc = 0.0;
-                        run = u;
-                    }
-#pragma unroll
-                    for (int b = 0; b < 4; ++b) {
-                        const float4 v = mine[((c & 1) * 8 + uu * 4 + b) * DAT_P_THREADS];
-                        acc = fma((double)v.x, (double)v.x, acc);
-                        acc = fma((double)v.y, (double)v.y, acc);
-                        acc = fma((double)v.z, (double)v.z, acc);
-                        acc = fma((double)v.w, (double)v.w, acc);
-                    }
-                }
+        for (int j = 0; j < q.nN; ++j) {
+            const int u = u0 + (j >> 1);
+            if ((u >> 2) != (run >> 2)) {
+                acc = dat_warp_sum(acc);
+                if (lane == 0) s_unit[run] = acc;
+                acc = 0.0;
+                run = u;
             }
-            issue(c + 2);                          // into the slots just read
+            float v[8];
+            p_take(j, v);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc = fma((double)v[k], (double)v[k], acc);
+            p_issue(a, q, j + DAT_P_DEPTH);        // into the slots just read
         }
-        p_cp_wait<0>();
     } else {
+        const int64_t begin = (pt.lo & ~(int64_t)7) + (int64_t)pt.tile * DAT_P_TILE;
 #pragma unroll 1
         for (int u = u0; u < u1; ++u) {
             if ((u >> 2) != (run >> 2)) {
@@ -254,13 +266,13 @@ __device__ __forceinline__ void p_norm_sums(const PArgs &a, const NormTile &nt, 
                 run = u;
             }
             const float *__restrict__ g = a.gp.p[u >> 2];
-            const int64_t e = nt.begin + (u & 3) * QUARTER + 4 * lane;
+            const int64_t e = begin + (u & 3) * (DAT_P_TILE / 4) + 4 * lane;
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
                 float t[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                if (e + 128 * b < nt.hi) dat_load4(g, e + 128 * b, nt.lo, nt.hi, t);
+                if (e + 128 * b < pt.hi) dat_load4(g, e + 128 * b, pt.lo, pt.hi, t);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) acc = fma((double)t[j], (double)t[j], acc);
+                for (int k = 0; k < 4; ++k) acc = fma((double)t[k], (double)t[k], acc);
             }
         }
     }
@@ -268,20 +280,20 @@ __device__ __forceinline__ void p_norm_sums(const PArgs &a, const NormTile &nt, 
         acc = dat_warp_sum(acc);
         if (lane == 0) s_unit[run] = acc;
     }
-    __syncthreads();
 }
 
 // Writes the tile's M partial sums, counts the tile in, and in the CTA that holds the layer's last
 // tile: nu_{i,l} = sqrt(sum over the tiles), nu_l = max_i, and the layer's two factors.
-__device__ __forceinline__ void p_norm_publish(const PArgs &a, int layer, int tile, const NormTile &nt, double *s_unit, float *s_norm, int *s_flag)
+__device__ __forceinline__ void p_norm_publish(const PArgs &a, const PipePart &pt, double *s_unit, float *s_norm, int *s_flag)
 {
-    const int M = a.M;
+    const int M = a.M, layer = pt.layer;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t tb = nt.tb;
-    const uint32_t T = nt.T;
+    const int64_t tb = pt.tb;
+    const uint32_t T = (uint32_t)pt.T;
+    __syncthreads();                               // every warp's unit sums are in s_unit
     if (threadIdx.x < M) {
         const double *s = s_unit + 4 * threadIdx.x;
-        a.partN[(tb + tile) * M + threadIdx.x] = ((s[0] + s[1]) + s[2]) + s[3];
+        a.partN[(tb + pt.tile) * M + threadIdx.x] = ((s[0] + s[1]) + s[2]) + s[3];
         __threadfence();
     }
     if (!p_arrive(a.cntN + layer, T, s_flag)) return;
@@ -343,42 +355,6 @@ __device__ __forceinline__ void p_finish_update_sums(const PArgs &a, int layer, 
     }
 }
 
-// ---- Q: levels (Eq. xi), signed sum over the workers and g_hat (Eq. grad_agg), m' and the layer sums
-// (Eq. 3, pass 1) of one tile; codes, sums and g_hat stay in registers ----------------------------
-// The gradients of a full tile are fetched ahead: a stage is one pair of workers (the thread's eight
-// elements of each, four slots), four stages in flight, the first four issued by p_quant_prefetch as
-// soon as the staging slots are free -- before the CTA knows whether the layer's norm is published.
-struct QuantTile {
-    int64_t lo, hi, tb, begin;
-    uint32_t T;
-    bool staged;                                   // every thread's eight elements lie inside the layer
-};
-
-__device__ __forceinline__ void p_quant_issue(const PArgs &a, int64_t e0, int t, int trips, uint64_t pol)
-{
-    if (t < trips) {
-        float4 *dst = p_stage + ((t & 3) * 4) * DAT_P_THREADS + threadIdx.x;
-        const int i0 = 2 * t, i1 = 2 * t + 1;
-        p_cp16(a, dst, a.gp.p[i0], e0, pol);
-        p_cp16(a, dst + DAT_P_THREADS, a.gp.p[i0], e0 + 4, pol);
-        if (i1 < a.M) {
-            p_cp16(a, dst + 2 * DAT_P_THREADS, a.gp.p[i1], e0, pol);
-            p_cp16(a, dst + 3 * DAT_P_THREADS, a.gp.p[i1], e0 + 4, pol);
-        }
-    }
-    p_cp_commit();
-}
-
-__device__ __forceinline__ void p_quant_prefetch(const PArgs &a, const QuantTile &qt)
-{
-    if (!qt.staged) return;
-    const int64_t e0 = qt.begin + 8 * (int64_t)threadIdx.x;
-    const int trips = (a.M + 1) >> 1;
-    const uint64_t pol = dat_policy_evict_first();   // a gradient is dead once its level is drawn
-#pragma unroll
-    for (int t = 0; t < 4; ++t) p_quant_issue(a, e0, t, trips, pol);
-}
-
 // One worker's eight elements: levels by the scaled form of Eq. xi, signed float sum (exact).
 template <bool RNG16>
 __device__ __forceinline__ void p_levels8(const float v[8], const uint32_t w[8], const QuConst &qc, float acc[8])
@@ -406,40 +382,13 @@ __device__ __forceinline__ void p_words8(const PArgs &a, int64_t e0, uint32_t wo
     }
 }
 
-__device__ __forceinline__ void p_unpack8(const float4 *slot, float v[8])
-{
-    const float4 a0 = slot[0], a1 = slot[DAT_P_THREADS];
-    v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
-}
-
-// The staged worker loop (prefetched by p_quant_prefetch).
-template <bool RNG16>
-__device__ __forceinline__ void p_rows_staged(const PArgs &a, const QuConst &qc, int64_t e0, float acc[8])
-{
-    const int M = a.M, trips = (M + 1) >> 1;
-    const uint64_t pol = dat_policy_evict_first();
-#pragma unroll 1
-    for (int t = 0; t < trips; ++t) {
-        p_cp_wait<3>();
-        const float4 *src = p_stage + ((t & 3) * 4) * DAT_P_THREADS + threadIdx.x;
-        const bool two = (2 * t + 1 < M);
-        float v0[8], v1[8];
-        p_unpack8(src, v0);
-        if (two) p_unpack8(src + 2 * DAT_P_THREADS, v1);
-        uint32_t w0[8], w1[8];
-        p_words8<RNG16>(a, e0, (uint32_t)(2 * t), w0);
-        if (two) p_words8<RNG16>(a, e0, (uint32_t)(2 * t + 1), w1);
-        p_levels8<RNG16>(v0, w0, qc, acc);
-        if (two) p_levels8<RNG16>(v1, w1, qc, acc);
-        p_quant_issue(a, e0, t + 4, trips, pol);   // into the slots just read
-    }
-}
-
+// ---- Q: levels (Eq. xi), signed sum over the workers and g_hat (Eq. grad_agg), m' and the layer sums
+// (Eq. 3, pass 1) of one tile; codes, sums and g_hat stay in registers ----------------------------
 template <bool RNG16, int MODE>
-__device__ __forceinline__ void p_part_quant(const PArgs &a, int layer, int tile, const QuantTile &qt, double *scratch, int *s_flag)
+__device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt, const Seq &q, double *scratch, int *s_flag)
 {
-    const int M = a.M;
-    const int64_t lo = qt.lo, hi = qt.hi;
+    const int M = a.M, layer = pt.layer;
+    const int64_t lo = pt.lo, hi = pt.hi;
     float t = 0.0f, f = 0.0f;
     if (MODE != P_MODE_IDENTITY) { t = __ldcg(a.qmul + layer); f = __ldcg(a.dq + layer); }
     const float two_b = a.S_f + 1.0f, inv_two_b = 1.0f / two_b;
@@ -447,13 +396,26 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, int layer, int tile
     const bool plain = (t != 0.0f) && !(t >= 1.17549435e-38f * two_b && t <= 3.402823466e38f);
     const QuConst qc = {t, t * inv_two_b, two_b, inv_two_b * (1.0f / 65536.0f), -127.0f * inv_two_b, __float_as_uint(inv_two_b)};
     double ss_theta = 0.0, ss_u = 0.0;
-    const int64_t e0 = qt.begin + 8 * (int64_t)threadIdx.x;
-    if (qt.staged && plain) p_cp_wait<0>();        // what was fetched ahead is not used: the general form reads for itself
+    const int64_t e0 = q.eQ;
+    const bool staged = q.nQ > 0;                  // the whole tile lies inside the layer and its rows were fetched ahead
     if (e0 < hi) {
         const bool full = (e0 >= lo && e0 + 8 <= hi);
         float acc[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+        if (staged) {
+#pragma unroll 1
+            for (int i = 0; i < M; ++i) {
+                float v[8];
+                p_take(q.nN + i, v);
+                if (!plain) {                       // nearly always
+                    uint32_t w[8];
+                    p_words8<RNG16>(a, e0, (uint32_t)i, w);
+                    p_levels8<RNG16>(v, w, qc, acc);
+                }
+                p_issue(a, q, q.nN + i + DAT_P_DEPTH);
+            }
+        }
         if (MODE == P_MODE_IDENTITY) {
 #pragma unroll 2
             for (int i = 0; i < M; ++i) {           // Q is the identity: the ordered fp32 sum of the workers' gradients
@@ -463,16 +425,23 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, int layer, int tile
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc[j] += v[j];
             }
-        } else if (qt.staged && !plain) p_rows_staged<RNG16>(a, qc, e0, acc);                        // nearly always
+        } else if (staged && !plain) { }
         else if (full && !plain) qu_rows<RNG16, true, false>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         else if (full) qu_rows<RNG16, true, true>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         else if (!plain) qu_rows<RNG16, false, false>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         else qu_rows<RNG16, false, true>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         float th[8], m[8];
-        p_load4_cg(a.theta, e0, lo, hi, th);
-        p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
-        p_load4_cg(a.mom, e0, lo, hi, m);
-        p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
+        if (staged) {
+            p_take(q.nN + M, th);
+            p_issue(a, q, q.nN + M + DAT_P_DEPTH);
+            p_take(q.nN + M + 1, m);
+            p_issue(a, q, q.nN + M + 1 + DAT_P_DEPTH);
+        } else {
+            p_load4_cg(a.theta, e0, lo, hi, th);
+            p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
+            p_load4_cg(a.mom, e0, lo, hi, m);
+            p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
+        }
         if (MODE != P_MODE_IDENTITY && a.code_sum) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -488,45 +457,52 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, int layer, int tile
         dat_store4(a.mom, e0, lo, hi, m);
         dat_store4(a.mom, e0 + 4, lo, hi, m + 4);
     }
-    p_cp_wait<0>();
     __threadfence();                               // m' is read by the U part of another CTA
     const double x = dat_block_sum(ss_theta, scratch);
     const double y = dat_block_sum(ss_u, scratch);
     if (threadIdx.x == 0) {
-        a.partQ[2 * (qt.tb + tile)] = x;
-        a.partQ[2 * (qt.tb + tile) + 1] = y;
+        a.partQ[2 * (pt.tb + pt.tile)] = x;
+        a.partQ[2 * (pt.tb + pt.tile) + 1] = y;
         __threadfence();
     }
-    if (p_arrive(a.cntQ + layer, qt.T, s_flag)) p_finish_update_sums(a, layer, qt.tb, qt.T, scratch);
+    if (p_arrive(a.cntQ + layer, (uint32_t)pt.T, s_flag)) p_finish_update_sums(a, layer, pt.tb, (uint32_t)pt.T, scratch);
 }
 
 // ---- U: theta' = theta - a_l m' (Eq. 3, pass 2) of one tile ---------------------------------------
-__device__ __forceinline__ void p_part_update(const PArgs &a, int layer, int tile)
+__device__ __forceinline__ void p_part_update(const PArgs &a, const PipePart &pt, const Seq &q)
 {
-    const int64_t lo = __ldg(a.off + layer), hi = __ldg(a.off + layer + 1);
-    const int64_t begin = (lo & ~(int64_t)7) + (int64_t)tile * DAT_P_TILE;
-    const float na = -__ldcg(a.step_a + layer);
-    const uint64_t pol_first = dat_policy_evict_first();
-    const int64_t e0 = begin + 8 * (int64_t)threadIdx.x;
+    const int64_t lo = pt.lo, hi = pt.hi;
+    const float na = -__ldcg(a.step_a + pt.layer);
+    const int64_t e0 = q.eU;
     if (e0 >= hi) return;
-    if (e0 >= lo && e0 + 8 <= hi) {
-        float4 t0 = dat_ld4_hint(a.theta + e0, pol_first), t1 = dat_ld4_hint(a.theta + e0 + 4, pol_first);
-        const float4 m0 = dat_ld4_hint(a.mom + e0, pol_first), m1 = dat_ld4_hint(a.mom + e0 + 4, pol_first);
-        t0.x = __fmaf_rn(na, m0.x, t0.x); t0.y = __fmaf_rn(na, m0.y, t0.y); t0.z = __fmaf_rn(na, m0.z, t0.z); t0.w = __fmaf_rn(na, m0.w, t0.w);
-        t1.x = __fmaf_rn(na, m1.x, t1.x); t1.y = __fmaf_rn(na, m1.y, t1.y); t1.z = __fmaf_rn(na, m1.z, t1.z); t1.w = __fmaf_rn(na, m1.w, t1.w);
-        dat_st4_hint(a.theta + e0, t0, pol_first);
-        dat_st4_hint(a.theta + e0 + 4, t1, pol_first);
+    float th[8], m[8];
+    if (q.nU > 0) {
+        p_take(q.nN + q.nQ, th);
+        p_issue(a, q, q.nN + q.nQ + DAT_P_DEPTH);
+        p_take(q.nN + q.nQ + 1, m);
+        p_issue(a, q, q.nN + q.nQ + 1 + DAT_P_DEPTH);
     } else {
-        float th[8], m[8];
         p_load4_cg(a.theta, e0, lo, hi, th);
         p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
         p_load4_cg(a.mom, e0, lo, hi, m);
         p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
+    }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) th[j] = __fmaf_rn(na, m[j], th[j]);
+    for (int j = 0; j < 8; ++j) th[j] = __fmaf_rn(na, m[j], th[j]);
+    if (e0 >= lo && e0 + 8 <= hi) {
+        const uint64_t pol_first = q.pol_first;
+        dat_st4_hint(a.theta + e0, make_float4(th[0], th[1], th[2], th[3]), pol_first);
+        dat_st4_hint(a.theta + e0 + 4, make_float4(th[4], th[5], th[6], th[7]), pol_first);
+    } else {
         dat_store4(a.theta, e0, lo, hi, th);
         dat_store4(a.theta, e0 + 4, lo, hi, th + 4);
     }
+}
+
+__device__ __forceinline__ bool p_tile_inside(const PipePart &pt)
+{
+    const int64_t begin = (pt.lo & ~(int64_t)7) + (int64_t)pt.tile * DAT_P_TILE;
+    return begin >= pt.lo && begin + DAT_P_TILE <= pt.hi;
 }
 
 template <bool RNG16, int MODE>
@@ -535,54 +511,74 @@ k_step_pipelined(const __grid_constant__ PArgs a)
 {
     __shared__ double s_unit[4 * DAT_MAX_WORKERS];
     __shared__ float s_norm[DAT_MAX_WORKERS];
+    __shared__ __align__(16) PipeItem s_item;
     __shared__ int s_flag;
-    __shared__ uint32_t s_ticket;
+    __shared__ int s_seen[2];                      // the layers this item waits for were already published when it started
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // items are taken in the order in which CTAs start, whatever order the hardware starts them in
-    if (threadIdx.x == 0) {
-        const uint32_t tk = atomicAdd(a.ticket, 1u);
-        if (tk == a.n_items - 1u) *a.ticket = 0u;      // every ticket of this call is out: ready for the next call
-        s_ticket = tk;
+    if (warp == 0) {
+        uint32_t tk = 0;
+        if (lane == 0) {
+            tk = atomicAdd(a.ticket, 1u);
+            if (tk == a.n_items - 1u) *a.ticket = 0u;  // every ticket of this call is out: ready for the next call
+        }
+        tk = __shfl_sync(0xFFFFFFFFu, tk, 0);
+        if (!P_CHECK(a, tk < a.n_items)) tk = 0;
+        if (lane < (int)(sizeof(PipeItem) / 16))
+            reinterpret_cast<uint4 *>(&s_item)[lane] = __ldg(reinterpret_cast<const uint4 *>(a.items + tk) + lane);
     }
+    for (int u = threadIdx.x; u < 4 * a.M; u += DAT_P_THREADS) s_unit[u] = 0.0;
     __syncthreads();
-    if (!P_CHECK(a, s_ticket < a.n_items)) return;
-    const PipeItem it = a.items[s_ticket];
+    const PipePart pn = s_item.n, pq = s_item.q, pu = s_item.u;
 #ifdef DAT_SELFCHECK
     {
-        bool ok = it.ln < a.h && it.lq < a.h && it.lu < a.h;
-        if (ok && it.ln >= 0) ok = it.tn >= 0 && it.tn < a.tile_base[it.ln + 1] - a.tile_base[it.ln] && a.tile_base[it.ln] + it.tn < a.n_tiles && a.off[it.ln + 1] <= a.d;
-        if (ok && it.lq >= 0) ok = it.tq >= 0 && it.tq < a.tile_base[it.lq + 1] - a.tile_base[it.lq] && a.tile_base[it.lq] + it.tq < a.n_tiles && a.off[it.lq + 1] <= a.d;
-        if (ok && it.lu >= 0) ok = it.tu >= 0 && it.tu < a.tile_base[it.lu + 1] - a.tile_base[it.lu] && a.off[it.lu + 1] <= a.d;
+        bool ok = pn.layer < a.h && pq.layer < a.h && pu.layer < a.h;
+        const PipePart *pp[3] = {&pn, &pq, &pu};
+        for (int k = 0; k < 3 && ok; ++k)
+            if (pp[k]->layer >= 0)
+                ok = pp[k]->tile >= 0 && pp[k]->tile < pp[k]->T && (int64_t)pp[k]->tb + pp[k]->tile < a.n_tiles &&
+                     pp[k]->lo >= 0 && pp[k]->lo < pp[k]->hi && pp[k]->hi <= a.d;
         if (!P_CHECK(a, ok)) return;
     }
 #endif
-    NormTile nt;
-    QuantTile qt;
-    if (it.ln >= 0) {
-        nt.lo = __ldg(a.off + it.ln); nt.hi = __ldg(a.off + it.ln + 1);
-        nt.tb = __ldg(a.tile_base + it.ln);
-        nt.T = (uint32_t)(__ldg(a.tile_base + it.ln + 1) - nt.tb);
-        nt.begin = (nt.lo & ~(int64_t)7) + (int64_t)it.tn * DAT_P_TILE;
-        nt.full = nt.begin >= nt.lo && nt.begin + DAT_P_TILE <= nt.hi;
-        p_norm_sums(a, nt, s_unit);
+    // what the other two parts wait for: look now, so that the answer is there when it is needed
+    if (threadIdx.x < 2) {
+        const bool want = (threadIdx.x == 0) ? (pq.layer >= 0 && MODE != P_MODE_IDENTITY) : (pu.layer >= 0);
+        const uint32_t *word = (threadIdx.x == 0) ? a.readyN + pq.layer : a.readyQ + pu.layer;
+        s_seen[threadIdx.x] = want ? (p_ld_acquire(word) == a.epoch) : 1;
     }
-    if (it.lq >= 0) {
-        qt.lo = __ldg(a.off + it.lq); qt.hi = __ldg(a.off + it.lq + 1);
-        qt.tb = __ldg(a.tile_base + it.lq);
-        qt.T = (uint32_t)(__ldg(a.tile_base + it.lq + 1) - qt.tb);
-        qt.begin = (qt.lo & ~(int64_t)7) + (int64_t)it.tq * DAT_P_TILE;
-        // (without quantisation the rows are read straight from global memory: there is no arithmetic to hide them behind)
-        qt.staged = MODE != P_MODE_IDENTITY && qt.begin >= qt.lo && qt.begin + DAT_P_TILE <= qt.hi;
-        p_quant_prefetch(a, qt);                   // the staging slots are free again: the copies run beside what follows
+    // the thread's sequence of entries
+    Seq q;
+    q.pol_last = DAT_P_N_POLICY();
+    q.pol_first = dat_policy_evict_first();
+    q.pol_normal = dat_policy_evict_normal();
+    q.u0 = warp * (4 * a.M) / 8;
+    q.nN = (pn.layer >= 0 && p_tile_inside(pn)) ? 2 * ((warp + 1) * (4 * a.M) / 8 - q.u0) : 0;
+    q.nQ = (pq.layer >= 0 && MODE != P_MODE_IDENTITY && p_tile_inside(pq)) ? a.M + 2 : 0;
+    q.nU = 0;                                      // known once s_seen[1] is
+    q.eN = (pn.lo & ~(int64_t)7) + (int64_t)pn.tile * DAT_P_TILE + 4 * lane;
+    q.eQ = (pq.lo & ~(int64_t)7) + (int64_t)pq.tile * DAT_P_TILE + 8 * (int64_t)threadIdx.x;
+    q.eU = (pu.lo & ~(int64_t)7) + (int64_t)pu.tile * DAT_P_TILE + 8 * (int64_t)threadIdx.x;
+    // DEPTH entries ahead; the first DEPTH entries never reach the U part unless N and Q are both absent or short,
+    // in which case U is fetched the plain way
+#pragma unroll
+    for (int j = 0; j < DAT_P_DEPTH; ++j) p_issue(a, q, j);
+
+    if (pn.layer >= 0) p_norm_sums(a, pn, q, s_unit);
+    __syncthreads();                               // s_seen is there (and every warp's unit sums)
+    // m' of the U tile may be fetched ahead only if its layer was seen published (then it is visible)
+    if (pu.layer >= 0 && s_seen[1] && p_tile_inside(pu) && q.nQ >= DAT_P_DEPTH) q.nU = 2;    // (its entries have not been passed yet)
+    if (pn.layer >= 0) p_norm_publish(a, pn, s_unit, s_norm, &s_flag);
+    bool alive = true;
+    if (pq.layer >= 0) {
+        alive = (MODE == P_MODE_IDENTITY) || s_seen[0] || p_wait(a, a.readyN + pq.layer, &s_flag);
+        if (alive) p_part_quant<RNG16, MODE>(a, pq, q, s_unit, &s_flag);
     }
-    if (it.ln >= 0) p_norm_publish(a, it.ln, it.tn, nt, s_unit, s_norm, &s_flag);
-    if (it.lq >= 0) {
-        const bool ok = (MODE == P_MODE_IDENTITY) || p_wait(a, a.readyN + it.lq, &s_flag);
-        if (ok) p_part_quant<RNG16, MODE>(a, it.lq, it.tq, qt, s_unit, &s_flag);
-        else p_cp_wait<0>();
+    if (alive && pu.layer >= 0) {
+        alive = s_seen[1] || p_wait(a, a.readyQ + pu.layer, &s_flag);
+        if (alive) p_part_update(a, pu, q);
     }
-    if (it.lu >= 0) {
-        if (p_wait(a, a.readyQ + it.lu, &s_flag)) p_part_update(a, it.lu, it.tu);
-    }
+    p_cp_wait<0>();
 }
 
 // ---- host: the item list -----------------------------------------------------------------------------
@@ -623,7 +619,12 @@ int dat_pipe_build(dat_plan_t *plan)
         });
         // slot of every tile in each of the three streams
         std::vector<PipeItem> items;
-        const PipeItem none = {-1, 0, -1, 0, -1, 0, 0, 0};
+        const PipePart nopart = {0, 1, 0, 1, -1, 0};
+        const PipeItem none = {nopart, nopart, nopart};
+        auto part = [&](int l, int64_t t) {
+            PipePart pp = {plan->offsets[l], plan->offsets[l + 1], (int32_t)tb[l], (int32_t)(tb[l + 1] - tb[l]), l, (int32_t)t};
+            return pp;
+        };
         auto at = [&](int64_t slot) -> PipeItem & {
             if ((int64_t)items.size() <= slot) items.resize((size_t)slot + 1, none);
             return items[(size_t)slot];
@@ -633,7 +634,7 @@ int dat_pipe_build(dat_plan_t *plan)
         if (!identity)
             for (int k = 0; k < h; ++k) {
                 const int l = order[k];
-                for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { PipeItem &it = at(slot); it.ln = l; it.tn = (int32_t)t; done_n[l] = slot++; }
+                for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { at(slot).n = part(l, t); done_n[l] = slot++; }
             }
         slot = 0;
         for (int k = 0; k < h; ++k) {
@@ -643,13 +644,13 @@ int dat_pipe_build(dat_plan_t *plan)
             // a layer that L2 cannot hold next to what streams in meanwhile is walked back from its last
             // tile (what N read last is read first); the others in N's order, every tile at the same distance
             const bool reverse = T >= DAT_P_REVERSE_FROM;
-            for (int64_t t = 0; t < T; ++t) { PipeItem &it = at(slot); it.lq = l; it.tq = (int32_t)(reverse ? T - 1 - t : t); done_q[l] = slot++; }
+            for (int64_t t = 0; t < T; ++t) { at(slot).q = part(l, reverse ? T - 1 - t : t); done_q[l] = slot++; }
         }
         slot = 0;
         for (int k = 0; k < h; ++k) {
             const int l = order[k];
             slot = std::max(slot, done_q[l] + DAT_P_LAG + 1);
-            for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { PipeItem &it = at(slot); it.lu = l; it.tu = (int32_t)t; ++slot; }
+            for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { at(slot).u = part(l, t); ++slot; }
         }
         g->n_items = (int64_t)items.size();
 
