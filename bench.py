@@ -307,8 +307,8 @@ def run_gpu(args):
                 api.dat_lalr_step(plan, theta, mom, u_ghat, hp)
         elif args.path == "passes":
             api.dat_step_passes(plan, theta, mom, grads, cfg.seed, step_index, hp)
-        elif args.path == "fused":
-            api.dat_step_sweep(plan, theta, mom, grads, cfg.seed, step_index, hp)
+        elif args.path == "pipelined":
+            api.dat_step_pipelined(plan, theta, mom, grads, cfg.seed, step_index, hp)
         else:
             api.dat_step(plan, theta, mom, grads, cfg.seed, step_index, hp)
 
@@ -325,13 +325,6 @@ def run_gpu(args):
     # ---- timed region: exactly K steps, per-step CUDA events on the launching stream
     K = args.steps
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K)]
-    # where the step is the three passes: events around its largest kernel, recorded by the library itself
-    probe = None
-    if args.path in ("step", "passes") and cfg.bits != 32 and (args.path == "passes" or cfg.d >= (1 << 20)):
-        probe = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K)]
-        for e in probe:
-            e.record(stream)                 # creates the event
-        torch.cuda.synchronize()
     sampler = ClockSampler(local)
     launches0 = api.dat_plan_launch_count(plan)
     barrier()
@@ -340,8 +333,6 @@ def run_gpu(args):
     for k in range(K):
         if flush is not None:
             flush.fill_(1.0)
-        if probe is not None:
-            api.dat_plan_set_probe(plan, probe[2 * k], probe[2 * k + 1])
         ev[2 * k].record(stream)
         one_step(step_no)
         ev[2 * k + 1].record(stream)
@@ -352,10 +343,6 @@ def run_gpu(args):
     clocks = sampler.stop()
     launches = api.dat_plan_launch_count(plan) - launches0
     step_ms = np.array([ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(K)])
-    probe_ms = None
-    if probe is not None:
-        api.dat_plan_set_probe(plan, None, None)
-        probe_ms = float(np.mean([probe[2 * k].elapsed_time(probe[2 * k + 1]) for k in range(K)]))
     region_ms = ev[0].elapsed_time(ev[2 * K - 1]) if flush is None else float(step_ms.sum())
     status = api.dat_get_status(plan)
     finite = bool(torch.isfinite(theta).all().item() and torch.isfinite(mom).all().item())
@@ -416,19 +403,12 @@ def run_gpu(args):
         else:
             algo_bytes = (4 * cfg.M + 16) * cfg.d
         achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
-        multi = (launches // K) > 1            # several kernels per step: the whole step is what is timed
-        traffic = None if multi else NCU_DRAM_BYTES_PER_LAUNCH.get("%s_b%d_rng%d" % (cfg.name, cfg.bits, cfg.rng_bits))
-        kernel_name = ("%s: %d kernels per step (whole step timed)" % (args.path, launches // K) if multi
-                       else "k_fused_step (one launch per step)")
-        whole_step = {"algorithmic_bytes": algo_bytes, "achieved": achieved, "frac": achieved / peak, "unit": "GB/s"}
-        roof_bytes, roof_achieved = algo_bytes, achieved
-        if probe_ms is not None:
-            # the dominant kernel of the step: reads the M gradient tiles, theta and m once, writes m'
-            roof_bytes = (4 * cfg.M + 12) * cfg.d
-            roof_achieved = roof_bytes / (probe_ms * 1e-3) / 1e9
-            kernel_name = ("k_quant_update, the largest of the %d kernels of a step (%.1f of %.1f us, CUDA events recorded "
-                           "around it by the library)" % (launches // K, 1e3 * probe_ms, 1e3 * kernel_ms))
-            traffic = NCU_DRAM_BYTES_PER_LAUNCH.get("k_quant_update_%s_b%d_rng%d" % (cfg.name, cfg.bits, cfg.rng_bits))
+        per_step = launches // K
+        traffic, traffic_src = ncu_traffic(args.path, cfg)
+        kernel_name = {"step": "dat_step (k_step_pipelined)", "pipelined": "dat_step_pipelined (k_step_pipelined)",
+                       "passes": "dat_step_passes"}.get(args.path, args.path)
+        kernel_name += ": %d launch%s per step, the whole step timed" % (per_step, "" if per_step == 1 else "es")
+        sm_mhz = clocks.get("sm_mhz") or 0
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": region_ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -437,10 +417,10 @@ def run_gpu(args):
             "step_latency_us": {"median": 1e3 * float(np.median(step_ms)), "min": 1e3 * float(step_ms.min()),
                                 "mean": 1e3 * kernel_ms},
             "pct_of_8TBps": 100.0 * achieved / NOMINAL_HBM_GBS,
-            "roofline": {"bound": "hbm", "achieved": roof_achieved, "peak": peak, "unit": "GB/s", "frac": roof_achieved / peak,
-                         "traffic": traffic, "algorithmic_bytes_per_launch": roof_bytes,
-                         "kernel": kernel_name, "peak_source": peak_src},
-            "whole_step": whole_step,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "traffic_source": traffic_src, "algorithmic_bytes_per_launch": algo_bytes // max(per_step, 1),
+                         "algorithmic_bytes_per_step": algo_bytes, "kernel": kernel_name, "peak_source": peak_src,
+                         "sm_cycles_per_step": (1e3 * kernel_ms) * sm_mhz if sm_mhz else None},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "status_word": int(status), "outputs_finite": finite, "wall_s_timed_region": t_wall,
         }
@@ -462,9 +442,9 @@ def main():
                     help="override the resolution of the quantizer's uniform number (0: the config's)")
     ap.add_argument("--impl", default="dat", choices=["dat", "reference"])
     ap.add_argument("--path", default="step",
-                    choices=["step", "fused", "passes", "unfused", "unfused_per_worker", "unfused_two_sided", "unfused_lamb"],
-                    help="step: dat_step (the headline; the three passes at this size); fused: dat_step_sweep, the "
-                         "single persistent kernel; passes: dat_step_passes; unfused: dat_quantize + dat_aggregate + dat_lalr_step; "
+                    choices=["step", "pipelined", "passes", "unfused", "unfused_per_worker", "unfused_two_sided", "unfused_lamb"],
+                    help="step: dat_step (the headline: one pipelined launch); pipelined: the same by its own name; "
+                         "passes: dat_step_passes, three streaming passes; unfused: dat_quantize + dat_aggregate + dat_lalr_step; "
                          "unfused_per_worker: the same with one quantizer norm per worker; unfused_two_sided: with "
                          "dat_requantize after the aggregation; unfused_lamb: with dat_lamb_step as the update")
     ap.add_argument("--e2e-steps", type=int, default=5)

@@ -19,7 +19,7 @@
  *   - The caller owns every data buffer.  The library never allocates, frees or retains them;
  *     after a call returns, only work already enqueued on `stream` refers to them.
  *     A plan owns only its own small device workspace (layout tables, partial sums,
- *     dependency counters, a status word) and, if dat_step_host is used, staging buffers.
+ *     arrival counters, a status word) and, if dat_step_host is used, staging buffers.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All device work
  *     is enqueued on it and is stream-ordered; calls return without synchronising unless
  *     stated otherwise.
@@ -79,8 +79,8 @@ typedef struct dat_lamb_hparams {
  * PER_WORKER: nu_{i,l} = ||g_l^(i)||_2, every worker's own norm, as Eq. rand_q and Eq. grad_agg
  *             are written: g_hat = (1/M) sum_i nu_{i,l} * sign * level / S, summed in fp32.  The
  *             message then carries M*h norms (index i*h + l), and no integer code sum exists.
- *             Available in the separate calls (dat_quantize, dat_aggregate); the fused dat_step
- *             sums integer codes and answers DAT_ERR_UNSUPPORTED for such a plan.              */
+ *             Available in the separate calls (dat_quantize, dat_aggregate); dat_step sums
+ *             integer codes and answers DAT_ERR_UNSUPPORTED for such a plan.                   */
 enum { DAT_SCALE_SHARED_MAX = 0, DAT_SCALE_PER_WORKER = 1 };
 
 /* Resolution of the quantizer's uniform number (see dat_plan_create). */
@@ -101,8 +101,8 @@ enum {
 /* Bits of the device status word. */
 enum {
     DAT_STATUS_NONFINITE = 1u, /* a quantizer norm or a layer norm was inf or NaN              */
-    DAT_STATUS_TIMEOUT = 2u,   /* a bounded device-side wait ran out; outputs of that call are
-                                  undefined, the plan stays usable                              */
+    DAT_STATUS_TIMEOUT = 2u,   /* a bounded device-side wait ran out; outputs are undefined until
+                                  dat_get_status has been called (which restores the plan)      */
     DAT_STATUS_BOUNDS = 4u     /* reserved for self-checking builds                             */
 };
 
@@ -149,8 +149,9 @@ int dat_plan_sizes(const dat_plan_t *plan, int64_t *level_bytes_per_worker,
  * dat_quantize -- Algorithm A1 Step 7: Q(g^(i)) for every worker (Eq. rand_q, Eq. xi).
  *   For worker i, layer l, element e (global index in the flat vector), with x = S*|g_e|/nu_l:
  *   level = floor(x) + 1 with probability x - floor(x), else floor(x); sign bit = (g_e < 0).
- *   Randomness: Philox4x32-10, counter (lo(e/4), hi(e/4), i, hi(seed)), key (lo(seed), step),
- *   word e mod 4; u1 = 1 + (low 23 bits)/2^23; level = min(floor(fma(|g_e|, S/nu_l, u1)) - 1, S).
+ *   Randomness: Philox4x32-10 keyed on (seed, step, worker i, element e); u1 = 1 + u with u the
+ *   plan's 23-bit or 16-bit uniform number (see rng_bits of dat_plan_create);
+ *   level = min(floor(fma(|g_e|, S/nu_l, u1)) - 1, S).
  *
  *   grads      host array of M device pointers, each fp32[d], read-only.
  *   seed,step  random-stream key; step must be < 2^32 (DAT_ERR_ARG).
@@ -255,13 +256,15 @@ int dat_lamb_step(dat_plan_t *plan, float *theta, float *mom, float *var, const 
  *   layer_norms_out device fp32[2h] or NULL, as in dat_lalr_step.
  * The result is bit-identical to dat_lalr_step on the same inputs.
  * First call on a device: it looks up the device address of the scratch array (once per device,
- * with that device current); make this first call outside any stream capture.  The call is
- * not thread-safe with respect to other first calls on the same device.
+ * with that device current).  The call copies its layer table from host memory on every call, so it
+ * cannot be recorded into a CUDA graph: while `stream` is capturing it answers DAT_ERR_UNSUPPORTED
+ * and enqueues nothing.  The call is not thread-safe with respect to other first calls on the same
+ * device, and the looked-up address does not survive a cudaDeviceReset of that device.
  * All calls on a device share the one scratch array, which keeps the previous call's contents;
  * the call clears what has to start at zero.  Two calls whose device work overlaps (different
  * streams, or different host threads) race on it: serialise them.  Non-finite norms are not
  * reported (there is no plan whose status word could carry the bit).
- * Errors: ARG, ALIGN, LAYOUT, TOO_LARGE, UNSUPPORTED (device ordinal >= 64), CUDA.
+ * Errors: ARG, ALIGN, LAYOUT, TOO_LARGE, UNSUPPORTED (device ordinal >= 64, or `stream` is capturing), CUDA.
  * ------------------------------------------------------------------------------------------- */
 #define DAT_STATIC_MAX_LAYERS 4096
 #define DAT_STATIC_MAX_TILES 32768
@@ -271,9 +274,9 @@ int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_offsets, float
 /* ---------------------------------------------------------------------------------------------
  * dat_step -- Steps 7, 9 and 12 of Algorithm A1 in one call: the result equals
  * dat_quantize -> dat_aggregate -> dat_lalr_step (or dat_average -> dat_lalr_step when b = 32),
- * but codes, code sums and g_hat are never written to device memory.  Inside, either one
- * persistent kernel that sweeps the vectors once (dat_step_sweep) or three streaming passes
- * (dat_step_passes), whichever is faster for the plan's size; both are also exported.
+ * but codes, code sums and g_hat are never written to device memory.  One kernel launch
+ * (dat_step_pipelined); nothing is allocated and nothing synchronises: every table the launch
+ * needs was built by dat_plan_create.
  *   theta, mom        device fp32[d], updated in place.
  *   grads             host array of M device pointers, fp32[d] each, read-only.
  *   seed, step        as in dat_quantize.
@@ -281,40 +284,43 @@ int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_offsets, float
  *   code_sum_out      device int32[d] or NULL (checking aid; ignored when b = 32).
  *   layer_norms_out   device fp32[2h] or NULL.
  *   scales_out        device fp32[h] or NULL: nu_l (not written when b = 32).
- * Errors: ARG, ALIGN, CUDA.
+ * Inside the launch a work item may have to wait for a layer's norm that another item is still
+ * producing; that wait is bounded (about two seconds).  If it ever runs out, the call returns as
+ * usual, DAT_STATUS_TIMEOUT is set in the status word, and the outputs of that call -- and of
+ * later calls on the plan -- are undefined until dat_get_status has been called, which reports the
+ * bit and restores the plan's counters.
+ * Errors: ARG, ALIGN, UNSUPPORTED (a plan with DAT_SCALE_PER_WORKER and b < 32), CUDA.
  * ------------------------------------------------------------------------------------------- */
 int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
              uint64_t seed, uint64_t step, const dat_hparams_t *hp,
              int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream);
 
-/* dat_step_sweep -- dat_step by the single persistent kernel, whatever the size (dat_step itself
- * takes the three passes of dat_step_passes from 2^20 elements on, where they are faster, and this
- * kernel below that).  Same arguments, results and errors as dat_step. */
-int dat_step_sweep(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
-                   uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
-                   float *layer_norms_out, float *scales_out, void *stream);
-
-/* dat_step_passes -- the same step as dat_step, with the same arguments and the same results bit for
- * bit up to the norms' last place, computed by three streaming passes in separate launches instead of
- * one persistent kernel: quantizer norms; then levels, signed sum over the workers, g_hat, m' and the
- * layer sums in one pass that keeps codes, sums and g_hat in registers; then the theta update.  The
- * gradients are read twice by construction.  For plans with b < 32 and the shared scale
- * (DAT_ERR_UNSUPPORTED otherwise).  Its first call on a plan allocates two small tables (synchronous). */
-int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
-                    uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
-                    float *layer_norms_out, float *scales_out, void *stream);
-
-/* dat_step_pipelined -- the same step as dat_step in one launch that reads every gradient from device
- * memory once.  Same arguments, results and errors as dat_step. */
+/* dat_step_pipelined -- what dat_step calls: the step as ONE launch of ordinary thread blocks.  The
+ * vector is cut into per-layer tiles; a work item holds one tile for each of three phases -- sums of
+ * squares for the quantizer norms (N), levels + signed sum + g_hat + m' + layer sums (Q), parameter
+ * update (U) -- with the Q tiles running a fixed distance behind the N tiles and the U tiles behind the
+ * Q tiles, so that a gradient read for its norm is still in the L2 cache when its level is drawn.
+ * Same arguments, results and errors as dat_step. */
 int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
                        uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
                        float *layer_norms_out, float *scales_out, void *stream);
 
-/* dat_plan_set_probe -- measurement aid: two CUDA events owned by the caller (cudaEvent_t passed as
- * void*; NULL, NULL switches it off) that later calls of dat_step_passes (and of dat_step where it
- * takes that path) record on their stream just before and just after k_quant_update, the largest
- * kernel of the step.  The events must outlive those calls.  Errors: ARG. */
-int dat_plan_set_probe(dat_plan_t *plan, void *event_before, void *event_after);
+/* dat_step_passes -- the same step as dat_step, with the same arguments and the same results bit for
+ * bit up to the norms' last place, computed by three streaming passes in separate launches: quantizer
+ * norms; then levels, signed sum over the workers, g_hat, m' and the layer sums in one pass that keeps
+ * codes, sums and g_hat in registers; then the theta update.  The gradients are read twice by
+ * construction.  For plans with b < 32 and the shared scale (DAT_ERR_UNSUPPORTED otherwise).  Its first
+ * call on a plan allocates two small tables (synchronous: not for use under stream capture). */
+int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                    uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
+                    float *layer_norms_out, float *scales_out, void *stream);
+
+/* dat_plan_test_stall -- TEST HOOK for the bounded wait of dat_step: sets the plan's wait limit to
+ * `wait_cycles` SM clock cycles (0 restores the default) and, if `layer` >= 0, marks that layer's norm
+ * as never completing for the next call (its tile counter is pre-set on the host side of the stream so
+ * that the count cannot be reached): work items that need the layer give up after the limit and the
+ * call ends with DAT_STATUS_TIMEOUT.  Nothing else uses this.  Errors: ARG, CUDA. */
+int dat_plan_test_stall(dat_plan_t *plan, int64_t wait_cycles, int64_t layer, void *stream);
 
 /* dat_step_host -- dat_step for callers whose data lives in HOST memory: copies theta, mom and
  * the M gradient buffers to plan-owned device staging buffers, runs dat_step, copies theta and
@@ -327,7 +333,8 @@ int dat_step_host(dat_plan_t *plan, float *theta_host, float *mom_host,
                   const float *const *grads_host, uint64_t seed, uint64_t step,
                   const dat_hparams_t *hp, void *stream);
 
-/* Synchronises `stream`, copies the plan's status word to *flags_out and clears it. */
+/* Synchronises `stream`, copies the plan's status word to *flags_out and clears it.  If the word carries
+ * DAT_STATUS_TIMEOUT, the counters that the interrupted call left mid-way are cleared as well. */
 int dat_get_status(dat_plan_t *plan, uint32_t *flags_out, void *stream);
 
 /* Number of kernels the library has launched for this plan since it was created. */

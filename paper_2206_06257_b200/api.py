@@ -31,7 +31,7 @@ DAT_STATUS_NONFINITE, DAT_STATUS_TIMEOUT, DAT_STATUS_BOUNDS = 1, 2, 4
 
 # every symbol include/dat.h declares
 EXPORTS = ["dat_plan_create", "dat_plan_destroy", "dat_plan_sizes", "dat_quantize", "dat_aggregate", "dat_requantize",
-           "dat_average", "dat_lalr_step", "dat_lamb_step", "dat_lalr_step_static", "dat_step", "dat_step_sweep", "dat_step_passes", "dat_step_pipelined", "dat_plan_set_probe", "dat_step_host", "dat_get_status",
+           "dat_average", "dat_lalr_step", "dat_lamb_step", "dat_lalr_step_static", "dat_step", "dat_step_passes", "dat_step_pipelined", "dat_plan_test_stall", "dat_step_host", "dat_get_status",
            "dat_plan_launch_count", "dat_strerror", "dat_last_cuda_error"]
 
 
@@ -57,8 +57,7 @@ _lib.dat_lalr_step.argtypes = [_p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
 _lib.dat_lamb_step.argtypes = [_p, _p, _p, _p, _p, C.POINTER(dat_lamb_hparams_t), _i64, _p, _p]
 _lib.dat_lalr_step_static.argtypes = [_i64, _p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
 _lib.dat_step.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
-_lib.dat_plan_set_probe.argtypes = [_p, _p, _p]
-_lib.dat_step_sweep.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
+_lib.dat_plan_test_stall.argtypes = [_p, _i64, _i64, _p]
 _lib.dat_step_pipelined.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_step_passes.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_step_host.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p]
@@ -188,20 +187,9 @@ def dat_step(plan, theta, mom, grads, seed, step, hp, code_sum_out=None, layer_n
                       _ptr(code_sum_out), _ptr(layer_norms_out), _ptr(scales_out), _stream(stream)), "dat_step")
 
 
-def dat_plan_set_probe(plan, event_before, event_after):
-    """event_*: torch.cuda.Event (already recorded once, so that it exists), a raw handle, or None."""
-    def handle(e):
-        if e is None:
-            return None
-        return _p(e.cuda_event if isinstance(e, torch.cuda.Event) else int(e))
-    _ok(_lib.dat_plan_set_probe(_p(plan), handle(event_before), handle(event_after)), "dat_plan_set_probe")
-
-
-def dat_step_sweep(plan, theta, mom, grads, seed, step, hp, code_sum_out=None, layer_norms_out=None,
-                   scales_out=None, stream=None):
-    h = _hp(hp)
-    _ok(_lib.dat_step_sweep(_p(plan), _ptr(theta), _ptr(mom), _ptr_array(grads), int(seed), int(step), C.byref(h),
-                            _ptr(code_sum_out), _ptr(layer_norms_out), _ptr(scales_out), _stream(stream)), "dat_step_sweep")
+def dat_plan_test_stall(plan, wait_cycles, layer=-1, stream=None):
+    """Test hook: wait limit in SM cycles (0: default) and a layer whose norm never completes next call."""
+    _ok(_lib.dat_plan_test_stall(_p(plan), int(wait_cycles), int(layer), _stream(stream)), "dat_plan_test_stall")
 
 
 def dat_step_passes(plan, theta, mom, grads, seed, step, hp, code_sum_out=None, layer_norms_out=None,

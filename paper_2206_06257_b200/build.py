@@ -12,7 +12,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 DEBUG = os.environ.get("DAT_DEBUG") == "1"        # the self-checking build: libdat_debug.so, with -DDAT_SELFCHECK
 LIB = os.path.join(HERE, "libdat_debug.so" if DEBUG else "libdat.so")
-SOURCES = ["dat_plan.cu", "dat_unfused.cu", "dat_step.cu", "dat_pipeline.cu"]
+SOURCES = ["dat_plan.cu", "dat_unfused.cu", "dat_pipeline.cu"]
 HEADERS = [os.path.join(CSRC, "dat_internal.cuh"), os.path.join(ROOT, "include", "dat.h")]
 
 NVCC_FLAGS = [

@@ -24,7 +24,6 @@ struct PhiloxKeys {
     uint32_t seed_hi;   // fourth counter word
 };
 
-struct FusedSchedule;   // dat_step.cu
 struct PipeSchedule;    // dat_pipeline.cu
 
 struct dat_plan {
@@ -51,16 +50,12 @@ struct dat_plan {
     float *d_norms = nullptr;          // 2h
     uint32_t *d_status = nullptr;      // 1
 
-    FusedSchedule *fused = nullptr;    // built lazily by dat_step_sweep
     PipeSchedule *pipe = nullptr;      // work items and tables of dat_step_pipelined, built with the plan
 
     // dat_step_passes: per-layer tiles that start on multiples of 8 elements, and their partial sums
     int64_t *d_tile_base8 = nullptr;   // h+1
     double *d_partials8 = nullptr;     // 2 per tile
     int64_t n_tiles8 = 0;
-
-    // dat_plan_set_probe: events recorded around the second pass of dat_step_passes (measurement aid)
-    void *probe_before = nullptr, *probe_after = nullptr;
 
     // staging buffers of dat_step_host
     float *stage = nullptr;
@@ -76,7 +71,6 @@ int dat_cuda_fail(dat_plan_t *plan, cudaError_t e);          // records e, retur
 bool dat_aligned16(const void *p);
 int dat_check_grads(const dat_plan_t *plan, const float *const *grads, GradPtrs *out);
 PhiloxKeys dat_make_keys(uint64_t seed, uint64_t step);
-void dat_fused_destroy(dat_plan_t *plan);                    // dat_step.cu
 int dat_pipe_build(dat_plan_t *plan);                        // dat_pipeline.cu (device current)
 void dat_pipe_destroy(dat_plan_t *plan);
 cudaError_t dat_pipe_reset(dat_plan_t *plan, cudaStream_t s);

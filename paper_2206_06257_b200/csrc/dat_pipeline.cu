@@ -21,19 +21,21 @@
 
 #include "dat_internal.cuh"
 
+#ifndef DAT_P_THREADS
 #define DAT_P_THREADS 256
-#define DAT_P_TILE 2048                           // elements per tile (eight per thread), tiles start on multiples of 8
+#endif
+#ifndef DAT_P_GROUPS                              // groups of eight consecutive elements per thread and tile
+#define DAT_P_GROUPS 2
+#endif
+#define DAT_P_TILE (DAT_P_THREADS * 8 * DAT_P_GROUPS)   // elements per tile, tiles start on multiples of 8
 #ifndef DAT_P_MINB
-#define DAT_P_MINB 4
+#define DAT_P_MINB (1024 / DAT_P_THREADS)         // 64 registers per thread
 #endif
 #ifndef DAT_P_LAG                                 // items between the last N tile of a layer and its first Q tile
-#define DAT_P_LAG 384
+#define DAT_P_LAG 256
 #endif
 #ifndef DAT_P_REVERSE_FROM                        // layers of at least this many tiles: Q walks back from the last tile
-#define DAT_P_REVERSE_FROM 640
-#endif
-#ifndef DAT_P_N_POLICY                            // L2 priority of the gradients when they are first read
-#define DAT_P_N_POLICY dat_policy_evict_last
+#define DAT_P_REVERSE_FROM 320
 #endif
 #define DAT_P_WAIT_CYCLES (4000000000ll)          // about two seconds
 
@@ -105,158 +107,95 @@ __device__ __forceinline__ void p_load4_cg(const float *__restrict__ p, int64_t 
     }
 }
 
-// Arrival of one tile of a layer: true (in every thread) in the CTA that arrives last.  Every
-// thread has fenced what it wrote for the layer.
-__device__ __forceinline__ bool p_arrive(uint32_t *cnt, uint32_t total, int *s_flag)
+// One thread: waits until `word` carries this call's epoch.  Bounded: when the limit runs out the status
+// word gets DAT_STATUS_TIMEOUT and the call's abort word is set, which ends every other wait at once.
+// Returns false if the part that needs the word must be skipped.
+__device__ __forceinline__ bool p_poll(const PArgs &a, const uint32_t *word)
 {
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        *s_flag = (atomicAdd(cnt, 1u) == total - 1u);
-    }
-    __syncthreads();
-    const bool last = (*s_flag != 0);
-    __syncthreads();
-    if (last) __threadfence();
-    return last;
-}
-
-// Waits until `word` carries this call's epoch.  Bounded: when the limit runs out the status word
-// gets DAT_STATUS_TIMEOUT and the call's abort word is set, which ends every other wait at once.
-// Returns false (in every thread) if the part must be skipped.
-__device__ __forceinline__ bool p_wait(const PArgs &a, const uint32_t *word, int *s_flag)
-{
-    if (threadIdx.x == 0) {
-        bool ok = (p_ld_acquire(word) == a.epoch);
-        if (!ok) {
-            const long long t0 = clock64();
-            for (;;) {
-                __nanosleep(128);
-                if (p_ld_acquire(word) == a.epoch) { ok = true; break; }
-                if (p_ld_acquire(a.abort_epoch) == a.epoch) break;
-                if (clock64() - t0 > a.wait_cycles) {
-                    atomicOr(a.status, DAT_STATUS_TIMEOUT);
-                    p_st_release(a.abort_epoch, a.epoch);
-                    break;
-                }
-            }
+    if (p_ld_acquire(word) == a.epoch) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        __nanosleep(128);
+        if (p_ld_acquire(word) == a.epoch) return true;
+        if (p_ld_acquire(a.abort_epoch) == a.epoch) return false;
+        if (clock64() - t0 > a.wait_cycles) {
+            atomicOr(a.status, DAT_STATUS_TIMEOUT);
+            p_st_release(a.abort_epoch, a.epoch);
+            return false;
         }
-        *s_flag = ok ? 1 : 0;
     }
-    __syncthreads();
-    const bool ok = (*s_flag != 0);
-    __syncthreads();
-    return ok;
 }
 
-// ---- staging through shared memory ---------------------------------------------------------------
-// Every thread streams its own sequence of 32-byte entries (two 16-byte slots) through a private
-// ring in shared memory: the parts of the N tile it sums, then for its eight elements of the Q tile
-// one entry per worker, theta and m, then theta and m' of its eight elements of the U tile.  Entry j
-// sits in ring position j mod DAT_P_DEPTH; it is fetched by two asynchronous 16-byte copies DEPTH
-// entries ahead of its use, across the borders of the three parts, and read back by the thread that
-// fetched it -- so the copies need no barrier, only the thread's own wait for its copy groups, and
-// what is in flight costs no registers.  Slot k of thread t is p_stage[k * 256 + t].
-extern __shared__ float4 p_stage[];
-#ifndef DAT_P_DEPTH
-#define DAT_P_DEPTH 6
-#endif
-#define DAT_P_STAGE_BYTES (2 * DAT_P_DEPTH * DAT_P_THREADS * 16)
-
-// Self-checking build (-DDAT_SELFCHECK): every address formed from an item is checked before it is used;
-// a violation sets DAT_STATUS_BOUNDS and the access is skipped, nothing faults.
+// Self-checking build (-DDAT_SELFCHECK): what an item says about its tiles is checked before it is used;
+// a violation sets DAT_STATUS_BOUNDS and the item is skipped, nothing faults.
 #ifdef DAT_SELFCHECK
 #define P_CHECK(a, cond) ((cond) ? true : (atomicOr((a).status, DAT_STATUS_BOUNDS), false))
 #else
 #define P_CHECK(a, cond) true
 #endif
 
-__device__ __forceinline__ void p_cp16(const PArgs &a, float4 *dst, const float *base, int64_t e, uint64_t pol)
+__device__ __forceinline__ int64_t p_tile_begin(const PipePart &pt)
 {
-    const float *src = base + e;
-#ifdef DAT_SELFCHECK
-    const int64_t slot_off = (const char *)dst - (const char *)p_stage;
-    if (!P_CHECK(a, e >= 0 && e + 4 <= a.d && ((uintptr_t)src & 15u) == 0 && slot_off >= 0 &&
-                    slot_off + 16 <= DAT_P_STAGE_BYTES && (slot_off & 15) == 0)) return;
-#endif
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
-    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" :: "r"(d), "l"(src), "l"(pol) : "memory");
+    return (pt.lo & ~(int64_t)7) + (int64_t)pt.tile * DAT_P_TILE;
 }
-__device__ __forceinline__ void p_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void p_cp_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
-
-// What a thread needs to know to fetch entry j of its sequence.
-struct Seq {
-    int nN, nQ, nU;                                // entries of the three parts (0: that part reads global memory itself)
-    int u0;                                        // N: first unit of this warp
-    int64_t eN, eQ, eU;                            // N: tile begin + 4 lane; Q, U: the thread's first element
-    uint64_t pol_last, pol_first, pol_normal;
-};
-
-__device__ __forceinline__ void p_issue(const PArgs &a, const Seq &q, int j)
+__device__ __forceinline__ bool p_tile_inside(const PipePart &pt)
 {
-    float4 *dst = p_stage + (2 * (j % DAT_P_DEPTH)) * DAT_P_THREADS + threadIdx.x;
-    if (j < q.nN) {
-        // unit u = u0 + j/2 (worker u/4, quarter u%4), its copies 2(j%2) and 2(j%2)+1 of four
-        const int u = q.u0 + (j >> 1);
-        const int64_t e = q.eN + (u & 3) * (DAT_P_TILE / 4) + 256 * (j & 1);
-        p_cp16(a, dst, a.gp.p[u >> 2], e, q.pol_last);
-        p_cp16(a, dst + DAT_P_THREADS, a.gp.p[u >> 2], e + 128, q.pol_last);
-    } else if (j < q.nN + q.nQ) {
-        const int i = j - q.nN;
-        const float *base = (i < a.M) ? a.gp.p[i] : (i == a.M ? a.theta : a.mom);
-        const uint64_t pol = (i < a.M) ? q.pol_first : q.pol_normal;     // a gradient is dead once its level is drawn
-        p_cp16(a, dst, base, q.eQ, pol);
-        p_cp16(a, dst + DAT_P_THREADS, base, q.eQ + 4, pol);
-    } else if (j < q.nN + q.nQ + q.nU) {
-        const float *base = (j == q.nN + q.nQ) ? a.theta : a.mom;
-        p_cp16(a, dst, base, q.eU, q.pol_first);
-        p_cp16(a, dst + DAT_P_THREADS, base, q.eU + 4, q.pol_first);
-    }
-    p_cp_commit();                                 // one group per entry, also past the end: the count stays uniform
-}
-
-// Entry j has arrived (every entry up to j + DEPTH - 1 has been issued): its eight floats.
-__device__ __forceinline__ void p_take(int j, float v[8])
-{
-    p_cp_wait<DAT_P_DEPTH - 1>();
-    const float4 *src = p_stage + (2 * (j % DAT_P_DEPTH)) * DAT_P_THREADS + threadIdx.x;
-    const float4 a0 = src[0], a1 = src[DAT_P_THREADS];
-    v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+    const int64_t begin = p_tile_begin(pt);
+    return begin >= pt.lo && begin + DAT_P_TILE <= pt.hi;
 }
 
 // ---- N: sums of squares of one tile, every worker ------------------------------------------------
-// A tile is cut into 4M units (worker, quarter tile of 512 elements); warp w takes the units
-// [w*4M/8, (w+1)*4M/8), a unit being two entries per lane.  Units of the same worker are summed per
-// lane before the warp reduction; the structure depends on M only, so the sums are the same from
-// run to run.
-__device__ __forceinline__ void p_norm_sums(const PArgs &a, const PipePart &pt, const Seq &q, double *s_unit)
+// A tile is cut into 4M units (worker, quarter tile); warp w of W takes the units [w*4M/W, (w+1)*4M/W),
+// lane j the 16-byte pieces j, j+32, ... of a unit, eight pieces in flight.  Units of the same worker
+// are summed per lane before the warp reduction; the structure depends on M only, so the sums are the
+// same from run to run.  Leaves one sum per run of units in s_unit (zero elsewhere).
+__device__ __forceinline__ void p_norm_sums(const PArgs &a, const PipePart &pt, double *s_unit)
 {
+    constexpr int W = DAT_P_THREADS / 32, QUARTER = DAT_P_TILE / 4, LPU = QUARTER / 128, UPB = 8 / LPU;   // units per batch of 8 loads
+    static_assert(LPU >= 1 && LPU <= 8 && UPB * LPU == 8, "quarter tiles of 128 .. 1024 elements");
     const int M = a.M;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int U = 4 * M;
-    const int u0 = warp * U / 8, u1 = (warp + 1) * U / 8;
+    const int u0 = warp * U / W, u1 = (warp + 1) * U / W;
+    const int64_t begin = p_tile_begin(pt);
     double acc = 0.0;
     int run = u0;
-    if (q.nN > 0) {
+    if (p_tile_inside(pt)) {
+        const uint64_t pol = dat_policy_evict_last();  // the Q part of a later item reads these lines again
 #pragma unroll 1
-        for (int j = 0; j < q.nN; ++j) {
-            const int u = u0 + (j >> 1);
-            if ((u >> 2) != (run >> 2)) {
-                acc = dat_warp_sum(acc);
-                if (lane == 0) s_unit[run] = acc;
-                acc = 0.0;
-                run = u;
-            }
-            float v[8];
-            p_take(j, v);
+        for (int ub = u0; ub < u1; ub += UPB) {
+            float4 v[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) acc = fma((double)v[k], (double)v[k], acc);
-            p_issue(a, q, j + DAT_P_DEPTH);        // into the slots just read
+            for (int k = 0; k < UPB; ++k) {
+                const int u = ub + k;
+                if (u < u1) {
+                    const float *g = a.gp.p[u >> 2] + begin + (u & 3) * QUARTER + 4 * lane;
+#pragma unroll
+                    for (int b = 0; b < LPU; ++b) v[k * LPU + b] = dat_ld4_hint(g + 128 * b, pol);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < UPB; ++k) {
+                const int u = ub + k;
+                if (u < u1) {
+                    if ((u >> 2) != (run >> 2)) {
+                        acc = dat_warp_sum(acc);
+                        if (lane == 0) s_unit[run] = acc;
+                        acc = 0.0;
+                        run = u;
+                    }
+#pragma unroll
+                    for (int b = 0; b < LPU; ++b) {
+                        const float4 x = v[k * LPU + b];
+                        acc = fma((double)x.x, (double)x.x, acc);
+                        acc = fma((double)x.y, (double)x.y, acc);
+                        acc = fma((double)x.z, (double)x.z, acc);
+                        acc = fma((double)x.w, (double)x.w, acc);
+                    }
+                }
+            }
         }
     } else {
-        const int64_t begin = (pt.lo & ~(int64_t)7) + (int64_t)pt.tile * DAT_P_TILE;
 #pragma unroll 1
         for (int u = u0; u < u1; ++u) {
             if ((u >> 2) != (run >> 2)) {
@@ -266,9 +205,9 @@ __device__ __forceinline__ void p_norm_sums(const PArgs &a, const PipePart &pt, 
                 run = u;
             }
             const float *__restrict__ g = a.gp.p[u >> 2];
-            const int64_t e = begin + (u & 3) * (DAT_P_TILE / 4) + 4 * lane;
+            const int64_t e = begin + (u & 3) * QUARTER + 4 * lane;
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
+            for (int b = 0; b < LPU; ++b) {
                 float t[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                 if (e + 128 * b < pt.hi) dat_load4(g, e + 128 * b, pt.lo, pt.hi, t);
 #pragma unroll
@@ -282,21 +221,34 @@ __device__ __forceinline__ void p_norm_sums(const PArgs &a, const PipePart &pt, 
     }
 }
 
-// Writes the tile's M partial sums, counts the tile in, and in the CTA that holds the layer's last
-// tile: nu_{i,l} = sqrt(sum over the tiles), nu_l = max_i, and the layer's two factors.
-__device__ __forceinline__ void p_norm_publish(const PArgs &a, const PipePart &pt, double *s_unit, float *s_norm, int *s_flag)
+// Warp 0, after the barrier that follows the N sums: writes the tile's M partial sums and counts the tile
+// in.  Returns (in lane 0) whether this was the layer's last tile.
+__device__ __forceinline__ bool p_norm_publish(const PArgs &a, const PipePart &pt, const double *s_unit)
+{
+    const int M = a.M, lane = threadIdx.x & 31;
+    for (int i = lane; i < M; i += 32) {
+        const double *s = s_unit + 4 * i;
+        a.partN[((int64_t)pt.tb + pt.tile) * M + i] = ((s[0] + s[1]) + s[2]) + s[3];
+    }
+    __threadfence();
+    __syncwarp();
+    bool last = false;
+    if (lane == 0) {
+        __threadfence();
+        last = (atomicAdd(a.cntN + pt.layer, 1u) == (uint32_t)pt.T - 1u);
+    }
+    return last;
+}
+
+// The CTA that counted in the layer's last N tile (every thread): nu_{i,l} = sqrt(sum over the tiles),
+// nu_l = max_i, and the layer's two factors, published with the call's epoch.
+__device__ __forceinline__ void p_norm_finish(const PArgs &a, const PipePart &pt, float *s_norm)
 {
     const int M = a.M, layer = pt.layer;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t tb = pt.tb;
     const uint32_t T = (uint32_t)pt.T;
-    __syncthreads();                               // every warp's unit sums are in s_unit
-    if (threadIdx.x < M) {
-        const double *s = s_unit + 4 * threadIdx.x;
-        a.partN[(tb + pt.tile) * M + threadIdx.x] = ((s[0] + s[1]) + s[2]) + s[3];
-        __threadfence();
-    }
-    if (!p_arrive(a.cntN + layer, T, s_flag)) return;
+    __threadfence();
     for (int i = warp; i < M; i += DAT_P_THREADS / 32) {
         double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
         uint32_t t = lane;
@@ -332,17 +284,28 @@ __device__ __forceinline__ void p_norm_publish(const PArgs &a, const PipePart &p
     }
 }
 
-// ---- the layer's step length from the partial sums of theta^2 and m'^2 (Eq. 3), by the last Q tile --
-__device__ __forceinline__ void p_finish_update_sums(const PArgs &a, int layer, int64_t tb, uint32_t T, double *scratch)
+// ---- the layer's step length from the partial sums of theta^2 and m'^2 (Eq. 3), by the CTA that counted
+// in the layer's last Q tile (every thread) ----------------------------------------------------------
+__device__ __forceinline__ void p_quant_finish(const PArgs &a, const PipePart &pt, double *scratch)
 {
+    const int layer = pt.layer;
+    const int64_t tb = pt.tb;
+    const uint32_t T = (uint32_t)pt.T;
+    __threadfence();
     double x = 0.0, y = 0.0;
     for (uint32_t t = threadIdx.x; t < T; t += DAT_P_THREADS) {
         x += __ldcg(a.partQ + 2 * (tb + t));
         y += __ldcg(a.partQ + 2 * (tb + t) + 1);
     }
-    x = dat_block_sum(x, scratch);
-    y = dat_block_sum(y, scratch);
+    x = dat_warp_sum(x);
+    y = dat_warp_sum(y);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) { scratch[2 * (threadIdx.x >> 5)] = x; scratch[2 * (threadIdx.x >> 5) + 1] = y; }
+    __syncthreads();
     if (threadIdx.x == 0) {
+        x = 0.0; y = 0.0;
+#pragma unroll
+        for (int w = 0; w < DAT_P_THREADS / 32; ++w) { x += scratch[2 * w]; y += scratch[2 * w + 1]; }
         const float n_theta = (float)sqrt(x), n_u = (float)sqrt(y);
         const float tau = fminf(fmaxf(n_theta, a.c_l), a.c_u);
         const float ratio = (n_u == 0.0f) ? 0.0f : tau / n_u;
@@ -355,37 +318,11 @@ __device__ __forceinline__ void p_finish_update_sums(const PArgs &a, int layer, 
     }
 }
 
-// One worker's eight elements: levels by the scaled form of Eq. xi, signed float sum (exact).
-template <bool RNG16>
-__device__ __forceinline__ void p_levels8(const float v[8], const uint32_t w[8], const QuConst &qc, float acc[8])
-{
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        float u1s;
-        if (RNG16) u1s = __fmaf_rn(__uint_as_float(__byte_perm(w[j >> 1], 0x4B000000u, (j & 1) ? 0x7632 : 0x7610)), qc.c0, qc.c1);
-        else u1s = __uint_as_float(qc.ubits | (w[j] & 0x007FFFFFu));
-        const float ys = __saturatef(__fmaf_rn(fabsf(v[j]), qc.ts, u1s));
-        const float lf = __fmaf_rz(ys, qc.two_b, 8388607.0f) - 8388608.0f;
-        const float sg = __uint_as_float((__float_as_uint(v[j]) & 0x80000000u) | 0x3F800000u);
-        acc[j] = __fmaf_rn(lf, sg, acc[j]);
-    }
-}
-
-template <bool RNG16>
-__device__ __forceinline__ void p_words8(const PArgs &a, int64_t e0, uint32_t worker, uint32_t w[8])
-{
-    if (RNG16) {
-        dat_random_words((uint64_t)e0 >> 3, worker, a.keys, w);
-    } else {
-        dat_random_words((uint64_t)e0 >> 2, worker, a.keys, w);
-        dat_random_words(((uint64_t)e0 >> 2) + 1, worker, a.keys, w + 4);
-    }
-}
-
 // ---- Q: levels (Eq. xi), signed sum over the workers and g_hat (Eq. grad_agg), m' and the layer sums
-// (Eq. 3, pass 1) of one tile; codes, sums and g_hat stay in registers ----------------------------
+// (Eq. 3, pass 1) of one tile; codes, sums and g_hat stay in registers.  Leaves the tile's two sums per
+// warp in scratch[2w], scratch[2w + 1]. -------------------------------------------------------------
 template <bool RNG16, int MODE>
-__device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt, const Seq &q, double *scratch, int *s_flag)
+__device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt, double *scratch)
 {
     const int M = a.M, layer = pt.layer;
     const int64_t lo = pt.lo, hi = pt.hi;
@@ -396,26 +333,15 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
     const bool plain = (t != 0.0f) && !(t >= 1.17549435e-38f * two_b && t <= 3.402823466e38f);
     const QuConst qc = {t, t * inv_two_b, two_b, inv_two_b * (1.0f / 65536.0f), -127.0f * inv_two_b, __float_as_uint(inv_two_b)};
     double ss_theta = 0.0, ss_u = 0.0;
-    const int64_t e0 = q.eQ;
-    const bool staged = q.nQ > 0;                  // the whole tile lies inside the layer and its rows were fetched ahead
-    if (e0 < hi) {
+    const int64_t begin = p_tile_begin(pt);
+#pragma unroll 1
+    for (int k = 0; k < DAT_P_GROUPS; ++k) {
+        const int64_t e0 = begin + 8 * (int64_t)(k * DAT_P_THREADS + threadIdx.x);
+        if (e0 >= hi) continue;
         const bool full = (e0 >= lo && e0 + 8 <= hi);
         float acc[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
-        if (staged) {
-#pragma unroll 1
-            for (int i = 0; i < M; ++i) {
-                float v[8];
-                p_take(q.nN + i, v);
-                if (!plain) {                       // nearly always
-                    uint32_t w[8];
-                    p_words8<RNG16>(a, e0, (uint32_t)i, w);
-                    p_levels8<RNG16>(v, w, qc, acc);
-                }
-                p_issue(a, q, q.nN + i + DAT_P_DEPTH);
-            }
-        }
         if (MODE == P_MODE_IDENTITY) {
 #pragma unroll 2
             for (int i = 0; i < M; ++i) {           // Q is the identity: the ordered fp32 sum of the workers' gradients
@@ -425,23 +351,16 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc[j] += v[j];
             }
-        } else if (staged && !plain) { }
-        else if (full && !plain) qu_rows<RNG16, true, false>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
+        } else if (full && !plain) qu_rows<RNG16, true, false>(a.gp, a.keys, qc, M, e0, lo, hi, acc);       // nearly always
         else if (full) qu_rows<RNG16, true, true>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         else if (!plain) qu_rows<RNG16, false, false>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         else qu_rows<RNG16, false, true>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
+        // theta and m only now: registers are what limits the number of resident warps here
         float th[8], m[8];
-        if (staged) {
-            p_take(q.nN + M, th);
-            p_issue(a, q, q.nN + M + DAT_P_DEPTH);
-            p_take(q.nN + M + 1, m);
-            p_issue(a, q, q.nN + M + 1 + DAT_P_DEPTH);
-        } else {
-            p_load4_cg(a.theta, e0, lo, hi, th);
-            p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
-            p_load4_cg(a.mom, e0, lo, hi, m);
-            p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
-        }
+        p_load4_cg(a.theta, e0, lo, hi, th);
+        p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
+        p_load4_cg(a.mom, e0, lo, hi, m);
+        p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
         if (MODE != P_MODE_IDENTITY && a.code_sum) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -458,51 +377,57 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
         dat_store4(a.mom, e0 + 4, lo, hi, m + 4);
     }
     __threadfence();                               // m' is read by the U part of another CTA
-    const double x = dat_block_sum(ss_theta, scratch);
-    const double y = dat_block_sum(ss_u, scratch);
-    if (threadIdx.x == 0) {
-        a.partQ[2 * (pt.tb + pt.tile)] = x;
-        a.partQ[2 * (pt.tb + pt.tile) + 1] = y;
-        __threadfence();
+    ss_theta = dat_warp_sum(ss_theta);
+    ss_u = dat_warp_sum(ss_u);
+    if ((threadIdx.x & 31) == 0) {
+        scratch[2 * (threadIdx.x >> 5)] = ss_theta;
+        scratch[2 * (threadIdx.x >> 5) + 1] = ss_u;
     }
-    if (p_arrive(a.cntQ + layer, (uint32_t)pt.T, s_flag)) p_finish_update_sums(a, layer, pt.tb, (uint32_t)pt.T, scratch);
+}
+
+// One thread, after the barrier that follows the Q part: the tile's two sums (warps in index order),
+// counted in.  Returns whether this was the layer's last tile.
+__device__ __forceinline__ bool p_quant_publish(const PArgs &a, const PipePart &pt, const double *scratch)
+{
+    double x = 0.0, y = 0.0;
+#pragma unroll
+    for (int w = 0; w < DAT_P_THREADS / 32; ++w) { x += scratch[2 * w]; y += scratch[2 * w + 1]; }
+    a.partQ[2 * ((int64_t)pt.tb + pt.tile)] = x;
+    a.partQ[2 * ((int64_t)pt.tb + pt.tile) + 1] = y;
+    __threadfence();
+    return atomicAdd(a.cntQ + pt.layer, 1u) == (uint32_t)pt.T - 1u;
 }
 
 // ---- U: theta' = theta - a_l m' (Eq. 3, pass 2) of one tile ---------------------------------------
-__device__ __forceinline__ void p_part_update(const PArgs &a, const PipePart &pt, const Seq &q)
+__device__ __forceinline__ void p_part_update(const PArgs &a, const PipePart &pt)
 {
     const int64_t lo = pt.lo, hi = pt.hi;
     const float na = -__ldcg(a.step_a + pt.layer);
-    const int64_t e0 = q.eU;
-    if (e0 >= hi) return;
-    float th[8], m[8];
-    if (q.nU > 0) {
-        p_take(q.nN + q.nQ, th);
-        p_issue(a, q, q.nN + q.nQ + DAT_P_DEPTH);
-        p_take(q.nN + q.nQ + 1, m);
-        p_issue(a, q, q.nN + q.nQ + 1 + DAT_P_DEPTH);
-    } else {
-        p_load4_cg(a.theta, e0, lo, hi, th);
-        p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
-        p_load4_cg(a.mom, e0, lo, hi, m);
-        p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
-    }
+    const uint64_t pol_first = dat_policy_evict_first();
+    const int64_t begin = p_tile_begin(pt);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) th[j] = __fmaf_rn(na, m[j], th[j]);
-    if (e0 >= lo && e0 + 8 <= hi) {
-        const uint64_t pol_first = q.pol_first;
-        dat_st4_hint(a.theta + e0, make_float4(th[0], th[1], th[2], th[3]), pol_first);
-        dat_st4_hint(a.theta + e0 + 4, make_float4(th[4], th[5], th[6], th[7]), pol_first);
-    } else {
-        dat_store4(a.theta, e0, lo, hi, th);
-        dat_store4(a.theta, e0 + 4, lo, hi, th + 4);
+    for (int k = 0; k < DAT_P_GROUPS; ++k) {
+        const int64_t e0 = begin + 8 * (int64_t)(k * DAT_P_THREADS + threadIdx.x);
+        if (e0 >= hi) continue;
+        if (e0 >= lo && e0 + 8 <= hi) {
+            float4 t0 = dat_ld4_hint(a.theta + e0, pol_first), t1 = dat_ld4_hint(a.theta + e0 + 4, pol_first);
+            const float4 m0 = dat_ld4_hint(a.mom + e0, pol_first), m1 = dat_ld4_hint(a.mom + e0 + 4, pol_first);
+            t0.x = __fmaf_rn(na, m0.x, t0.x); t0.y = __fmaf_rn(na, m0.y, t0.y); t0.z = __fmaf_rn(na, m0.z, t0.z); t0.w = __fmaf_rn(na, m0.w, t0.w);
+            t1.x = __fmaf_rn(na, m1.x, t1.x); t1.y = __fmaf_rn(na, m1.y, t1.y); t1.z = __fmaf_rn(na, m1.z, t1.z); t1.w = __fmaf_rn(na, m1.w, t1.w);
+            dat_st4_hint(a.theta + e0, t0, pol_first);
+            dat_st4_hint(a.theta + e0 + 4, t1, pol_first);
+        } else {
+            float th[8], m[8];
+            p_load4_cg(a.theta, e0, lo, hi, th);
+            p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
+            p_load4_cg(a.mom, e0, lo, hi, m);
+            p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) th[j] = __fmaf_rn(na, m[j], th[j]);
+            dat_store4(a.theta, e0, lo, hi, th);
+            dat_store4(a.theta, e0 + 4, lo, hi, th + 4);
+        }
     }
-}
-
-__device__ __forceinline__ bool p_tile_inside(const PipePart &pt)
-{
-    const int64_t begin = (pt.lo & ~(int64_t)7) + (int64_t)pt.tile * DAT_P_TILE;
-    return begin >= pt.lo && begin + DAT_P_TILE <= pt.hi;
 }
 
 template <bool RNG16, int MODE>
@@ -512,8 +437,7 @@ k_step_pipelined(const __grid_constant__ PArgs a)
     __shared__ double s_unit[4 * DAT_MAX_WORKERS];
     __shared__ float s_norm[DAT_MAX_WORKERS];
     __shared__ __align__(16) PipeItem s_item;
-    __shared__ int s_flag;
-    __shared__ int s_seen[2];                      // the layers this item waits for were already published when it started
+    __shared__ int s_ctl[4];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // items are taken in the order in which CTAs start, whatever order the hardware starts them in
     if (warp == 0) {
@@ -541,44 +465,35 @@ k_step_pipelined(const __grid_constant__ PArgs a)
         if (!P_CHECK(a, ok)) return;
     }
 #endif
-    // what the other two parts wait for: look now, so that the answer is there when it is needed
-    if (threadIdx.x < 2) {
-        const bool want = (threadIdx.x == 0) ? (pq.layer >= 0 && MODE != P_MODE_IDENTITY) : (pu.layer >= 0);
-        const uint32_t *word = (threadIdx.x == 0) ? a.readyN + pq.layer : a.readyQ + pu.layer;
-        s_seen[threadIdx.x] = want ? (p_ld_acquire(word) == a.epoch) : 1;
+    // The CTA meets at five barriers: item read; N sums in shared memory; (A) tile counted in and the Q part's
+    // layer known to be published; Q sums in shared memory; (B) tile counted in and the U part's layer
+    // published.  Between them warp 0 does the publishing and the polling.
+    if (pn.layer >= 0) p_norm_sums(a, pn, s_unit);
+    __syncthreads();
+    if (warp == 0) {
+        bool n_last = false, q_go = true;
+        if (pn.layer >= 0) n_last = p_norm_publish(a, pn, s_unit);
+        if (lane == 0) {
+            if (pq.layer >= 0 && MODE != P_MODE_IDENTITY) q_go = p_poll(a, a.readyN + pq.layer);
+            s_ctl[0] = n_last;
+            s_ctl[1] = q_go;
+        }
     }
-    // the thread's sequence of entries
-    Seq q;
-    q.pol_last = DAT_P_N_POLICY();
-    q.pol_first = dat_policy_evict_first();
-    q.pol_normal = dat_policy_evict_normal();
-    q.u0 = warp * (4 * a.M) / 8;
-    q.nN = (pn.layer >= 0 && p_tile_inside(pn)) ? 2 * ((warp + 1) * (4 * a.M) / 8 - q.u0) : 0;
-    q.nQ = (pq.layer >= 0 && MODE != P_MODE_IDENTITY && p_tile_inside(pq)) ? a.M + 2 : 0;
-    q.nU = 0;                                      // known once s_seen[1] is
-    q.eN = (pn.lo & ~(int64_t)7) + (int64_t)pn.tile * DAT_P_TILE + 4 * lane;
-    q.eQ = (pq.lo & ~(int64_t)7) + (int64_t)pq.tile * DAT_P_TILE + 8 * (int64_t)threadIdx.x;
-    q.eU = (pu.lo & ~(int64_t)7) + (int64_t)pu.tile * DAT_P_TILE + 8 * (int64_t)threadIdx.x;
-    // DEPTH entries ahead; the first DEPTH entries never reach the U part unless N and Q are both absent or short,
-    // in which case U is fetched the plain way
-#pragma unroll
-    for (int j = 0; j < DAT_P_DEPTH; ++j) p_issue(a, q, j);
-
-    if (pn.layer >= 0) p_norm_sums(a, pn, q, s_unit);
-    __syncthreads();                               // s_seen is there (and every warp's unit sums)
-    // m' of the U tile may be fetched ahead only if its layer was seen published (then it is visible)
-    if (pu.layer >= 0 && s_seen[1] && p_tile_inside(pu) && q.nQ >= DAT_P_DEPTH) q.nU = 2;    // (its entries have not been passed yet)
-    if (pn.layer >= 0) p_norm_publish(a, pn, s_unit, s_norm, &s_flag);
-    bool alive = true;
-    if (pq.layer >= 0) {
-        alive = (MODE == P_MODE_IDENTITY) || s_seen[0] || p_wait(a, a.readyN + pq.layer, &s_flag);
-        if (alive) p_part_quant<RNG16, MODE>(a, pq, q, s_unit, &s_flag);
+    __syncthreads();                               // (A)
+    if (s_ctl[0]) p_norm_finish(a, pn, s_norm);
+    const bool alive = (s_ctl[1] != 0);
+    if (alive && pq.layer >= 0) p_part_quant<RNG16, MODE>(a, pq, s_unit);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bool q_last = false, u_go = alive;
+        if (alive && pq.layer >= 0) q_last = p_quant_publish(a, pq, s_unit);
+        if (alive && pu.layer >= 0) u_go = p_poll(a, a.readyQ + pu.layer);
+        s_ctl[2] = q_last;
+        s_ctl[3] = u_go;
     }
-    if (alive && pu.layer >= 0) {
-        alive = s_seen[1] || p_wait(a, a.readyQ + pu.layer, &s_flag);
-        if (alive) p_part_update(a, pu, q);
-    }
-    p_cp_wait<0>();
+    __syncthreads();                               // (B)
+    if (s_ctl[2]) p_quant_finish(a, pq, s_unit);
+    if (s_ctl[3] && pu.layer >= 0) p_part_update(a, pu);
 }
 
 // ---- host: the item list -----------------------------------------------------------------------------
@@ -661,10 +576,7 @@ int dat_pipe_build(dat_plan_t *plan)
         g->sync_bytes = (2 + 4 * (size_t)h) * 4;
         const size_t o_sync = take(g->sync_bytes);
         g->mem_bytes = off;
-        cudaError_t e = cudaFuncSetAttribute(k_step_pipelined<true, P_MODE_IDENTITY>, cudaFuncAttributeMaxDynamicSharedMemorySize, DAT_P_STAGE_BYTES);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_step_pipelined<true, P_MODE_SHARED>, cudaFuncAttributeMaxDynamicSharedMemorySize, DAT_P_STAGE_BYTES);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_step_pipelined<false, P_MODE_SHARED>, cudaFuncAttributeMaxDynamicSharedMemorySize, DAT_P_STAGE_BYTES);
-        if (e != cudaSuccess) return dat_cuda_fail(plan, e);
+        cudaError_t e;
         e = cudaMalloc((void **)&g->mem, off);
         if (e != cudaSuccess) { g->mem = nullptr; plan->last_cuda = (int)e; (void)cudaGetLastError(); return DAT_ERR_NOMEM; }
         g->d_items = (PipeItem *)(g->mem + o_items);
@@ -751,9 +663,26 @@ extern "C" int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, co
     a.n_tiles = g->n_tiles;
     cudaStream_t s = (cudaStream_t)stream;
     const unsigned grid = (unsigned)g->n_items;
-    if (identity) k_step_pipelined<true, P_MODE_IDENTITY><<<grid, DAT_P_THREADS, DAT_P_STAGE_BYTES, s>>>(a);
-    else if (plan->rng_bits == 16) k_step_pipelined<true, P_MODE_SHARED><<<grid, DAT_P_THREADS, DAT_P_STAGE_BYTES, s>>>(a);
-    else k_step_pipelined<false, P_MODE_SHARED><<<grid, DAT_P_THREADS, DAT_P_STAGE_BYTES, s>>>(a);
+    if (identity) k_step_pipelined<true, P_MODE_IDENTITY><<<grid, DAT_P_THREADS, 0, s>>>(a);
+    else if (plan->rng_bits == 16) k_step_pipelined<true, P_MODE_SHARED><<<grid, DAT_P_THREADS, 0, s>>>(a);
+    else k_step_pipelined<false, P_MODE_SHARED><<<grid, DAT_P_THREADS, 0, s>>>(a);
     DAT_LAUNCHED(plan);
+    return DAT_OK;
+}
+
+// Test hook (see dat.h): a short wait limit, and a layer whose norm never completes in the next call.
+extern "C" int dat_plan_test_stall(dat_plan_t *plan, int64_t wait_cycles, int64_t layer, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    PipeSchedule *g = plan->pipe;
+    if (!g || !g->mem || wait_cycles < 0 || layer >= plan->h) return DAT_ERR_ARG;
+    g->wait_cycles = wait_cycles ? (long long)wait_cycles : DAT_P_WAIT_CYCLES;
+    if (layer >= 0) {
+        // a count that the layer's tiles cannot bring to T - 1: nobody becomes the layer's last tile
+        static const uint32_t far = 0x40000000u;
+        DAT_CUDA(plan, cudaMemcpyAsync(g->d_sync + 2 + layer, &far, sizeof far, cudaMemcpyHostToDevice, (cudaStream_t)stream));
+        DAT_CUDA(plan, cudaStreamSynchronize((cudaStream_t)stream));
+    }
     return DAT_OK;
 }

@@ -145,7 +145,6 @@ extern "C" int dat_plan_destroy(dat_plan_t *plan)
     if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
     if (prev != plan->device) cudaSetDevice(plan->device);
     if (cudaDeviceSynchronize() != cudaSuccess) rc = DAT_ERR_CUDA;
-    dat_fused_destroy(plan);
     dat_pipe_destroy(plan);
     if (plan->stage) cudaFree(plan->stage);
     if (plan->d_tile_base8) cudaFree(plan->d_tile_base8);

@@ -793,6 +793,11 @@ extern "C" int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_off
     }
     StaticScratch *sc = g_static_ptr[dev];
     cudaStream_t s = (cudaStream_t)stream;
+    // the tables are copied from host memory (one of them from this function's stack) on every call:
+    // a captured graph would replay those copies from dead memory
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) { (void)cudaGetLastError(); return DAT_ERR_CUDA; }
+    if (cap != cudaStreamCaptureStatusNone) return DAT_ERR_UNSUPPORTED;
     const size_t table = (size_t)(num_layers + 1) * sizeof(int64_t);
     cudaError_t e = cudaMemcpyAsync(sc->off, layer_offsets, table, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess) e = cudaMemcpyAsync(sc->tile_base, tile_base, table, cudaMemcpyHostToDevice, s);
@@ -931,7 +936,6 @@ extern "C" int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const
     DAT_LAUNCHED(plan);
     if (scales_out) DAT_CUDA(plan, cudaMemcpyAsync(scales_out, plan->d_scales, (size_t)h * 4, cudaMemcpyDeviceToDevice, s));
     const PhiloxKeys keys = dat_make_keys(seed, step);
-    if (plan->probe_before) DAT_CUDA(plan, cudaEventRecord((cudaEvent_t)plan->probe_before, s));
     if (plan->rng_bits == 16)
         k_quant_update<true><<<(unsigned)plan->n_tiles8, DAT_QU_THREADS, 0, s>>>(gp, keys, plan->d_offsets, plan->d_tile_base8, h, plan->M,
                                                                                  plan->d_qmul, plan->d_dq, theta, mom, S_f, hp->momentum,
@@ -941,7 +945,6 @@ extern "C" int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const
                                                                                   plan->d_qmul, plan->d_dq, theta, mom, S_f, hp->momentum,
                                                                                   hp->weight_decay, plan->d_partials8, code_sum_out);
     DAT_LAUNCHED(plan);
-    if (plan->probe_after) DAT_CUDA(plan, cudaEventRecord((cudaEvent_t)plan->probe_after, s));
     k_lalr_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base8, plan->d_partials8, hp->lr, hp->c_l, hp->c_u, plan->d_step_a,
                                               layer_norms_out, plan->d_status);
     DAT_LAUNCHED(plan);
@@ -951,30 +954,11 @@ extern "C" int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const
 }
 
 // ------------------------------------------------------------------------------------------
-// dat_step: one call for Steps 7, 9 and 12.  Two implementations give the same results (the norms
-// may differ in their last place, everything else follows from them bit for bit): the single
-// persistent sweep (dat_step_sweep) and the three passes above (dat_step_passes).  The passes are
-// the faster of the two from about a million elements on (measured on ResNet-18 .. 1B-parameter
-// shapes, M = 6 .. 32); below that the sweep's single launch wins.
+// dat_step: one call for Steps 7, 9 and 12 -- the single pipelined launch of dat_pipeline.cu.
 // ------------------------------------------------------------------------------------------
-#define DAT_STEP_PASSES_FROM ((int64_t)1 << 20)
-
 extern "C" int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
                         uint64_t seed, uint64_t step, const dat_hparams_t *hp,
                         int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
 {
-    if (plan && (plan->bits == 32 || plan->scale_mode == DAT_SCALE_SHARED_MAX))
-        return dat_step_pipelined(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
-    return dat_step_sweep(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
-}
-
-// Measurement aid: two CUDA events of the caller's (or NULL, NULL to switch it off) that the next
-// calls of dat_step_passes record on their stream just before and just after k_quant_update, the
-// largest kernel of the step, so that its duration can be read without a profiler.
-extern "C" int dat_plan_set_probe(dat_plan_t *plan, void *event_before, void *event_after)
-{
-    if (!plan || ((event_before == nullptr) != (event_after == nullptr))) return DAT_ERR_ARG;
-    plan->probe_before = event_before;
-    plan->probe_after = event_after;
-    return DAT_OK;
+    return dat_step_pipelined(plan, theta, mom, grads, seed, step, hp, code_sum_out, layer_norms_out, scales_out, stream);
 }

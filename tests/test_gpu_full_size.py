@@ -1,8 +1,7 @@
-"""Parity at the full sizes of the workloads, in the launch configuration bench.py times
-(dat_step, which takes the three passes at these sizes, and the persistent sweep by itself; inputs
-generated on the device).  The oracle recomputes sampled layers one by
-one (its window mode keeps the global element index, hence the same random stream); properties
-that hold at any size are checked on everything."""
+"""Parity at the full sizes of the workloads, in the launch configuration bench.py times (dat_step;
+inputs generated on the device).  The oracle recomputes sampled layers one by one (its window mode
+keeps the global element index, hence the same random stream); properties that hold at any size are
+checked on everything."""
 import numpy as np
 import pytest
 import torch
@@ -12,7 +11,7 @@ from helpers import assert_close_per_layer, hp_tuple, np_of, ulp_diff
 pytestmark = pytest.mark.gpu
 
 
-ENTRIES = ["dat_step", "dat_step_sweep"]
+ENTRIES = ["dat_step", "dat_step_passes"]
 
 
 def _run_and_check(oracle, cfg, sample_layers, step=0, entry="dat_step"):
@@ -42,6 +41,7 @@ def _run_and_check(oracle, cfg, sample_layers, step=0, entry="dat_step"):
     csum = torch.cat([torch.zeros(1, dtype=torch.float64, device=dev), torch.cumsum(d64, 0)])
     idx = torch.from_numpy(offs).to(dev)
     step_len = torch.sqrt((csum[idx[1:]] - csum[idx[:-1]]).clamp_min(0)).cpu().numpy()
+    del d64, csum
     for l in range(cfg.h):
         tau = min(max(float(norms_h[l, 0]), cfg.c_l), cfg.c_u)
         expect = cfg.lr * tau if norms_h[l, 1] != 0 else 0.0
@@ -71,29 +71,46 @@ def test_resnet50_bench_configuration_every_layer(oracle, entry):
     _run_and_check(oracle, cfg, range(cfg.h), entry=entry)
 
 
+def test_resnet50_every_layer_23_bit_uniform(oracle):
+    """The bench workload once more at the other resolution of the quantizer's uniform number."""
+    from paper_2206_06257_b200 import synth
+    cfg = synth.config("resnet50")
+    cfg.rng_bits = 23
+    _run_and_check(oracle, cfg, range(cfg.h), step=3)
+
+
 @pytest.mark.parametrize("entry", ENTRIES)
 def test_resnet50_m32_b4_student_t_with_zero_layers(oracle, entry):
+    """M = 32: a large layer's gradients (302 MB) do not fit the L2 cache.  One of the largest layers
+    (2.36 M elements) is among those compared element by element."""
     from paper_2206_06257_b200 import synth
     cfg = synth.config("resnet50_m32")
     zg, zp = cfg.zero_grad_layers[0], cfg.zero_param_layers[0]
+    sizes = np.diff(cfg.offsets)
     sample = sorted(set(list(range(0, cfg.h, 7)) + [zg, zp, 159, 160]))
-    sample = [l for l in sample if cfg.offsets[l + 1] - cfg.offsets[l] <= 1_100_000]
+    sample = [l for l in sample if sizes[l] <= 1_100_000] + [int(np.argmax(sizes))]
     theta, mom = _run_and_check(oracle, cfg, sample, entry=entry)
     a, b = int(cfg.offsets[zp]), int(cfg.offsets[zp + 1])
     assert not theta[a:b].any() and mom[a:b].any()          # all-zero tensor does not move (c_l = 0)
 
 
 @pytest.mark.parametrize("entry", ENTRIES)
-@pytest.mark.parametrize("bits", [2, 8])
+@pytest.mark.parametrize("bits", [2, 4, 8])
 def test_flat_1b_sampled_layers(oracle, bits, entry):
+    """The 1B-parameter model at every bit width of its sweep.  Compared element by element: the two
+    smallest layers, layers near the median and the lower third, the first and the last layer, one of
+    about 300 k elements, one between 0.42 M and 2 M elements (several tiles of one layer per thread
+    block row), and the largest layer (about 16 M elements)."""
     from paper_2206_06257_b200 import synth
     if torch.cuda.get_device_properties(0).total_memory < 80e9:
         pytest.skip("needs about 60 GB of device memory")
     cfg = synth.config("flat1b", bits=bits)
     sizes = np.diff(cfg.offsets)
     order = np.argsort(sizes)
+    mid = [int(l) for l in order if 420_000 <= sizes[l] <= 2_000_000]
     sample = sorted(set([int(order[0]), int(order[1]), int(order[len(order) // 2]), int(order[len(order) // 3]),
-                         0, cfg.h - 1, int(np.argmin(np.abs(sizes - 300_000)))]))
-    sample = [l for l in sample if sizes[l] <= 2_000_000]
+                         0, cfg.h - 1, int(np.argmin(np.abs(sizes - 300_000))), mid[len(mid) // 2], int(order[-1])]))
+    if entry != "dat_step":                                  # the large layers once per bit width are enough
+        sample = [l for l in sample if sizes[l] <= 2_000_000]
     _run_and_check(oracle, cfg, sample, entry=entry)
     torch.cuda.empty_cache()

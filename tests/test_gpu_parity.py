@@ -261,6 +261,52 @@ def test_step_passes_worker_counts_and_extreme_scales(api, oracle, M, rng_bits):
     _check_fused(api, oracle, offs, grads, theta, mom, 8, HP, rng_bits=rng_bits, entry="dat_step_passes")
 
 
+def test_bounded_wait_runs_out_and_plan_recovers(api, oracle):
+    """The wait of a work item for a layer's norm is bounded.  With the test hook the limit is set to about a
+    millisecond and one layer's tile counter is pre-set so that the layer never completes: the call must
+    return, the status word must carry DAT_STATUS_TIMEOUT, and after dat_get_status the next ordinary call
+    on the same plan must give what a fresh plan gives, bit for bit."""
+    import time
+    offs, grads, theta, mom = _random_problem(77, [5000, 300, 9000, 40], 3)
+    g_dev = [torch.from_numpy(g).cuda() for g in grads]
+    with GpuPlan(api, offs, 3, 8) as P:
+        api.dat_plan_test_stall(P.plan, 2_000_000, 2)
+        th, mo = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        t0 = time.time()
+        api.dat_step(P.plan, th, mo, g_dev, 5, 9, HP)
+        torch.cuda.synchronize()
+        assert time.time() - t0 < 10.0
+        assert P.status() & api.DAT_STATUS_TIMEOUT
+        assert P.status() == 0                                  # read and cleared
+        api.dat_plan_test_stall(P.plan, 0, -1)                  # the default limit again
+        th1, mo1 = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        api.dat_step(P.plan, th1, mo1, g_dev, 5, 9, HP)
+        torch.cuda.synchronize()
+        assert P.status() == 0
+        with GpuPlan(api, offs, 3, 8) as P2:
+            th2, mo2 = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+            api.dat_step(P2.plan, th2, mo2, g_dev, 5, 9, HP)
+            torch.cuda.synchronize()
+        assert torch.equal(th1, th2) and torch.equal(mo1, mo2)
+        ref = oracle.step(offs, theta, mom, grads, 8, 5, 9, *HP)
+        assert_close_per_layer(np_of(th1), ref["theta"], offs, "theta after recovery")
+
+
+def test_self_checking_build_runs_the_ragged_cases():
+    """The build with -DDAT_SELFCHECK (DAT_DEBUG=1: every tile an item names is checked before use, a
+    violation sets DAT_STATUS_BOUNDS instead of faulting) passes the ragged parity cases with a clean status."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    if not os.path.exists(os.path.join(root, "paper_2206_06257_b200", "libdat_debug.so")):
+        pytest.skip("libdat_debug.so has not been built (DAT_DEBUG=1 python -m paper_2206_06257_b200.build)")
+    r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", os.path.join(root, "tests", "test_gpu_parity.py"),
+                        "-k", "test_fused_parity_ragged and rng16"], env=dict(os.environ, DAT_DEBUG="1"),
+                       cwd=root, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
 def test_step_passes_equals_fused_on_resnet18(api, oracle):
     from paper_2206_06257_b200 import synth
     cfg = synth.config("resnet18")
