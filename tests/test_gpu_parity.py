@@ -299,10 +299,10 @@ def test_self_checking_build_runs_the_ragged_cases():
     import subprocess
     import sys
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    if not os.path.exists(os.path.join(root, "paper_2206_06257_b200", "libdat_debug.so")):
-        pytest.skip("libdat_debug.so has not been built (DAT_DEBUG=1 python -m paper_2206_06257_b200.build)")
+    env = dict(os.environ, DAT_DEBUG="1")
+    subprocess.check_call([sys.executable, "-m", "paper_2206_06257_b200.build"], cwd=root, env=env)   # no-op when up to date
     r = subprocess.run([sys.executable, "-m", "pytest", "-q", "-x", "-m", "gpu", os.path.join(root, "tests", "test_gpu_parity.py"),
-                        "-k", "test_fused_parity_ragged and rng16"], env=dict(os.environ, DAT_DEBUG="1"),
+                        "-k", "test_fused_parity_ragged and rng16"], env=env,
                        cwd=root, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
 
