@@ -79,8 +79,8 @@ typedef struct dat_lamb_hparams {
  * PER_WORKER: nu_{i,l} = ||g_l^(i)||_2, every worker's own norm, as Eq. rand_q and Eq. grad_agg
  *             are written: g_hat = (1/M) sum_i nu_{i,l} * sign * level / S, summed in fp32.  The
  *             message then carries M*h norms (index i*h + l), and no integer code sum exists.
- *             Available in the separate calls (dat_quantize, dat_aggregate); dat_step sums
- *             integer codes and answers DAT_ERR_UNSUPPORTED for such a plan.                   */
+ *             dat_step_passes, which sums integer codes, answers DAT_ERR_UNSUPPORTED for such a
+ *             plan; every other call takes it.                                                  */
 enum { DAT_SCALE_SHARED_MAX = 0, DAT_SCALE_PER_WORKER = 1 };
 
 /* Resolution of the quantizer's uniform number (see dat_plan_create). */
@@ -289,7 +289,10 @@ int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_offsets, float
  * usual, DAT_STATUS_TIMEOUT is set in the status word, and the outputs of that call -- and of
  * later calls on the plan -- are undefined until dat_get_status has been called, which reports the
  * bit and restores the plan's counters.
- * Errors: ARG, ALIGN, UNSUPPORTED (a plan with DAT_SCALE_PER_WORKER and b < 32), CUDA.
+ * With a DAT_SCALE_PER_WORKER plan the step follows Eq. grad_agg as written (every worker on its own grid,
+ * fp32 sum in ascending worker order): scales_out then has M*h entries (index i*h + l) and code_sum_out is
+ * ignored (no integer sums exist).
+ * Errors: ARG, ALIGN, CUDA.
  * ------------------------------------------------------------------------------------------- */
 int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
              uint64_t seed, uint64_t step, const dat_hparams_t *hp,
@@ -304,6 +307,16 @@ int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *gra
 int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
                        uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,
                        float *layer_norms_out, float *scales_out, void *stream);
+
+/* dat_step_lamb -- dat_step with LAMB (Algorithm A2) as the outer-minimisation oracle instead of the momentum
+ * direction: Steps 7 and 9 as in dat_step, then m', v', the bias-corrected direction and the layer-wise update
+ * exactly as dat_lamb_step computes them from g_hat -- in the same single launch, g_hat never stored.
+ *   var   device fp32[d], the second moment, updated in place;  t >= 1 the iteration count;  hp as in dat_lamb_step.
+ * Other arguments, the bounded wait and its status bit as in dat_step.
+ * Errors: ARG (null pointer, t < 1, beta outside (0,1)), ALIGN, CUDA. */
+int dat_step_lamb(dat_plan_t *plan, float *theta, float *mom, float *var, const float *const *grads,
+                  uint64_t seed, uint64_t step, const dat_lamb_hparams_t *hp, int64_t t,
+                  int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream);
 
 /* dat_step_passes -- the same step as dat_step, with the same arguments and the same results bit for
  * bit up to the norms' last place, computed by three streaming passes in separate launches: quantizer

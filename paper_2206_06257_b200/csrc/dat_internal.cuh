@@ -26,6 +26,12 @@ struct PhiloxKeys {
 
 struct PipeSchedule;    // dat_pipeline.cu
 
+// LAMB (Algorithm A2): what the kernels need of the hyper-parameters at iteration t.
+struct LambConst {
+    float beta1, beta2, om1, om2, bc1, bc2, zeta, wd;
+};
+LambConst dat_lamb_const(const dat_lamb_hparams_t *hp, int64_t t);   // dat_plan.cu
+
 struct dat_plan {
     int device = 0;
     int64_t h = 0, d = 0;
@@ -257,6 +263,15 @@ __device__ __forceinline__ void dat_store4(float *__restrict__ p, int64_t e0, in
     }
 }
 
+// The LAMB direction of one element from the stored moments: u = m^/(sqrt(v^) + zeta) + wd*theta with the
+// bias-corrected m^ = m'/(1 - beta1^t), v^ = v'/(1 - beta2^t) (Algorithm A2; one rounding per operation).
+__device__ __forceinline__ float dat_lamb_direction(const LambConst &c, float m_new, float v_new, float theta)
+{
+    const float m_hat = m_new / c.bc1;
+    const float v_hat = v_new / c.bc2;
+    return __fmaf_rn(c.wd, theta, m_hat / (sqrtf(v_hat) + c.zeta));
+}
+
 // ------------------------------------------------------------------------------------------
 // 16-byte global loads and stores that stay out of L1 and carry an L2 eviction priority.
 // ------------------------------------------------------------------------------------------
@@ -321,7 +336,10 @@ template <bool RNG16, bool FULL, bool PLAIN>
 __device__ __forceinline__ void qu_rows_body(const GradPtrs &gp, const PhiloxKeys &keys, const QuConst &qc, int M, int64_t e0,
                                              int64_t lo, int64_t hi, float acc[8])
 {
-    const uint64_t pol = dat_policy_evict_first();   // a gradient is dead once its level is drawn
+#ifndef DAT_QU_POLICY
+#define DAT_QU_POLICY dat_policy_evict_first
+#endif
+    const uint64_t pol = DAT_QU_POLICY();             // a gradient is dead once its level is drawn
     DAT_QU_UNROLL_N(DAT_QU_UNROLL)
     for (int i = 0; i < M; ++i) {
         float v[8];

@@ -34,12 +34,16 @@
 #ifndef DAT_P_LAG                                 // items between the last N tile of a layer and its first Q tile
 #define DAT_P_LAG 256
 #endif
+#ifndef DAT_P_LAG_U                               // items between the last Q tile of a layer and its first U tile
+#define DAT_P_LAG_U DAT_P_LAG
+#endif
 #ifndef DAT_P_REVERSE_FROM                        // layers of at least this many tiles: Q walks back from the last tile
 #define DAT_P_REVERSE_FROM 320
 #endif
 #define DAT_P_WAIT_CYCLES (4000000000ll)          // about two seconds
 
-enum { P_MODE_SHARED = 0, P_MODE_IDENTITY = 2 };
+enum { P_MODE_SHARED = 0, P_MODE_PER_WORKER = 1, P_MODE_IDENTITY = 2 };
+enum { P_OPT_MOMENTUM = 0, P_OPT_LAMB = 1 };     // the descent direction u of Eq. 3: heavy-ball momentum, or Algorithm A2
 
 struct PipePart {                                 // one tile of one layer; layer < 0: none
     int64_t lo, hi;                               // the layer's element range
@@ -70,7 +74,8 @@ struct PArgs {
     PhiloxKeys keys;
     const PipeItem *items;
     const int64_t *off, *tile_base;
-    float *theta, *mom;
+    float *theta, *mom, *var;                     // var: second moment (LAMB only)
+    LambConst lamb;
     double *partN, *partQ;
     uint32_t *ticket, *abort_epoch, *cntN, *cntQ, *readyN, *readyQ, *status;
     float *worker_norms, *scales, *qmul, *dq, *step_a;
@@ -161,7 +166,10 @@ __device__ __forceinline__ void p_norm_sums(const PArgs &a, const PipePart &pt, 
     double acc = 0.0;
     int run = u0;
     if (p_tile_inside(pt)) {
-        const uint64_t pol = dat_policy_evict_last();  // the Q part of a later item reads these lines again
+#ifndef DAT_P_N_POLICY
+#define DAT_P_N_POLICY dat_policy_evict_last
+#endif
+        const uint64_t pol = DAT_P_N_POLICY();         // the Q part of a later item reads these lines again
 #pragma unroll 1
         for (int ub = u0; ub < u1; ub += UPB) {
             float4 v[8];
@@ -242,6 +250,7 @@ __device__ __forceinline__ bool p_norm_publish(const PArgs &a, const PipePart &p
 
 // The CTA that counted in the layer's last N tile (every thread): nu_{i,l} = sqrt(sum over the tiles),
 // nu_l = max_i, and the layer's two factors, published with the call's epoch.
+template <int MODE>
 __device__ __forceinline__ void p_norm_finish(const PArgs &a, const PipePart &pt, float *s_norm)
 {
     const int M = a.M, layer = pt.layer;
@@ -273,10 +282,18 @@ __device__ __forceinline__ void p_norm_finish(const PArgs &a, const PipePart &pt
             bad |= !isfinite(s_norm[i]);
             nu = (s_norm[i] > nu) ? s_norm[i] : nu;
         }
-        a.scales[layer] = nu;
-        a.qmul[layer] = (nu == 0.0f) ? 0.0f : a.S_f / nu;
-        a.dq[layer] = (nu == 0.0f) ? 0.0f : nu / a.SM_f;
-        if (a.scales_out) a.scales_out[layer] = nu;
+        if (MODE == P_MODE_PER_WORKER) {
+            // every worker keeps its own norm (Eq. rand_q as written): index i*h + l; nu_{i,l} itself is in worker_norms
+            for (int i = 0; i < M; ++i) {
+                a.qmul[(int64_t)i * a.h + layer] = (s_norm[i] == 0.0f) ? 0.0f : a.S_f / s_norm[i];
+                if (a.scales_out) a.scales_out[(int64_t)i * a.h + layer] = s_norm[i];
+            }
+        } else {
+            a.scales[layer] = nu;
+            a.qmul[layer] = (nu == 0.0f) ? 0.0f : a.S_f / nu;
+            a.dq[layer] = (nu == 0.0f) ? 0.0f : nu / a.SM_f;
+            if (a.scales_out) a.scales_out[layer] = nu;
+        }
         if (bad) atomicOr(a.status, DAT_STATUS_NONFINITE);
         a.cntN[layer] = 0u;
         __threadfence();
@@ -318,16 +335,52 @@ __device__ __forceinline__ void p_quant_finish(const PArgs &a, const PipePart &p
     }
 }
 
+// Eq. grad_agg as written, every worker on its own grid: acc = sum_i nu_{i,l} * (signed level_i), in fp32
+// with one fused multiply-add per worker, ascending; the caller divides by S*M.  Levels by the plain form
+// of Eq. xi with the worker's own S/nu_{i,l}.
+template <bool RNG16>
+__device__ __forceinline__ void p_rows_per_worker(const PArgs &a, int layer, int64_t e0, int64_t lo, int64_t hi, float acc[8])
+{
+    const bool full = (e0 >= lo && e0 + 8 <= hi);
+    const uint64_t pol = dat_policy_evict_first();
+    const float two_b = a.S_f + 1.0f;
+#pragma unroll 1
+    for (int i = 0; i < a.M; ++i) {
+        float v[8];
+        if (full) {
+            const float4 a0 = dat_ld4_hint(a.gp.p[i] + e0, pol), a1 = dat_ld4_hint(a.gp.p[i] + e0 + 4, pol);
+            v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+        } else {
+            dat_load4(a.gp.p[i], e0, lo, hi, v);
+            dat_load4(a.gp.p[i], e0 + 4, lo, hi, v + 4);
+        }
+        const float t = __ldcg(a.qmul + (int64_t)i * a.h + layer), nu = __ldcg(a.worker_norms + (int64_t)i * a.h + layer);
+        uint32_t w[8];
+        if (RNG16) {
+            dat_random_words((uint64_t)e0 >> 3, (uint32_t)i, a.keys, w);
+        } else {
+            dat_random_words((uint64_t)e0 >> 2, (uint32_t)i, a.keys, w);
+            dat_random_words(((uint64_t)e0 >> 2) + 1, (uint32_t)i, a.keys, w + 4);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float u1 = RNG16 ? dat_u1_from_half((j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xFFFFu)) : dat_u1_from_word(w[j]);
+            const float lf = (float)dat_level_u1(v[j], t, two_b, u1);
+            acc[j] = __fmaf_rn(nu, (v[j] < 0.0f) ? -lf : lf, acc[j]);
+        }
+    }
+}
+
 // ---- Q: levels (Eq. xi), signed sum over the workers and g_hat (Eq. grad_agg), m' and the layer sums
 // (Eq. 3, pass 1) of one tile; codes, sums and g_hat stay in registers.  Leaves the tile's two sums per
 // warp in scratch[2w], scratch[2w + 1]. -------------------------------------------------------------
-template <bool RNG16, int MODE>
+template <bool RNG16, int MODE, int OPT>
 __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt, double *scratch)
 {
     const int M = a.M, layer = pt.layer;
     const int64_t lo = pt.lo, hi = pt.hi;
     float t = 0.0f, f = 0.0f;
-    if (MODE != P_MODE_IDENTITY) { t = __ldcg(a.qmul + layer); f = __ldcg(a.dq + layer); }
+    if (MODE == P_MODE_SHARED) { t = __ldcg(a.qmul + layer); f = __ldcg(a.dq + layer); }
     const float two_b = a.S_f + 1.0f, inv_two_b = 1.0f / two_b;
     // scaled form of Eq. xi: valid while t 2^-b is a normal number
     const bool plain = (t != 0.0f) && !(t >= 1.17549435e-38f * two_b && t <= 3.402823466e38f);
@@ -351,7 +404,8 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
 #pragma unroll
                 for (int j = 0; j < 8; ++j) acc[j] += v[j];
             }
-        } else if (full && !plain) qu_rows<RNG16, true, false>(a.gp, a.keys, qc, M, e0, lo, hi, acc);       // nearly always
+        } else if (MODE == P_MODE_PER_WORKER) p_rows_per_worker<RNG16>(a, layer, e0, lo, hi, acc);
+        else if (full && !plain) qu_rows<RNG16, true, false>(a.gp, a.keys, qc, M, e0, lo, hi, acc);       // nearly always
         else if (full) qu_rows<RNG16, true, true>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         else if (!plain) qu_rows<RNG16, false, false>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         else qu_rows<RNG16, false, true>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
@@ -361,22 +415,41 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
         p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
         p_load4_cg(a.mom, e0, lo, hi, m);
         p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
-        if (MODE != P_MODE_IDENTITY && a.code_sum) {
+        if (MODE == P_MODE_SHARED && a.code_sum) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
                 if (e0 + j >= lo && e0 + j < hi) a.code_sum[e0 + j] = (int)acc[j];
         }
+        if (OPT == P_OPT_LAMB) {
+            // Algorithm A2: both moments are stored, the direction is formed on the fly for the layer sums
+            float v[8];
+            p_load4_cg(a.var, e0, lo, hi, v);
+            p_load4_cg(a.var, e0 + 4, lo, hi, v + 4);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float ghat = (MODE == P_MODE_IDENTITY) ? acc[j] / a.M_f : acc[j] * f;
-            m[j] = __fmaf_rn(a.mu, m[j], __fmaf_rn(a.wd, th[j], ghat));
-            ss_theta = fma((double)th[j], (double)th[j], ss_theta);
-            ss_u = fma((double)m[j], (double)m[j], ss_u);
+            for (int j = 0; j < 8; ++j) {
+                const float ghat = (MODE == P_MODE_IDENTITY) ? acc[j] / a.M_f : (MODE == P_MODE_PER_WORKER) ? acc[j] / a.SM_f : acc[j] * f;
+                m[j] = __fmaf_rn(a.lamb.beta1, m[j], __fmul_rn(a.lamb.om1, ghat));
+                v[j] = __fmaf_rn(a.lamb.beta2, v[j], __fmul_rn(a.lamb.om2, __fmul_rn(ghat, ghat)));
+                const bool inside = (e0 + j >= lo && e0 + j < hi);
+                const float u = inside ? dat_lamb_direction(a.lamb, m[j], v[j], th[j]) : 0.0f;
+                ss_theta = fma((double)th[j], (double)th[j], ss_theta);
+                ss_u = fma((double)u, (double)u, ss_u);
+            }
+            dat_store4(a.var, e0, lo, hi, v);
+            dat_store4(a.var, e0 + 4, lo, hi, v + 4);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const float ghat = (MODE == P_MODE_IDENTITY) ? acc[j] / a.M_f : (MODE == P_MODE_PER_WORKER) ? acc[j] / a.SM_f : acc[j] * f;
+                m[j] = __fmaf_rn(a.mu, m[j], __fmaf_rn(a.wd, th[j], ghat));
+                ss_theta = fma((double)th[j], (double)th[j], ss_theta);
+                ss_u = fma((double)m[j], (double)m[j], ss_u);
+            }
         }
         dat_store4(a.mom, e0, lo, hi, m);
         dat_store4(a.mom, e0 + 4, lo, hi, m + 4);
     }
-    __threadfence();                               // m' is read by the U part of another CTA
+    __threadfence();                               // m' (and v') are read by the U part of another CTA
     ss_theta = dat_warp_sum(ss_theta);
     ss_u = dat_warp_sum(ss_u);
     if ((threadIdx.x & 31) == 0) {
@@ -399,6 +472,7 @@ __device__ __forceinline__ bool p_quant_publish(const PArgs &a, const PipePart &
 }
 
 // ---- U: theta' = theta - a_l m' (Eq. 3, pass 2) of one tile ---------------------------------------
+template <int OPT>
 __device__ __forceinline__ void p_part_update(const PArgs &a, const PipePart &pt)
 {
     const int64_t lo = pt.lo, hi = pt.hi;
@@ -409,7 +483,24 @@ __device__ __forceinline__ void p_part_update(const PArgs &a, const PipePart &pt
     for (int k = 0; k < DAT_P_GROUPS; ++k) {
         const int64_t e0 = begin + 8 * (int64_t)(k * DAT_P_THREADS + threadIdx.x);
         if (e0 >= hi) continue;
-        if (e0 >= lo && e0 + 8 <= hi) {
+        if (OPT == P_OPT_LAMB) {
+            // the direction once more from the stored moments: the same fp32 operations give the same bits
+            float th[8], m[8], v[8];
+            p_load4_cg(a.theta, e0, lo, hi, th);
+            p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
+            p_load4_cg(a.mom, e0, lo, hi, m);
+            p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
+            p_load4_cg(a.var, e0, lo, hi, v);
+            p_load4_cg(a.var, e0 + 4, lo, hi, v + 4);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const bool inside = (e0 + j >= lo && e0 + j < hi);
+                const float u = inside ? dat_lamb_direction(a.lamb, m[j], v[j], th[j]) : 0.0f;
+                th[j] = __fmaf_rn(na, u, th[j]);
+            }
+            dat_store4(a.theta, e0, lo, hi, th);
+            dat_store4(a.theta, e0 + 4, lo, hi, th + 4);
+        } else if (e0 >= lo && e0 + 8 <= hi) {
             float4 t0 = dat_ld4_hint(a.theta + e0, pol_first), t1 = dat_ld4_hint(a.theta + e0 + 4, pol_first);
             const float4 m0 = dat_ld4_hint(a.mom + e0, pol_first), m1 = dat_ld4_hint(a.mom + e0 + 4, pol_first);
             t0.x = __fmaf_rn(na, m0.x, t0.x); t0.y = __fmaf_rn(na, m0.y, t0.y); t0.z = __fmaf_rn(na, m0.z, t0.z); t0.w = __fmaf_rn(na, m0.w, t0.w);
@@ -430,7 +521,7 @@ __device__ __forceinline__ void p_part_update(const PArgs &a, const PipePart &pt
     }
 }
 
-template <bool RNG16, int MODE>
+template <bool RNG16, int MODE, int OPT>
 __global__ void __launch_bounds__(DAT_P_THREADS, DAT_P_MINB)
 k_step_pipelined(const __grid_constant__ PArgs a)
 {
@@ -480,9 +571,9 @@ k_step_pipelined(const __grid_constant__ PArgs a)
         }
     }
     __syncthreads();                               // (A)
-    if (s_ctl[0]) p_norm_finish(a, pn, s_norm);
+    if (s_ctl[0]) p_norm_finish<MODE>(a, pn, s_norm);
     const bool alive = (s_ctl[1] != 0);
-    if (alive && pq.layer >= 0) p_part_quant<RNG16, MODE>(a, pq, s_unit);
+    if (alive && pq.layer >= 0) p_part_quant<RNG16, MODE, OPT>(a, pq, s_unit);
     __syncthreads();
     if (threadIdx.x == 0) {
         bool q_last = false, u_go = alive;
@@ -493,7 +584,7 @@ k_step_pipelined(const __grid_constant__ PArgs a)
     }
     __syncthreads();                               // (B)
     if (s_ctl[2]) p_quant_finish(a, pq, s_unit);
-    if (s_ctl[3] && pu.layer >= 0) p_part_update(a, pu);
+    if (s_ctl[3] && pu.layer >= 0) p_part_update<OPT>(a, pu);
 }
 
 // ---- host: the item list -----------------------------------------------------------------------------
@@ -564,7 +655,7 @@ int dat_pipe_build(dat_plan_t *plan)
         slot = 0;
         for (int k = 0; k < h; ++k) {
             const int l = order[k];
-            slot = std::max(slot, done_q[l] + DAT_P_LAG + 1);
+            slot = std::max(slot, done_q[l] + DAT_P_LAG_U + 1);
             for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { at(slot).u = part(l, t); ++slot; }
         }
         g->n_items = (int64_t)items.size();
@@ -603,24 +694,22 @@ cudaError_t dat_pipe_reset(dat_plan_t *plan, cudaStream_t s)
     return cudaMemsetAsync(g->d_sync, 0, g->sync_bytes, s);
 }
 
-extern "C" int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
-                                  uint64_t seed, uint64_t step, const dat_hparams_t *hp,
-                                  int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
+// One launch of the step.  lamb == nullptr: the momentum direction with hp; else Algorithm A2 with *lamb.
+static int p_launch(dat_plan_t *plan, float *theta, float *mom, float *var, const float *const *grads,
+                    uint64_t seed, uint64_t step, const dat_hparams_t *hp, const LambConst *lamb, float lr, float c_l, float c_u,
+                    int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
 {
-    int rc = dat_check_plan(plan);
-    if (rc != DAT_OK) return rc;
-    if (!theta || !mom || !hp) return DAT_ERR_ARG;
-    if (plan->bits != 32 && plan->scale_mode != DAT_SCALE_SHARED_MAX) return DAT_ERR_UNSUPPORTED;
     if (step >> 32) return DAT_ERR_ARG;
-    if (!dat_aligned16(theta) || !dat_aligned16(mom) || (code_sum_out && !dat_aligned16(code_sum_out)) ||
+    if (!dat_aligned16(theta) || !dat_aligned16(mom) || (var && !dat_aligned16(var)) || (code_sum_out && !dat_aligned16(code_sum_out)) ||
         (layer_norms_out && !dat_aligned16(layer_norms_out)) || (scales_out && !dat_aligned16(scales_out)))
         return DAT_ERR_ALIGN;
     PArgs a;
-    rc = dat_check_grads(plan, grads, &a.gp);
+    int rc = dat_check_grads(plan, grads, &a.gp);
     if (rc != DAT_OK) return rc;
     PipeSchedule *g = plan->pipe;
     if (!g || !g->mem) return DAT_ERR_ARG;
     const bool identity = (plan->bits == 32);
+    const bool per_worker = !identity && plan->scale_mode == DAT_SCALE_PER_WORKER;
     const size_t h = (size_t)plan->h;
     a.keys = dat_make_keys(seed, step);
     a.items = g->d_items;
@@ -628,6 +717,9 @@ extern "C" int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, co
     a.tile_base = g->d_tile_base;
     a.theta = theta;
     a.mom = mom;
+    a.var = var;
+    if (lamb) a.lamb = *lamb;
+    else a.lamb = LambConst{0.0f, 0.0f, 0.0f, 0.0f, 1.0f, 1.0f, 1.0f, 0.0f};
     a.partN = g->d_partN;
     a.partQ = g->d_partQ;
     a.ticket = g->d_sync;
@@ -644,16 +736,16 @@ extern "C" int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, co
     a.step_a = plan->d_step_a;
     a.norms_out = layer_norms_out;
     a.scales_out = identity ? nullptr : scales_out;
-    a.code_sum = identity ? nullptr : code_sum_out;
+    a.code_sum = (identity || per_worker) ? nullptr : code_sum_out;
     a.wait_cycles = g->wait_cycles;
     a.S_f = (float)plan->S;
     a.SM_f = (float)((uint64_t)plan->S * (uint64_t)plan->M);
     a.M_f = (float)plan->M;
-    a.mu = hp->momentum;
-    a.wd = hp->weight_decay;
-    a.lr = hp->lr;
-    a.c_l = hp->c_l;
-    a.c_u = hp->c_u;
+    a.mu = hp ? hp->momentum : 0.0f;
+    a.wd = hp ? hp->weight_decay : 0.0f;
+    a.lr = lr;
+    a.c_l = c_l;
+    a.c_u = c_u;
     if (++g->epoch == 0u) ++g->epoch;              // 0 is what the words hold before the first call
     a.epoch = g->epoch;
     a.n_items = (uint32_t)g->n_items;
@@ -663,11 +755,42 @@ extern "C" int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, co
     a.n_tiles = g->n_tiles;
     cudaStream_t s = (cudaStream_t)stream;
     const unsigned grid = (unsigned)g->n_items;
-    if (identity) k_step_pipelined<true, P_MODE_IDENTITY><<<grid, DAT_P_THREADS, 0, s>>>(a);
-    else if (plan->rng_bits == 16) k_step_pipelined<true, P_MODE_SHARED><<<grid, DAT_P_THREADS, 0, s>>>(a);
-    else k_step_pipelined<false, P_MODE_SHARED><<<grid, DAT_P_THREADS, 0, s>>>(a);
+    const bool rng16 = (plan->rng_bits == 16);
+#define P_GO(R, MODE, OPT) k_step_pipelined<R, MODE, OPT><<<grid, DAT_P_THREADS, 0, s>>>(a)
+#define P_GO_OPT(R, MODE) do { if (lamb) P_GO(R, MODE, P_OPT_LAMB); else P_GO(R, MODE, P_OPT_MOMENTUM); } while (0)
+    if (identity) P_GO_OPT(true, P_MODE_IDENTITY);
+    else if (per_worker && rng16) P_GO_OPT(true, P_MODE_PER_WORKER);
+    else if (per_worker) P_GO_OPT(false, P_MODE_PER_WORKER);
+    else if (rng16) P_GO_OPT(true, P_MODE_SHARED);
+    else P_GO_OPT(false, P_MODE_SHARED);
+#undef P_GO_OPT
+#undef P_GO
     DAT_LAUNCHED(plan);
     return DAT_OK;
+}
+
+extern "C" int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                                  uint64_t seed, uint64_t step, const dat_hparams_t *hp,
+                                  int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (!theta || !mom || !hp) return DAT_ERR_ARG;
+    return p_launch(plan, theta, mom, nullptr, grads, seed, step, hp, nullptr, hp->lr, hp->c_l, hp->c_u, code_sum_out,
+                    layer_norms_out, scales_out, stream);
+}
+
+extern "C" int dat_step_lamb(dat_plan_t *plan, float *theta, float *mom, float *var, const float *const *grads,
+                             uint64_t seed, uint64_t step, const dat_lamb_hparams_t *hp, int64_t t,
+                             int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (!theta || !mom || !var || !hp || t < 1) return DAT_ERR_ARG;
+    if (!(hp->beta1 > 0.0f && hp->beta1 < 1.0f && hp->beta2 > 0.0f && hp->beta2 < 1.0f)) return DAT_ERR_ARG;
+    const LambConst c = dat_lamb_const(hp, t);
+    return p_launch(plan, theta, mom, var, grads, seed, step, nullptr, &c, hp->lr, hp->c_l, hp->c_u, code_sum_out,
+                    layer_norms_out, scales_out, stream);
 }
 
 // Test hook (see dat.h): a short wait limit, and a layer whose norm never completes in the next call.

@@ -1,4 +1,5 @@
 // Plan object, argument validation, status word and the host-buffer entry point.
+#include <cmath>
 #include <new>
 
 #include "dat_internal.cuh"
@@ -34,6 +35,20 @@ int dat_check_grads(const dat_plan_t *plan, const float *const *grads, GradPtrs 
     }
     for (int i = plan->M; i < DAT_MAX_WORKERS; ++i) out->p[i] = nullptr;
     return DAT_OK;
+}
+
+LambConst dat_lamb_const(const dat_lamb_hparams_t *hp, int64_t t)
+{
+    LambConst c;
+    c.beta1 = hp->beta1;
+    c.beta2 = hp->beta2;
+    c.om1 = 1.0f - hp->beta1;
+    c.om2 = 1.0f - hp->beta2;
+    c.bc1 = (float)(1.0 - pow((double)hp->beta1, (double)t));      // 1 - beta^t in double, rounded once
+    c.bc2 = (float)(1.0 - pow((double)hp->beta2, (double)t));
+    c.zeta = hp->zeta;
+    c.wd = hp->weight_decay;
+    return c;
 }
 
 PhiloxKeys dat_make_keys(uint64_t seed, uint64_t step)

@@ -631,17 +631,6 @@ extern "C" int dat_lalr_step(dat_plan_t *plan, float *theta, float *mom, const f
 // of theta^2 and u^2.  Finalize as for LALR.  Pass 2 forms u again from the stored moments (the same
 // fp32 operations give the same bits) and moves theta.
 // ------------------------------------------------------------------------------------------
-struct LambConst {
-    float beta1, beta2, om1, om2, bc1, bc2, zeta, wd;
-};
-
-__device__ __forceinline__ float dat_lamb_direction(const LambConst &c, float m_new, float v_new, float theta)
-{
-    const float m_hat = m_new / c.bc1;
-    const float v_hat = v_new / c.bc2;
-    return __fmaf_rn(c.wd, theta, m_hat / (sqrtf(v_hat) + c.zeta));
-}
-
 __global__ void __launch_bounds__(DAT_THREADS)
 k_lamb_pass1(const float *__restrict__ theta, float *__restrict__ mom, float *__restrict__ var,
              const float *__restrict__ g_hat, const int64_t *__restrict__ off,
@@ -717,15 +706,7 @@ extern "C" int dat_lamb_step(dat_plan_t *plan, float *theta, float *mom, float *
         return DAT_ERR_ALIGN;
     cudaStream_t s = (cudaStream_t)stream;
     const int h = (int)plan->h;
-    LambConst c;
-    c.beta1 = hp->beta1;
-    c.beta2 = hp->beta2;
-    c.om1 = 1.0f - hp->beta1;
-    c.om2 = 1.0f - hp->beta2;
-    c.bc1 = (float)(1.0 - pow((double)hp->beta1, (double)t));      // 1 - beta^t in double, rounded once
-    c.bc2 = (float)(1.0 - pow((double)hp->beta2, (double)t));
-    c.zeta = hp->zeta;
-    c.wd = hp->weight_decay;
+    const LambConst c = dat_lamb_const(hp, t);
     k_lamb_pass1<<<(unsigned)plan->n_tiles, DAT_THREADS, 0, s>>>(theta, mom, var, g_hat, plan->d_offsets,
                                                                  plan->d_tile_base, h, c, plan->d_partials);
     DAT_LAUNCHED(plan);

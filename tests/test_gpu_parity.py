@@ -154,9 +154,20 @@ def _check_unfused_per_worker(api, oracle, offs, grads, theta, mom, bits, hp, se
         with pytest.raises(api.DatError) as e:
             api.dat_aggregate(P.plan, lv, sg, sc, cs, gh)
         assert e.value.code == api.DAT_ERR_ARG
-        with pytest.raises(api.DatError) as e:
-            api.dat_step(P.plan, th_d, mo_d, g_dev, seed, step, hp)
-        assert e.value.code == api.DAT_ERR_UNSUPPORTED
+        # the same in one call: dat_step on a per-worker plan (M*h norms out, no integer code sums)
+        th_s, mo_s = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        sc_s = torch.zeros(M * h, dtype=torch.float32, device="cuda")
+        norms = torch.zeros(2 * h, dtype=torch.float32, device="cuda")
+        api.dat_step(P.plan, th_s, mo_s, g_dev, seed, step, hp, None, norms, sc_s)
+        torch.cuda.synchronize()
+        assert P.status() == 0
+        sc_step = np_of(sc_s).reshape(M, h)
+        assert ulp_diff(sc_step, sc_ref).max() <= 1
+        ref = oracle.step(offs, theta, mom, grads, bits, seed, step, *hp, scale_mode=oracle.SCALE_PER_WORKER,
+                          scales_in=sc_step, rng_bits=rng_bits)
+        assert np.array_equal(np_of(mo_s).view(np.uint32), ref["mom"].view(np.uint32))
+        assert ulp_diff(np_of(norms).reshape(-1, 2), ref["layer_norms"]).max() <= 1
+        assert_close_per_layer(np_of(th_s), ref["theta"], offs, "theta (dat_step, per-worker scales)")
 
 
 @pytest.mark.parametrize("bits", [1, 4, 8, 16])
@@ -228,6 +239,49 @@ def test_lamb_step_parity_three_steps(api, oracle):
         assert P.status() == 0
         with pytest.raises(api.DatError) as e:
             api.dat_lamb_step(P.plan, th_d, mo_d, va_d, th_d, LAMB_HP, 0)
+        assert e.value.code == api.DAT_ERR_ARG
+
+
+@pytest.mark.parametrize("mode", ["shared", "per_worker", "b32"])
+def test_step_lamb_parity_three_steps(api, oracle, mode):
+    """dat_step_lamb: Steps 7 and 9 followed by Algorithm A2 and Eq. upth in the one launch, over t = 1, 2, 3
+    with fresh gradients and an advancing step counter.  The oracle gets the GPU's quantizer norms and the
+    GPU's theta history; then g_hat is its own, and m', v' must agree bit for bit, theta' within the tolerance."""
+    M, bits = 4, (32 if mode == "b32" else 8)
+    sm = oracle.SCALE_PER_WORKER if mode == "per_worker" else oracle.SCALE_SHARED_MAX
+    offs, _, theta, _ = _random_problem(93, SIZES_RAGGED + [50000], M)
+    d, h = int(offs[-1]), len(offs) - 1
+    theta[int(offs[4]):int(offs[5])] = 0.0                     # an all-zero parameter tensor
+    mom, var = np.zeros(d, dtype=np.float32), np.zeros(d, dtype=np.float32)
+    with GpuPlan(api, offs, M, bits, 16, scale_mode=api.DAT_SCALE_PER_WORKER if mode == "per_worker" else 0) as P:
+        th_d, mo_d, va_d = (torch.from_numpy(x.copy()).cuda() for x in (theta, mom, var))
+        norms = torch.zeros(2 * h, dtype=torch.float32, device="cuda")
+        sc = torch.zeros(P.num_scales, dtype=torch.float32, device="cuda")
+        mo_ref, va_ref = mom, var
+        for t in (1, 2, 3):
+            _, grads, _, _ = _random_problem(200 + t, SIZES_RAGGED + [50000], M)
+            if t == 2:
+                for g in grads:
+                    g[int(offs[10]):int(offs[11])] = 0.0       # a layer with zero gradient
+            th_in = np_of(th_d).copy()
+            api.dat_step_lamb(P.plan, th_d, mo_d, va_d, [torch.from_numpy(g).cuda() for g in grads], 7, t, LAMB_HP, t, None, norms, sc)
+            torch.cuda.synchronize()
+            assert P.status() == 0
+            if bits == 32:
+                gh = oracle.average(offs, grads)
+            else:
+                sc_gpu = np_of(sc)
+                sc_ref = oracle.scales(oracle.worker_norms(offs, grads), sm)
+                assert ulp_diff(sc_gpu.reshape(sc_ref.shape), sc_ref).max() <= 1
+                level, neg = oracle.quantize(offs, grads, bits, 7, t, sc_gpu, sm, rng_bits=16)
+                _, gh = oracle.aggregate(offs, level, neg, sc_gpu, bits, sm)
+            th_ref, mo_ref, va_ref, n_ref = oracle.lamb(offs, th_in, mo_ref, va_ref, gh, t, *LAMB_HP)
+            assert np.array_equal(np_of(mo_d).view(np.uint32), mo_ref.view(np.uint32))
+            assert np.array_equal(np_of(va_d).view(np.uint32), va_ref.view(np.uint32))
+            assert ulp_diff(np_of(norms).reshape(-1, 2), n_ref).max() <= 1
+            assert_close_per_layer(np_of(th_d), th_ref, offs, "theta (dat_step_lamb, t = %d)" % t)
+        with pytest.raises(api.DatError) as e:
+            api.dat_step_lamb(P.plan, th_d, mo_d, va_d, [torch.from_numpy(g).cuda() for g in grads], 7, 4, LAMB_HP, 0)
         assert e.value.code == api.DAT_ERR_ARG
 
 
