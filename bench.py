@@ -260,7 +260,7 @@ def run_gpu(args):
     theta, mom = synth.make_params(cfg, device=dev)
     grads = synth.make_grads(cfg, 0, device=dev)
     hp = (cfg.lr, cfg.momentum, cfg.weight_decay, cfg.c_l, cfg.c_u)
-    variant = args.path[len("unfused_"):] if args.path.startswith("unfused_") else ""
+    variant = args.path.split("_", 1)[1] if args.path.startswith(("unfused_", "step_")) else ""
     plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits, rng_bits=cfg.rng_bits,
                                scale_mode=api.DAT_SCALE_PER_WORKER if variant == "per_worker" else api.DAT_SCALE_SHARED_MAX)
     stream = torch.cuda.current_stream()
@@ -291,9 +291,9 @@ def run_gpu(args):
             s_levels = torch.empty(lb, dtype=torch.uint8, device=dev)
             s_signs = torch.empty(sb, dtype=torch.uint8, device=dev)
             s_scales = torch.empty(cfg.h, dtype=torch.float32, device=dev)
-        if variant == "lamb":           # Algorithm A2: second moment, the paper's ImageNet hyper-parameters
-            var = torch.zeros(cfg.d, dtype=torch.float32, device=dev)
-            lamb_hp = (cfg.lr, 0.9, 0.999, 1e-6, 1e-4, cfg.c_l, cfg.c_u)
+    if variant == "lamb":               # Algorithm A2: second moment, the paper's ImageNet hyper-parameters
+        var = torch.zeros(cfg.d, dtype=torch.float32, device=dev)
+        lamb_hp = (cfg.lr, 0.9, 0.999, 1e-6, 1e-4, cfg.c_l, cfg.c_u)
 
     def one_step(step_index):
         if unfused:
@@ -307,6 +307,8 @@ def run_gpu(args):
                 api.dat_lalr_step(plan, theta, mom, u_ghat, hp)
         elif args.path == "passes":
             api.dat_step_passes(plan, theta, mom, grads, cfg.seed, step_index, hp)
+        elif args.path == "step_lamb":
+            api.dat_step_lamb(plan, theta, mom, var, grads, cfg.seed, step_index, lamb_hp, step_index + 1)
         elif args.path == "pipelined":
             api.dat_step_pipelined(plan, theta, mom, grads, cfg.seed, step_index, hp)
         else:
@@ -353,7 +355,7 @@ def run_gpu(args):
 
     # ---- end to end through the host-buffer entry point (H2D + step + D2H inside the timed region)
     e2e = None
-    if not args.no_e2e and not unfused:
+    if not args.no_e2e and not unfused and not variant:
         th_h = theta.detach().cpu().pin_memory()
         mo_h = mom.detach().cpu().pin_memory()
         g_h = [g.detach().cpu().pin_memory() for g in grads]
@@ -402,6 +404,8 @@ def run_gpu(args):
                 algo_bytes += 12 * cfg.d
         else:
             algo_bytes = (4 * cfg.M + 16) * cfg.d
+            if variant == "lamb":       # v read and written in the Q part, read again in the U part
+                algo_bytes += 8 * cfg.d
         achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
         per_step = launches // K
         traffic, traffic_src = ncu_traffic(args.path, cfg)
@@ -442,8 +446,9 @@ def main():
                     help="override the resolution of the quantizer's uniform number (0: the config's)")
     ap.add_argument("--impl", default="dat", choices=["dat", "reference"])
     ap.add_argument("--path", default="step",
-                    choices=["step", "pipelined", "passes", "unfused", "unfused_per_worker", "unfused_two_sided", "unfused_lamb"],
+                    choices=["step", "step_per_worker", "step_lamb", "pipelined", "passes", "unfused", "unfused_per_worker", "unfused_two_sided", "unfused_lamb"],
                     help="step: dat_step (the headline: one pipelined launch); pipelined: the same by its own name; "
+                         "step_per_worker: dat_step on a plan with one quantizer norm per worker; step_lamb: dat_step_lamb; "
                          "passes: dat_step_passes, three streaming passes; unfused: dat_quantize + dat_aggregate + dat_lalr_step; "
                          "unfused_per_worker: the same with one quantizer norm per worker; unfused_two_sided: with "
                          "dat_requantize after the aggregation; unfused_lamb: with dat_lamb_step as the update")
