@@ -434,6 +434,81 @@ def run_gpu(args):
     return 0
 
 
+def run_sharded(args):
+    """The sharded step (paper_2206_06257_b200/sharded.py): total work fixed, divided over the ranks."""
+    import torch
+    import torch.distributed as dist
+    from paper_2206_06257_b200 import api, synth
+    from paper_2206_06257_b200.sharded import CudaOps, ShardedStep
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for this path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    cfg = synth.config(args.config)
+    if args.bits:
+        cfg.bits = args.bits
+    if args.rng_bits:
+        cfg.rng_bits = args.rng_bits
+    if cfg.M % world:
+        raise SystemExit("--sharded needs the workload's %d workers to divide over %d ranks" % (cfg.M, world))
+    M_loc = cfg.M // world
+    theta, mom = synth.make_params(cfg, device=dev)
+    grads = synth.make_grads(cfg, 0, device=dev)[rank * M_loc:(rank + 1) * M_loc]      # this rank's workers
+    hp = (cfg.lr, cfg.momentum, cfg.weight_decay, cfg.c_l, cfg.c_u)
+    ops = CudaOps(api, cfg.offsets, cfg.M, M_loc, rank, world, cfg.bits, cfg.rng_bits)
+    st = ShardedStep(ops, cfg.offsets, cfg.M, rank, world)
+    mom_own = mom[st.own.a8:st.own.b].clone()
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    step_no = 0
+    for _ in range(max(args.warmup, 3)):
+        st.step(theta, mom_own, grads, cfg.seed, step_no, hp)
+        step_no += 1
+    K = args.steps
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    e0.record(stream)
+    for _ in range(K):
+        st.step(theta, mom_own, grads, cfg.seed, step_no, hp)
+        step_no += 1
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    finite = bool(torch.isfinite(theta).all().item())
+    own_bytes = sum(ops.plane_bytes(rg)[0] + ops.plane_bytes(rg)[1] for q, rg in enumerate(st.ranges) if q != rank) * M_loc
+    ops.close()
+    if rank == 0:
+        peak, peak_src = measured_peaks()
+        value = cfg.M * cfg.d * K / (ms * 1e-3)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": dict(workload_config(cfg, "inputs larger than L2, no flush"), parallelism="sharded: %d worker(s) and one layer range per rank" % M_loc,
+                           path="sharded (dat_worker_norms, dat_quantize, plane exchange, dat_aggregate, dat_lalr_step, theta broadcast)"),
+            "roofline": None, "cpu_baseline": None, "e2e": None,
+            "sent_plane_bytes_per_rank_and_step": int(own_bytes), "clocks": clocks, "outputs_finite": finite,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -452,12 +527,17 @@ def main():
                          "passes: dat_step_passes, three streaming passes; unfused: dat_quantize + dat_aggregate + dat_lalr_step; "
                          "unfused_per_worker: the same with one quantizer norm per worker; unfused_two_sided: with "
                          "dat_requantize after the aggregation; unfused_lamb: with dat_lamb_step as the update")
+    ap.add_argument("--sharded", action="store_true",
+                    help="the step sharded over the --gpus ranks (layer ranges owned by ranks, planes exchanged, "
+                         "theta broadcast) instead of independent replicas; the M workers are divided over the ranks")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.sharded:
+        return run_sharded(args)
     return run_gpu(args)
 
 

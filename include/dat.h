@@ -132,6 +132,14 @@ enum {
 int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64_t *layer_offsets,
                     int num_workers, int bits, int scale_mode, int rng_bits);
 
+/* dat_plan_set_origin -- for a plan that covers a SLICE of a larger problem (a contiguous range of layers
+ * and a subset of the workers, as one rank of a sharded step holds them): the global index of the plan's
+ * element 0 (a multiple of 8) and of its worker 0.  dat_quantize and dat_requantize then draw exactly the
+ * random numbers the unsliced problem would draw for those elements and workers (the paper's Q is keyed on
+ * (seed, step, worker, element) here).  dat_step and dat_step_passes answer DAT_ERR_UNSUPPORTED for a plan
+ * with a non-zero origin.  Errors: ARG. */
+int dat_plan_set_origin(dat_plan_t *plan, int64_t elem_base, int64_t worker_base);
+
 /* Frees the plan and its workspace (synchronises the device).  NULL is accepted. */
 int dat_plan_destroy(dat_plan_t *plan);
 
@@ -169,6 +177,14 @@ int dat_plan_sizes(const dat_plan_t *plan, int64_t *level_bytes_per_worker,
 int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_t seed, uint64_t step,
                  uint8_t *levels, uint8_t *signs, float *scales, const float *scales_in,
                  void *stream);
+
+/* dat_worker_norms -- the norms of Eq. rand_q by themselves: nu_{i,l} = ||g_l^(i)||_2 for every worker and
+ * layer (fp64 sums of exact squares, one rounding), without drawing any level.  A sharded step needs them
+ * before it can agree on the shared norm max_i nu_{i,l} across ranks.
+ *   grads      host array of M device pointers, fp32[d] each, read-only.
+ *   norms_out  device fp32[M*h], written: nu_{i,l} at i*h + l.
+ * Errors: ARG, ALIGN, CUDA. */
+int dat_worker_norms(dat_plan_t *plan, const float *const *grads, float *norms_out, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * dat_aggregate -- Algorithm A1 Step 9, Eq. grad_agg, on the packed messages:

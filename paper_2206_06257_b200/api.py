@@ -30,7 +30,7 @@ DAT_STATIC_MAX_LAYERS, DAT_STATIC_MAX_TILES = 4096, 32768
 DAT_STATUS_NONFINITE, DAT_STATUS_TIMEOUT, DAT_STATUS_BOUNDS = 1, 2, 4
 
 # every symbol include/dat.h declares
-EXPORTS = ["dat_plan_create", "dat_plan_destroy", "dat_plan_sizes", "dat_quantize", "dat_aggregate", "dat_requantize",
+EXPORTS = ["dat_plan_create", "dat_plan_set_origin", "dat_plan_destroy", "dat_plan_sizes", "dat_worker_norms", "dat_quantize", "dat_aggregate", "dat_requantize",
            "dat_average", "dat_lalr_step", "dat_lamb_step", "dat_lalr_step_static", "dat_step", "dat_step_lamb", "dat_step_passes", "dat_step_pipelined", "dat_plan_test_stall", "dat_step_host", "dat_get_status",
            "dat_plan_launch_count", "dat_strerror", "dat_last_cuda_error"]
 
@@ -48,6 +48,8 @@ class dat_lamb_hparams_t(C.Structure):
 _p, _i64, _u64, _int = C.c_void_p, C.c_int64, C.c_uint64, C.c_int
 _lib.dat_plan_create.argtypes = [C.POINTER(_p), _i64, _p, _int, _int, _int, _int]
 _lib.dat_plan_destroy.argtypes = [_p]
+_lib.dat_plan_set_origin.argtypes = [_p, _i64, _i64]
+_lib.dat_worker_norms.argtypes = [_p, _p, _p, _p]
 _lib.dat_plan_sizes.argtypes = [_p, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]
 _lib.dat_quantize.argtypes = [_p, _p, _u64, _u64, _p, _p, _p, _p, _p]
 _lib.dat_aggregate.argtypes = [_p, _p, _p, _p, _p, _p, _p]
@@ -127,6 +129,14 @@ def dat_plan_create(layer_offsets, num_workers, bits, scale_mode=DAT_SCALE_SHARE
     _ok(_lib.dat_plan_create(C.byref(out), offs.size - 1, _ptr(offs), int(num_workers), int(bits),
                              int(scale_mode), int(rng_bits)), "dat_plan_create")
     return out.value
+
+
+def dat_plan_set_origin(plan, elem_base, worker_base):
+    _ok(_lib.dat_plan_set_origin(_p(plan), int(elem_base), int(worker_base)), "dat_plan_set_origin")
+
+
+def dat_worker_norms(plan, grads, norms_out, stream=None):
+    _ok(_lib.dat_worker_norms(_p(plan), _ptr_array(grads), _ptr(norms_out), _stream(stream)), "dat_worker_norms")
 
 
 def dat_plan_destroy(plan):

@@ -36,6 +36,8 @@ struct dat_plan {
     int device = 0;
     int64_t h = 0, d = 0;
     int M = 0, bits = 0, scale_mode = 0, rng_bits = 16;
+    int64_t elem_base = 0;             // global index of the plan's element 0 and of its worker 0 in the random
+    uint32_t worker_base = 0;          // streams (dat_plan_set_origin: a plan that covers a slice of a larger problem)
     uint32_t S = 0;
     std::vector<int64_t> offsets;      // host copy, h+1
     std::vector<int64_t> tile_base;    // host copy, h+1: first per-layer tile of each layer

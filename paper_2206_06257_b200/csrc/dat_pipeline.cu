@@ -700,6 +700,7 @@ static int p_launch(dat_plan_t *plan, float *theta, float *mom, float *var, cons
                     int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
 {
     if (step >> 32) return DAT_ERR_ARG;
+    if (plan->elem_base || plan->worker_base) return DAT_ERR_UNSUPPORTED;     // a slice of a larger problem: separate calls only
     if (!dat_aligned16(theta) || !dat_aligned16(mom) || (var && !dat_aligned16(var)) || (code_sum_out && !dat_aligned16(code_sum_out)) ||
         (layer_norms_out && !dat_aligned16(layer_norms_out)) || (scales_out && !dat_aligned16(scales_out)))
         return DAT_ERR_ALIGN;

@@ -152,6 +152,14 @@ extern "C" int dat_plan_create(dat_plan_t **out, int64_t num_layers, const int64
     return DAT_OK;
 }
 
+extern "C" int dat_plan_set_origin(dat_plan_t *plan, int64_t elem_base, int64_t worker_base)
+{
+    if (!plan || elem_base < 0 || (elem_base & 7) || worker_base < 0 || worker_base + plan->M > ((int64_t)1 << 32)) return DAT_ERR_ARG;
+    plan->elem_base = elem_base;
+    plan->worker_base = (uint32_t)worker_base;
+    return DAT_OK;
+}
+
 extern "C" int dat_plan_destroy(dat_plan_t *plan)
 {
     if (!plan) return DAT_OK;

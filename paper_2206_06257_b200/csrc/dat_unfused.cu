@@ -100,7 +100,7 @@ template <int BITS>
 __global__ void __launch_bounds__(DAT_THREADS)
 k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h, int64_t d,
            const float *__restrict__ qmul_all, uint8_t *__restrict__ levels, uint8_t *__restrict__ signs,
-           int64_t level_bytes, int64_t sign_bytes, bool rng16, bool per_worker, uint32_t stream_base)
+           int64_t level_bytes, int64_t sign_bytes, bool rng16, bool per_worker, uint32_t stream_base, int64_t elem_base)
 {
     constexpr int GROUPS = DAT_TILE / 4;                     // aligned groups per tile
     constexpr int LEVEL_TILE_BYTES = DAT_TILE * BITS / 8;
@@ -132,7 +132,7 @@ k_quantize(GradPtrs gp, PhiloxKeys keys, const int64_t *__restrict__ off, int h,
         const int64_t e0 = e_tile + 4 * (int64_t)v;
         const float *gv = gall[it];
         float u1[4];
-        dat_u1x4((uint64_t)e0, stream_base + (uint32_t)worker, keys, rng16, u1);     // the worker's random stream
+        dat_u1x4((uint64_t)(e0 + elem_base), stream_base + (uint32_t)worker, keys, rng16, u1);     // the worker's random stream
         uint32_t lev[4], neg = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -220,7 +220,7 @@ extern "C" int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_
     dim3 grid((unsigned)flat_tiles, (unsigned)plan->M);
 #define DAT_Q(B)                                                                                           \
     k_quantize<B><<<grid, DAT_THREADS, 0, s>>>(gp, keys, plan->d_offsets, h, plan->d, plan->d_qmul, levels, \
-                                               signs, plan->level_bytes, plan->sign_bytes, plan->rng_bits == 16, per_worker, 0u)
+                                               signs, plan->level_bytes, plan->sign_bytes, plan->rng_bits == 16, per_worker, plan->worker_base, plan->elem_base)
     switch (plan->bits) {
     case 1: DAT_Q(1); break;
     case 2: DAT_Q(2); break;
@@ -230,6 +230,28 @@ extern "C" int dat_quantize(dat_plan_t *plan, const float *const *grads, uint64_
     }
 #undef DAT_Q
     DAT_LAUNCHED(plan);
+    return DAT_OK;
+}
+
+// S1 by itself: the quantizer norm of every (worker, layer), nu_{i,l} = ||g_l^(i)||_2 (Eq. rand_q).
+extern "C" int dat_worker_norms(dat_plan_t *plan, const float *const *grads, float *norms_out, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (!norms_out) return DAT_ERR_ARG;
+    if (!dat_aligned16(norms_out)) return DAT_ERR_ALIGN;
+    GradPtrs gp;
+    rc = dat_check_grads(plan, grads, &gp);
+    if (rc != DAT_OK) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int h = (int)plan->h;
+    dim3 grid((unsigned)plan->n_tiles, (unsigned)plan->M);
+    k_sumsq_partial<<<grid, DAT_THREADS, 0, s>>>(gp, plan->d_offsets, plan->d_tile_base, h, plan->M, plan->d_partials);
+    DAT_LAUNCHED(plan);
+    k_scales_finalize<<<h, DAT_THREADS, 0, s>>>(plan->d_tile_base, h, plan->M, (float)plan->S, plan->d_partials,
+                                                plan->d_worker_norms, plan->d_scales, plan->d_qmul, plan->d_status, false);
+    DAT_LAUNCHED(plan);
+    DAT_CUDA(plan, cudaMemcpyAsync(norms_out, plan->d_worker_norms, (size_t)plan->M * h * 4, cudaMemcpyDeviceToDevice, s));
     return DAT_OK;
 }
 
@@ -425,7 +447,7 @@ extern "C" int dat_requantize(dat_plan_t *plan, float *g_hat, uint64_t seed, uin
     do {                                                                                                            \
         k_quantize<B><<<qgrid, DAT_THREADS, 0, s>>>(gp, keys, plan->d_offsets, h, plan->d, plan->d_qmul, levels,    \
                                                     signs, plan->level_bytes, plan->sign_bytes,                     \
-                                                    plan->rng_bits == 16, false, (uint32_t)plan->M);                \
+                                                    plan->rng_bits == 16, false, plan->worker_base + (uint32_t)plan->M, plan->elem_base); \
         DAT_LAUNCHED(plan);                                                                                         \
         k_aggregate<B><<<agrid, DAT_THREADS, 0, s>>>(levels, signs, plan->level_bytes, plan->sign_bytes, 1,          \
                                                      plan->d_offsets, h, plan->d, plan->d_dq, nullptr, g_hat);      \
@@ -873,7 +895,7 @@ extern "C" int dat_step_passes(dat_plan_t *plan, float *theta, float *mom, const
     int rc = dat_check_plan(plan);
     if (rc != DAT_OK) return rc;
     if (!theta || !mom || !hp) return DAT_ERR_ARG;
-    if (plan->bits == 32 || plan->scale_mode != DAT_SCALE_SHARED_MAX) return DAT_ERR_UNSUPPORTED;
+    if (plan->bits == 32 || plan->scale_mode != DAT_SCALE_SHARED_MAX || plan->elem_base || plan->worker_base) return DAT_ERR_UNSUPPORTED;
     if (step >> 32) return DAT_ERR_ARG;
     if (!dat_aligned16(theta) || !dat_aligned16(mom) || (code_sum_out && !dat_aligned16(code_sum_out)) ||
         (layer_norms_out && !dat_aligned16(layer_norms_out)) || (scales_out && !dat_aligned16(scales_out)))
