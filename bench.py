@@ -291,6 +291,8 @@ def run_gpu(args):
             s_levels = torch.empty(lb, dtype=torch.uint8, device=dev)
             s_signs = torch.empty(sb, dtype=torch.uint8, device=dev)
             s_scales = torch.empty(cfg.h, dtype=torch.float32, device=dev)
+    if args.path == "step_two_sided":   # workspace for the aggregate / the receiver's value (Algorithm A1 Step 10)
+        ts_ghat = torch.empty(cfg.d, dtype=torch.float32, device=dev)
     if variant == "lamb":               # Algorithm A2: second moment, the paper's ImageNet hyper-parameters
         var = torch.zeros(cfg.d, dtype=torch.float32, device=dev)
         lamb_hp = (cfg.lr, 0.9, 0.999, 1e-6, 1e-4, cfg.c_l, cfg.c_u)
@@ -309,6 +311,8 @@ def run_gpu(args):
             api.dat_step_passes(plan, theta, mom, grads, cfg.seed, step_index, hp)
         elif args.path == "step_lamb":
             api.dat_step_lamb(plan, theta, mom, var, grads, cfg.seed, step_index, lamb_hp, step_index + 1)
+        elif args.path == "step_two_sided":
+            api.dat_step_two_sided(plan, theta, mom, grads, cfg.seed, step_index, hp, ts_ghat)
         elif args.path == "pipelined":
             api.dat_step_pipelined(plan, theta, mom, grads, cfg.seed, step_index, hp)
         else:
@@ -406,7 +410,12 @@ def run_gpu(args):
             algo_bytes = (4 * cfg.M + 16) * cfg.d
             if variant == "lamb":       # v read and written in the Q part, read again in the U part
                 algo_bytes += 8 * cfg.d
+            if variant == "two_sided":  # g_hat written once (the receiver's value is the call's output)
+                algo_bytes += 4 * cfg.d
         achieved = algo_bytes / (kernel_ms * 1e-3) / 1e9
+        # the quantizer norm forces a second read of a layer whose M gradients (4 M n_l bytes) exceed the L2 cache
+        sizes = np.diff(np.asarray(cfg.offsets, dtype=np.int64))
+        second_read = int(4 * cfg.M * sizes[4 * cfg.M * sizes > l2_bytes].sum()) if not unfused and cfg.bits != 32 else 0
         per_step = launches // K
         traffic, traffic_src = ncu_traffic(args.path, cfg)
         kernel_name = {"step": "dat_step (k_step_pipelined)", "pipelined": "dat_step_pipelined (k_step_pipelined)",
@@ -424,7 +433,9 @@ def run_gpu(args):
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "traffic_source": traffic_src, "algorithmic_bytes_per_launch": algo_bytes // max(per_step, 1),
                          "algorithmic_bytes_per_step": algo_bytes, "kernel": kernel_name, "peak_source": peak_src,
-                         "sm_cycles_per_step": (1e3 * kernel_ms) * sm_mhz if sm_mhz else None},
+                         "sm_cycles_per_step": (1e3 * kernel_ms) * sm_mhz if sm_mhz else None,
+                         "bytes_2pass": algo_bytes + second_read,
+                         "frac_2pass": (algo_bytes + second_read) / (kernel_ms * 1e-3) / 1e9 / peak},
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "status_word": int(status), "outputs_finite": finite, "wall_s_timed_region": t_wall,
         }
@@ -521,9 +532,9 @@ def main():
                     help="override the resolution of the quantizer's uniform number (0: the config's)")
     ap.add_argument("--impl", default="dat", choices=["dat", "reference"])
     ap.add_argument("--path", default="step",
-                    choices=["step", "step_per_worker", "step_lamb", "pipelined", "passes", "unfused", "unfused_per_worker", "unfused_two_sided", "unfused_lamb"],
+                    choices=["step", "step_per_worker", "step_lamb", "step_two_sided", "pipelined", "passes", "unfused", "unfused_per_worker", "unfused_two_sided", "unfused_lamb"],
                     help="step: dat_step (the headline: one pipelined launch); pipelined: the same by its own name; "
-                         "step_per_worker: dat_step on a plan with one quantizer norm per worker; step_lamb: dat_step_lamb; "
+                         "step_per_worker: dat_step on a plan with one quantizer norm per worker; step_lamb: dat_step_lamb; step_two_sided: dat_step_two_sided (Step 10 in the same launch); "
                          "passes: dat_step_passes, three streaming passes; unfused: dat_quantize + dat_aggregate + dat_lalr_step; "
                          "unfused_per_worker: the same with one quantizer norm per worker; unfused_two_sided: with "
                          "dat_requantize after the aggregation; unfused_lamb: with dat_lamb_step as the update")

@@ -334,6 +334,30 @@ int dat_step_lamb(dat_plan_t *plan, float *theta, float *mom, float *var, const 
                   uint64_t seed, uint64_t step, const dat_lamb_hparams_t *hp, int64_t t,
                   int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream);
 
+/* dat_step_two_sided -- dat_step with two-sided quantisation (Algorithm A1 Step 10, the parameter-server
+ * setting): after Steps 7 and 9 the server quantizes the aggregate itself, g_hat <- Q(g_hat), with its own
+ * norm nu^_l = ||g_hat_l||_2 per layer and the levels of Eq. xi drawn on the random stream of index M (the
+ * first one no worker uses) -- what dat_requantize computes -- and Step 12 uses the receiver's value.  All in
+ * the same single launch: a fourth stream of tiles runs between the Q and the U tiles, waiting (bounded, as
+ * in dat_step) for the layer's nu^_l.  Neither the workers' nor the server's packed message is written.
+ *   g_hat               device fp32[d], caller-owned, 16-byte aligned: workspace (the aggregate is stored
+ *                       here between the two phases) and output: on return the receiver's value
+ *                       nu^_l * sign * level / S of every element.
+ *   server_scales_out   device fp32[h] or NULL: nu^_l.
+ * Other arguments, the bounded wait and its status bit as in dat_step; shared or per-worker plans.
+ * Errors: ARG, ALIGN, BITS (b = 32: nothing to quantize with), UNSUPPORTED (plan with an origin), CUDA. */
+int dat_step_two_sided(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                       uint64_t seed, uint64_t step, const dat_hparams_t *hp, float *g_hat,
+                       int32_t *code_sum_out, float *layer_norms_out, float *scales_out,
+                       float *server_scales_out, void *stream);
+
+/* dat_step_lamb_two_sided -- dat_step_lamb with Step 10 between the aggregation and Algorithm A2, as in
+ * dat_step_two_sided (same g_hat and server_scales_out). */
+int dat_step_lamb_two_sided(dat_plan_t *plan, float *theta, float *mom, float *var, const float *const *grads,
+                            uint64_t seed, uint64_t step, const dat_lamb_hparams_t *hp, int64_t t, float *g_hat,
+                            int32_t *code_sum_out, float *layer_norms_out, float *scales_out,
+                            float *server_scales_out, void *stream);
+
 /* dat_step_passes -- the same step as dat_step, with the same arguments and the same results bit for
  * bit up to the norms' last place, computed by three streaming passes in separate launches: quantizer
  * norms; then levels, signed sum over the workers, g_hat, m' and the layer sums in one pass that keeps

@@ -31,7 +31,7 @@ DAT_STATUS_NONFINITE, DAT_STATUS_TIMEOUT, DAT_STATUS_BOUNDS = 1, 2, 4
 
 # every symbol include/dat.h declares
 EXPORTS = ["dat_plan_create", "dat_plan_set_origin", "dat_plan_destroy", "dat_plan_sizes", "dat_worker_norms", "dat_quantize", "dat_aggregate", "dat_requantize",
-           "dat_average", "dat_lalr_step", "dat_lamb_step", "dat_lalr_step_static", "dat_step", "dat_step_lamb", "dat_step_passes", "dat_step_pipelined", "dat_plan_test_stall", "dat_step_host", "dat_get_status",
+           "dat_average", "dat_lalr_step", "dat_lamb_step", "dat_lalr_step_static", "dat_step", "dat_step_lamb", "dat_step_two_sided", "dat_step_lamb_two_sided", "dat_step_passes", "dat_step_pipelined", "dat_plan_test_stall", "dat_step_host", "dat_get_status",
            "dat_plan_launch_count", "dat_strerror", "dat_last_cuda_error"]
 
 
@@ -61,6 +61,8 @@ _lib.dat_lalr_step_static.argtypes = [_i64, _p, _p, _p, _p, C.POINTER(dat_hparam
 _lib.dat_step.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_plan_test_stall.argtypes = [_p, _i64, _i64, _p]
 _lib.dat_step_lamb.argtypes = [_p, _p, _p, _p, _p, _u64, _u64, C.POINTER(dat_lamb_hparams_t), _i64, _p, _p, _p, _p]
+_lib.dat_step_two_sided.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p, _p, _p]
+_lib.dat_step_lamb_two_sided.argtypes = [_p, _p, _p, _p, _p, _u64, _u64, C.POINTER(dat_lamb_hparams_t), _i64, _p, _p, _p, _p, _p, _p]
 _lib.dat_step_pipelined.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_step_passes.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p, _p, _p, _p]
 _lib.dat_step_host.argtypes = [_p, _p, _p, _p, _u64, _u64, C.POINTER(dat_hparams_t), _p]
@@ -204,6 +206,23 @@ def dat_step_lamb(plan, theta, mom, var, grads, seed, step, hp, t, code_sum_out=
     h = hp if isinstance(hp, dat_lamb_hparams_t) else dat_lamb_hparams_t(*[float(x) for x in hp])
     _ok(_lib.dat_step_lamb(_p(plan), _ptr(theta), _ptr(mom), _ptr(var), _ptr_array(grads), int(seed), int(step), C.byref(h),
                            int(t), _ptr(code_sum_out), _ptr(layer_norms_out), _ptr(scales_out), _stream(stream)), "dat_step_lamb")
+
+
+def dat_step_two_sided(plan, theta, mom, grads, seed, step, hp, g_hat, code_sum_out=None, layer_norms_out=None,
+                       scales_out=None, server_scales_out=None, stream=None):
+    """g_hat: fp32[d] workspace; on return the receiver's value of Algorithm A1 Step 10."""
+    h = _hp(hp)
+    _ok(_lib.dat_step_two_sided(_p(plan), _ptr(theta), _ptr(mom), _ptr_array(grads), int(seed), int(step), C.byref(h),
+                                _ptr(g_hat), _ptr(code_sum_out), _ptr(layer_norms_out), _ptr(scales_out),
+                                _ptr(server_scales_out), _stream(stream)), "dat_step_two_sided")
+
+
+def dat_step_lamb_two_sided(plan, theta, mom, var, grads, seed, step, hp, t, g_hat, code_sum_out=None,
+                            layer_norms_out=None, scales_out=None, server_scales_out=None, stream=None):
+    h = hp if isinstance(hp, dat_lamb_hparams_t) else dat_lamb_hparams_t(*[float(x) for x in hp])
+    _ok(_lib.dat_step_lamb_two_sided(_p(plan), _ptr(theta), _ptr(mom), _ptr(var), _ptr_array(grads), int(seed), int(step),
+                                     C.byref(h), int(t), _ptr(g_hat), _ptr(code_sum_out), _ptr(layer_norms_out),
+                                     _ptr(scales_out), _ptr(server_scales_out), _stream(stream)), "dat_step_lamb_two_sided")
 
 
 def dat_plan_test_stall(plan, wait_cycles, layer=-1, stream=None):

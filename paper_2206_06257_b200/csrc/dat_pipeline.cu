@@ -15,6 +15,11 @@
 // CTAs that started earlier and never wait themselves.  The last CTA to finish a layer's N (or Q)
 // tiles reduces the layer's partial sums in a fixed order and publishes the layer's factors with the
 // call's epoch; a Q (or U) part whose layer is not published yet polls that word, with a limit.
+//
+// Two-sided quantisation (Algorithm A1 Step 10) adds a fourth stream between Q and U: the Q part then
+// stops at g_hat (stored, with the tile's sum of squares), the layer's last Q tile publishes
+// nu^_l = ||g_hat_l||_2, and the R part of a later item draws the server's levels of its tile on the
+// random stream of index M, forms the receiver's value and goes on with m' and the layer sums.
 #include <algorithm>
 #include <new>
 #include <vector>
@@ -51,18 +56,22 @@ struct PipePart {                                 // one tile of one layer; laye
     int32_t layer, tile;
 };
 struct PipeItem {
-    PipePart n, q, u;
+    PipePart n, q, u, r;                          // r: the server's quantizer (two-sided schedules only)
 };
 
 struct PipeSchedule {
     char *mem = nullptr;                          // one device allocation, carved up
     size_t mem_bytes = 0;
-    PipeItem *d_items = nullptr;
+    PipeItem *d_items = nullptr;                  // the three streams N, Q, U
     int64_t n_items = 0;
+    PipeItem *d_items2 = nullptr;                 // the four streams N, Q, R, U of the two-sided step
+    int64_t n_items2 = 0;
+    double *d_partR = nullptr;                    // n_tiles
+    float *d_server = nullptr;                    // 2h: S / nu^_l and nu^_l / S
     int64_t *d_tile_base = nullptr;               // h + 1
     double *d_partN = nullptr;                    // n_tiles * M
     double *d_partQ = nullptr;                    // n_tiles * 2
-    uint32_t *d_sync = nullptr;                   // [0] ticket, [1] abort epoch, then cntN[h], cntQ[h], readyN[h], readyQ[h]
+    uint32_t *d_sync = nullptr;                   // [0] ticket, [1] abort epoch, then cntN[h], cntQ[h], readyN[h], readyQ[h], cntR[h], readyR[h]
     size_t sync_bytes = 0;
     int64_t n_tiles = 0;
     uint32_t epoch = 0;                           // calls made so far
@@ -76,10 +85,11 @@ struct PArgs {
     const int64_t *off, *tile_base;
     float *theta, *mom, *var;                     // var: second moment (LAMB only)
     LambConst lamb;
-    double *partN, *partQ;
-    uint32_t *ticket, *abort_epoch, *cntN, *cntQ, *readyN, *readyQ, *status;
+    double *partN, *partQ, *partR;
+    uint32_t *ticket, *abort_epoch, *cntN, *cntQ, *readyN, *readyQ, *cntR, *readyR, *status;
     float *worker_norms, *scales, *qmul, *dq, *step_a;
-    float *norms_out, *scales_out;
+    float *ghat, *qmul2, *dq2;                    // two-sided: g_hat / the receiver's value (d), the server's factors (h each)
+    float *norms_out, *scales_out, *server_scales_out;
     int32_t *code_sum;
     long long wait_cycles;
     float S_f, SM_f, M_f, mu, wd, lr, c_l, c_u;
@@ -371,10 +381,50 @@ __device__ __forceinline__ void p_rows_per_worker(const PArgs &a, int layer, int
     }
 }
 
+// ---- m' (or m', v') and the layer sums of Eq. 3, pass 1, for one thread's group of eight elements whose
+// g_hat is in registers: theta and m are loaded only now (registers limit the resident warps here).
+template <int OPT>
+__device__ __forceinline__ void p_direction(const PArgs &a, int64_t e0, int64_t lo, int64_t hi, const float ghat[8],
+                                            double &ss_theta, double &ss_u)
+{
+    float th[8], m[8];
+    p_load4_cg(a.theta, e0, lo, hi, th);
+    p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
+    p_load4_cg(a.mom, e0, lo, hi, m);
+    p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
+    if (OPT == P_OPT_LAMB) {
+        // Algorithm A2: both moments are stored, the direction is formed on the fly for the layer sums
+        float v[8];
+        p_load4_cg(a.var, e0, lo, hi, v);
+        p_load4_cg(a.var, e0 + 4, lo, hi, v + 4);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            m[j] = __fmaf_rn(a.lamb.beta1, m[j], __fmul_rn(a.lamb.om1, ghat[j]));
+            v[j] = __fmaf_rn(a.lamb.beta2, v[j], __fmul_rn(a.lamb.om2, __fmul_rn(ghat[j], ghat[j])));
+            const bool inside = (e0 + j >= lo && e0 + j < hi);
+            const float u = inside ? dat_lamb_direction(a.lamb, m[j], v[j], th[j]) : 0.0f;
+            ss_theta = fma((double)th[j], (double)th[j], ss_theta);
+            ss_u = fma((double)u, (double)u, ss_u);
+        }
+        dat_store4(a.var, e0, lo, hi, v);
+        dat_store4(a.var, e0 + 4, lo, hi, v + 4);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            m[j] = __fmaf_rn(a.mu, m[j], __fmaf_rn(a.wd, th[j], ghat[j]));
+            ss_theta = fma((double)th[j], (double)th[j], ss_theta);
+            ss_u = fma((double)m[j], (double)m[j], ss_u);
+        }
+    }
+    dat_store4(a.mom, e0, lo, hi, m);
+    dat_store4(a.mom, e0 + 4, lo, hi, m + 4);
+}
+
 // ---- Q: levels (Eq. xi), signed sum over the workers and g_hat (Eq. grad_agg), m' and the layer sums
 // (Eq. 3, pass 1) of one tile; codes, sums and g_hat stay in registers.  Leaves the tile's two sums per
-// warp in scratch[2w], scratch[2w + 1]. -------------------------------------------------------------
-template <bool RNG16, int MODE, int OPT>
+// warp in scratch[2w], scratch[2w + 1].  TWO (Algorithm A1 Step 10 follows): stops at g_hat, which is
+// stored, and leaves the tile's sum of g_hat^2 per warp in scratch[2w]. ----------------------------
+template <bool RNG16, int MODE, int OPT, bool TWO>
 __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt, double *scratch)
 {
     const int M = a.M, layer = pt.layer;
@@ -409,7 +459,24 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
         else if (full) qu_rows<RNG16, true, true>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         else if (!plain) qu_rows<RNG16, false, false>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
         else qu_rows<RNG16, false, true>(a.gp, a.keys, qc, M, e0, lo, hi, acc);
-        // theta and m only now: registers are what limits the number of resident warps here
+        if (TWO) {
+            if (MODE == P_MODE_SHARED && a.code_sum) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (e0 + j >= lo && e0 + j < hi) a.code_sum[e0 + j] = (int)acc[j];
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                acc[j] = (MODE == P_MODE_IDENTITY) ? acc[j] / a.M_f : (MODE == P_MODE_PER_WORKER) ? acc[j] / a.SM_f : acc[j] * f;
+            dat_store4(a.ghat, e0, lo, hi, acc);
+            dat_store4(a.ghat, e0 + 4, lo, hi, acc + 4);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) ss_theta = fma((double)acc[j], (double)acc[j], ss_theta);
+            continue;
+        }
+        // theta and m only now: registers are what limits the number of resident warps here.  (The same
+        // arithmetic as p_direction, spelled out so that the loads are issued before g_hat is scaled: the step
+        // is 3 % slower with the call.)
         float th[8], m[8];
         p_load4_cg(a.theta, e0, lo, hi, th);
         p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
@@ -449,12 +516,97 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
         dat_store4(a.mom, e0, lo, hi, m);
         dat_store4(a.mom, e0 + 4, lo, hi, m + 4);
     }
-    __threadfence();                               // m' (and v') are read by the U part of another CTA
+    __threadfence();                               // m' (and v'), or g_hat, are read by a later part of another CTA
     ss_theta = dat_warp_sum(ss_theta);
     ss_u = dat_warp_sum(ss_u);
     if ((threadIdx.x & 31) == 0) {
         scratch[2 * (threadIdx.x >> 5)] = ss_theta;
         scratch[2 * (threadIdx.x >> 5) + 1] = ss_u;
+    }
+}
+
+// ---- R: Algorithm A1 Step 10 on one tile.  g_hat <- nu^_l * sign * level / S with the level of Eq. xi
+// drawn on the random stream of index M (the first one no worker uses), then m' and the layer sums as in
+// the Q part of the one-sided step. ------------------------------------------------------------------
+template <bool RNG16, int OPT>
+__device__ __forceinline__ void p_part_requant(const PArgs &a, const PipePart &pt, double *scratch)
+{
+    const int64_t lo = pt.lo, hi = pt.hi;
+    const float t = __ldcg(a.qmul2 + pt.layer), f = __ldcg(a.dq2 + pt.layer);
+    const float two_b = a.S_f + 1.0f;
+    double ss_theta = 0.0, ss_u = 0.0;
+    const int64_t begin = p_tile_begin(pt);
+#pragma unroll 1
+    for (int k = 0; k < DAT_P_GROUPS; ++k) {
+        const int64_t e0 = begin + 8 * (int64_t)(k * DAT_P_THREADS + threadIdx.x);
+        if (e0 >= hi) continue;
+        float v[8];
+        p_load4_cg(a.ghat, e0, lo, hi, v);
+        p_load4_cg(a.ghat, e0 + 4, lo, hi, v + 4);
+        uint32_t w[8];
+        if (RNG16) {
+            dat_random_words((uint64_t)e0 >> 3, (uint32_t)a.M, a.keys, w);
+        } else {
+            dat_random_words((uint64_t)e0 >> 2, (uint32_t)a.M, a.keys, w);
+            dat_random_words(((uint64_t)e0 >> 2) + 1, (uint32_t)a.M, a.keys, w + 4);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float u1 = RNG16 ? dat_u1_from_half((j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xFFFFu)) : dat_u1_from_word(w[j]);
+            const int lev = (int)dat_level_u1(v[j], t, two_b, u1);
+            v[j] = (float)((v[j] < 0.0f) ? -lev : lev) * f;
+        }
+        dat_store4(a.ghat, e0, lo, hi, v);          // the receiver's value
+        dat_store4(a.ghat, e0 + 4, lo, hi, v + 4);
+        p_direction<OPT>(a, e0, lo, hi, v, ss_theta, ss_u);
+    }
+    __threadfence();
+    ss_theta = dat_warp_sum(ss_theta);
+    ss_u = dat_warp_sum(ss_u);
+    if ((threadIdx.x & 31) == 0) {
+        scratch[2 * (threadIdx.x >> 5)] = ss_theta;
+        scratch[2 * (threadIdx.x >> 5) + 1] = ss_u;
+    }
+}
+
+// Two-sided step, one thread after the barrier that follows the Q part: the tile's sum of g_hat^2 (warps in
+// index order), counted in.  Returns whether this was the layer's last tile.
+__device__ __forceinline__ bool p_server_publish(const PArgs &a, const PipePart &pt, const double *scratch)
+{
+    double x = 0.0;
+#pragma unroll
+    for (int w = 0; w < DAT_P_THREADS / 32; ++w) x += scratch[2 * w];
+    a.partR[(int64_t)pt.tb + pt.tile] = x;
+    __threadfence();
+    return atomicAdd(a.cntR + pt.layer, 1u) == (uint32_t)pt.T - 1u;
+}
+
+// The CTA that counted in the layer's last Q tile of a two-sided step (every thread): the server's norm
+// nu^_l = ||g_hat_l||_2 from the tiles' sums in index order, and its two factors, published with the epoch.
+__device__ __forceinline__ void p_server_finish(const PArgs &a, const PipePart &pt, double *scratch)
+{
+    const int layer = pt.layer;
+    const int64_t tb = pt.tb;
+    const uint32_t T = (uint32_t)pt.T;
+    __threadfence();
+    double x = 0.0;
+    for (uint32_t t = threadIdx.x; t < T; t += DAT_P_THREADS) x += __ldcg(a.partR + tb + t);
+    x = dat_warp_sum(x);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        x = 0.0;
+#pragma unroll
+        for (int w = 0; w < DAT_P_THREADS / 32; ++w) x += scratch[w];
+        const float nu = (float)sqrt(x);
+        a.qmul2[layer] = (nu == 0.0f) ? 0.0f : a.S_f / nu;
+        a.dq2[layer] = (nu == 0.0f) ? 0.0f : nu / a.S_f;
+        if (a.server_scales_out) a.server_scales_out[layer] = nu;
+        if (!isfinite(nu)) atomicOr(a.status, DAT_STATUS_NONFINITE);
+        a.cntR[layer] = 0u;
+        __threadfence();
+        p_st_release(a.readyR + layer, a.epoch);
     }
 }
 
@@ -521,7 +673,7 @@ __device__ __forceinline__ void p_part_update(const PArgs &a, const PipePart &pt
     }
 }
 
-template <bool RNG16, int MODE, int OPT>
+template <bool RNG16, int MODE, int OPT, bool TWO>
 __global__ void __launch_bounds__(DAT_P_THREADS, DAT_P_MINB)
 k_step_pipelined(const __grid_constant__ PArgs a)
 {
@@ -539,17 +691,20 @@ k_step_pipelined(const __grid_constant__ PArgs a)
         }
         tk = __shfl_sync(0xFFFFFFFFu, tk, 0);
         if (!P_CHECK(a, tk < a.n_items)) tk = 0;
-        if (lane < (int)(sizeof(PipeItem) / 16))
+        if (lane < (int)((TWO ? sizeof(PipeItem) : 3 * sizeof(PipePart)) / 16))
             reinterpret_cast<uint4 *>(&s_item)[lane] = __ldg(reinterpret_cast<const uint4 *>(a.items + tk) + lane);
     }
     for (int u = threadIdx.x; u < 4 * a.M; u += DAT_P_THREADS) s_unit[u] = 0.0;
     __syncthreads();
     const PipePart pn = s_item.n, pq = s_item.q, pu = s_item.u;
+    PipePart pm = pq;                               // the part that leaves m' and the tile's two sums of Eq. 3
 #ifdef DAT_SELFCHECK
     {
         bool ok = pn.layer < a.h && pq.layer < a.h && pu.layer < a.h;
-        const PipePart *pp[3] = {&pn, &pq, &pu};
-        for (int k = 0; k < 3 && ok; ++k)
+        const PipePart pr = TWO ? s_item.r : pq;
+        ok = ok && pr.layer < a.h;
+        const PipePart *pp[4] = {&pn, &pq, &pu, &pr};
+        for (int k = 0; k < 4 && ok; ++k)
             if (pp[k]->layer >= 0)
                 ok = pp[k]->tile >= 0 && pp[k]->tile < pp[k]->T && (int64_t)pp[k]->tb + pp[k]->tile < a.n_tiles &&
                      pp[k]->lo >= 0 && pp[k]->lo < pp[k]->hi && pp[k]->hi <= a.d;
@@ -572,18 +727,31 @@ k_step_pipelined(const __grid_constant__ PArgs a)
     }
     __syncthreads();                               // (A)
     if (s_ctl[0]) p_norm_finish<MODE>(a, pn, s_norm);
-    const bool alive = (s_ctl[1] != 0);
-    if (alive && pq.layer >= 0) p_part_quant<RNG16, MODE, OPT>(a, pq, s_unit);
+    bool alive = (s_ctl[1] != 0);
+    if (alive && pq.layer >= 0) p_part_quant<RNG16, MODE, OPT, TWO>(a, pq, s_unit);
     __syncthreads();
+    if (TWO) {
+        // Step 10: the tile's sum of g_hat^2 counted in; the layer's last tile publishes the server's norm;
+        // then the R part of this item (a tile of an earlier layer) once that layer's norm is published
+        pm = s_item.r;
+        if (threadIdx.x == 0) s_ctl[2] = (alive && pq.layer >= 0) ? (int)p_server_publish(a, pq, s_unit) : 0;
+        __syncthreads();
+        if (s_ctl[2]) p_server_finish(a, pq, s_unit);
+        if (threadIdx.x == 0) s_ctl[1] = (alive && pm.layer >= 0) ? (int)p_poll(a, a.readyR + pm.layer) : (int)alive;
+        __syncthreads();
+        alive = (s_ctl[1] != 0);
+        if (alive && pm.layer >= 0) p_part_requant<RNG16, OPT>(a, pm, s_unit);
+        __syncthreads();
+    }
     if (threadIdx.x == 0) {
         bool q_last = false, u_go = alive;
-        if (alive && pq.layer >= 0) q_last = p_quant_publish(a, pq, s_unit);
+        if (alive && pm.layer >= 0) q_last = p_quant_publish(a, pm, s_unit);
         if (alive && pu.layer >= 0) u_go = p_poll(a, a.readyQ + pu.layer);
         s_ctl[2] = q_last;
         s_ctl[3] = u_go;
     }
     __syncthreads();                               // (B)
-    if (s_ctl[2]) p_quant_finish(a, pq, s_unit);
+    if (s_ctl[2]) p_quant_finish(a, pm, s_unit);
     if (s_ctl[3] && pu.layer >= 0) p_part_update<OPT>(a, pu);
 }
 
@@ -623,60 +791,81 @@ int dat_pipe_build(dat_plan_t *plan)
         std::stable_sort(order.begin(), order.end(), [&](int x, int y) {
             return plan->offsets[x + 1] - plan->offsets[x] < plan->offsets[y + 1] - plan->offsets[y];
         });
-        // slot of every tile in each of the three streams
-        std::vector<PipeItem> items;
+        // slot of every tile in each of the three streams (four with the server's quantizer between Q and U)
         const PipePart nopart = {0, 1, 0, 1, -1, 0};
-        const PipeItem none = {nopart, nopart, nopart};
+        const PipeItem none = {nopart, nopart, nopart, nopart};
         auto part = [&](int l, int64_t t) {
             PipePart pp = {plan->offsets[l], plan->offsets[l + 1], (int32_t)tb[l], (int32_t)(tb[l + 1] - tb[l]), l, (int32_t)t};
             return pp;
         };
-        auto at = [&](int64_t slot) -> PipeItem & {
-            if ((int64_t)items.size() <= slot) items.resize((size_t)slot + 1, none);
-            return items[(size_t)slot];
-        };
-        std::vector<int64_t> done_n((size_t)h, -1 - (int64_t)DAT_P_LAG), done_q((size_t)h, 0);
-        int64_t slot = 0;
-        if (!identity)
+        auto build = [&](bool two) {
+            std::vector<PipeItem> items;
+            auto at = [&](int64_t slot) -> PipeItem & {
+                if ((int64_t)items.size() <= slot) items.resize((size_t)slot + 1, none);
+                return items[(size_t)slot];
+            };
+            std::vector<int64_t> done_n((size_t)h, -1 - (int64_t)DAT_P_LAG), done_q((size_t)h, 0), done_r((size_t)h, 0);
+            int64_t slot = 0;
+            if (!identity)
+                for (int k = 0; k < h; ++k) {
+                    const int l = order[k];
+                    for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { at(slot).n = part(l, t); done_n[l] = slot++; }
+                }
+            slot = 0;
             for (int k = 0; k < h; ++k) {
                 const int l = order[k];
-                for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { at(slot).n = part(l, t); done_n[l] = slot++; }
+                const int64_t T = tb[l + 1] - tb[l];
+                slot = std::max(slot, done_n[l] + DAT_P_LAG + 1);
+                // a layer that L2 cannot hold next to what streams in meanwhile is walked back from its last
+                // tile (what N read last is read first); the others in N's order, every tile at the same distance
+                const bool reverse = T >= DAT_P_REVERSE_FROM;
+                for (int64_t t = 0; t < T; ++t) { at(slot).q = part(l, reverse ? T - 1 - t : t); done_q[l] = slot++; }
             }
-        slot = 0;
-        for (int k = 0; k < h; ++k) {
-            const int l = order[k];
-            const int64_t T = tb[l + 1] - tb[l];
-            slot = std::max(slot, done_n[l] + DAT_P_LAG + 1);
-            // a layer that L2 cannot hold next to what streams in meanwhile is walked back from its last
-            // tile (what N read last is read first); the others in N's order, every tile at the same distance
-            const bool reverse = T >= DAT_P_REVERSE_FROM;
-            for (int64_t t = 0; t < T; ++t) { at(slot).q = part(l, reverse ? T - 1 - t : t); done_q[l] = slot++; }
-        }
-        slot = 0;
-        for (int k = 0; k < h; ++k) {
-            const int l = order[k];
-            slot = std::max(slot, done_q[l] + DAT_P_LAG_U + 1);
-            for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { at(slot).u = part(l, t); ++slot; }
-        }
+            if (two) {
+                slot = 0;
+                for (int k = 0; k < h; ++k) {
+                    const int l = order[k];
+                    slot = std::max(slot, done_q[l] + DAT_P_LAG_U + 1);
+                    for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { at(slot).r = part(l, t); done_r[l] = slot++; }
+                }
+            }
+            slot = 0;
+            for (int k = 0; k < h; ++k) {
+                const int l = order[k];
+                slot = std::max(slot, (two ? done_r[l] : done_q[l]) + DAT_P_LAG_U + 1);
+                for (int64_t t = 0; t < tb[l + 1] - tb[l]; ++t) { at(slot).u = part(l, t); ++slot; }
+            }
+            return items;
+        };
+        const std::vector<PipeItem> items = build(false);
+        const std::vector<PipeItem> items2 = identity ? std::vector<PipeItem>() : build(true);
+        g->n_items2 = (int64_t)items2.size();
         g->n_items = (int64_t)items.size();
 
         size_t off = 0;
         auto take = [&](size_t bytes) { size_t o = off; off = p_align(off + bytes); return o; };
-        const size_t o_items = take(items.size() * sizeof(PipeItem)), o_tb = take(((size_t)h + 1) * 8);
-        const size_t o_pn = take((size_t)nt * (size_t)M * 8), o_pq = take((size_t)nt * 16);
-        g->sync_bytes = (2 + 4 * (size_t)h) * 4;
+        const size_t o_items = take(items.size() * sizeof(PipeItem)), o_items2 = take(items2.size() * sizeof(PipeItem));
+        const size_t o_tb = take(((size_t)h + 1) * 8);
+        const size_t o_pn = take((size_t)nt * (size_t)M * 8), o_pq = take((size_t)nt * 16), o_pr = take((size_t)nt * 8);
+        const size_t o_server = take(2 * (size_t)h * 4);
+        g->sync_bytes = (2 + 6 * (size_t)h) * 4;
         const size_t o_sync = take(g->sync_bytes);
         g->mem_bytes = off;
         cudaError_t e;
         e = cudaMalloc((void **)&g->mem, off);
         if (e != cudaSuccess) { g->mem = nullptr; plan->last_cuda = (int)e; (void)cudaGetLastError(); return DAT_ERR_NOMEM; }
         g->d_items = (PipeItem *)(g->mem + o_items);
+        g->d_items2 = (PipeItem *)(g->mem + o_items2);
+        g->d_partR = (double *)(g->mem + o_pr);
+        g->d_server = (float *)(g->mem + o_server);
         g->d_tile_base = (int64_t *)(g->mem + o_tb);
         g->d_partN = (double *)(g->mem + o_pn);
         g->d_partQ = (double *)(g->mem + o_pq);
         g->d_sync = (uint32_t *)(g->mem + o_sync);
         e = cudaMemset(g->mem, 0, off);
         if (e == cudaSuccess) e = cudaMemcpy(g->d_items, items.data(), items.size() * sizeof(PipeItem), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess && !items2.empty())
+            e = cudaMemcpy(g->d_items2, items2.data(), items2.size() * sizeof(PipeItem), cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = cudaMemcpy(g->d_tile_base, tb.data(), ((size_t)h + 1) * 8, cudaMemcpyHostToDevice);
         if (e != cudaSuccess) return dat_cuda_fail(plan, e);
     } catch (...) {
@@ -695,15 +884,20 @@ cudaError_t dat_pipe_reset(dat_plan_t *plan, cudaStream_t s)
 }
 
 // One launch of the step.  lamb == nullptr: the momentum direction with hp; else Algorithm A2 with *lamb.
+// g_hat != nullptr: the two-sided step (Algorithm A1 Step 10 between the aggregation and the update).
 static int p_launch(dat_plan_t *plan, float *theta, float *mom, float *var, const float *const *grads,
                     uint64_t seed, uint64_t step, const dat_hparams_t *hp, const LambConst *lamb, float lr, float c_l, float c_u,
-                    int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream)
+                    int32_t *code_sum_out, float *layer_norms_out, float *scales_out, void *stream,
+                    float *g_hat = nullptr, float *server_scales_out = nullptr)
 {
     if (step >> 32) return DAT_ERR_ARG;
     if (plan->elem_base || plan->worker_base) return DAT_ERR_UNSUPPORTED;     // a slice of a larger problem: separate calls only
     if (!dat_aligned16(theta) || !dat_aligned16(mom) || (var && !dat_aligned16(var)) || (code_sum_out && !dat_aligned16(code_sum_out)) ||
-        (layer_norms_out && !dat_aligned16(layer_norms_out)) || (scales_out && !dat_aligned16(scales_out)))
+        (layer_norms_out && !dat_aligned16(layer_norms_out)) || (scales_out && !dat_aligned16(scales_out)) ||
+        (g_hat && !dat_aligned16(g_hat)) || (server_scales_out && !dat_aligned16(server_scales_out)))
         return DAT_ERR_ALIGN;
+    const bool two = (g_hat != nullptr);
+    if (two && plan->bits == 32) return DAT_ERR_BITS;      // nothing to quantize with
     PArgs a;
     int rc = dat_check_grads(plan, grads, &a.gp);
     if (rc != DAT_OK) return rc;
@@ -713,7 +907,7 @@ static int p_launch(dat_plan_t *plan, float *theta, float *mom, float *var, cons
     const bool per_worker = !identity && plan->scale_mode == DAT_SCALE_PER_WORKER;
     const size_t h = (size_t)plan->h;
     a.keys = dat_make_keys(seed, step);
-    a.items = g->d_items;
+    a.items = two ? g->d_items2 : g->d_items;
     a.off = plan->d_offsets;
     a.tile_base = g->d_tile_base;
     a.theta = theta;
@@ -723,12 +917,19 @@ static int p_launch(dat_plan_t *plan, float *theta, float *mom, float *var, cons
     else a.lamb = LambConst{0.0f, 0.0f, 0.0f, 0.0f, 1.0f, 1.0f, 1.0f, 0.0f};
     a.partN = g->d_partN;
     a.partQ = g->d_partQ;
+    a.partR = g->d_partR;
     a.ticket = g->d_sync;
     a.abort_epoch = g->d_sync + 1;
     a.cntN = g->d_sync + 2;
     a.cntQ = a.cntN + h;
     a.readyN = a.cntQ + h;
     a.readyQ = a.readyN + h;
+    a.cntR = a.readyQ + h;
+    a.readyR = a.cntR + h;
+    a.ghat = g_hat;
+    a.qmul2 = g->d_server;
+    a.dq2 = g->d_server + h;
+    a.server_scales_out = server_scales_out;
     a.status = plan->d_status;
     a.worker_norms = plan->d_worker_norms;
     a.scales = plan->d_scales;
@@ -749,17 +950,22 @@ static int p_launch(dat_plan_t *plan, float *theta, float *mom, float *var, cons
     a.c_u = c_u;
     if (++g->epoch == 0u) ++g->epoch;              // 0 is what the words hold before the first call
     a.epoch = g->epoch;
-    a.n_items = (uint32_t)g->n_items;
+    a.n_items = (uint32_t)(two ? g->n_items2 : g->n_items);
     a.M = plan->M;
     a.h = (int)plan->h;
     a.d = plan->d;
     a.n_tiles = g->n_tiles;
     cudaStream_t s = (cudaStream_t)stream;
-    const unsigned grid = (unsigned)g->n_items;
+    const unsigned grid = a.n_items;
     const bool rng16 = (plan->rng_bits == 16);
-#define P_GO(R, MODE, OPT) k_step_pipelined<R, MODE, OPT><<<grid, DAT_P_THREADS, 0, s>>>(a)
-#define P_GO_OPT(R, MODE) do { if (lamb) P_GO(R, MODE, P_OPT_LAMB); else P_GO(R, MODE, P_OPT_MOMENTUM); } while (0)
-    if (identity) P_GO_OPT(true, P_MODE_IDENTITY);
+#define P_GO(R, MODE, OPT, TWO) k_step_pipelined<R, MODE, OPT, TWO><<<grid, DAT_P_THREADS, 0, s>>>(a)
+#define P_GO_OPT(R, MODE)                                                                                           \
+    do {                                                                                                            \
+        if (two) { if (lamb) P_GO(R, MODE, P_OPT_LAMB, true); else P_GO(R, MODE, P_OPT_MOMENTUM, true); }           \
+        else if (lamb) P_GO(R, MODE, P_OPT_LAMB, false);                                                            \
+        else P_GO(R, MODE, P_OPT_MOMENTUM, false);                                                                  \
+    } while (0)
+    if (identity) { if (lamb) P_GO(true, P_MODE_IDENTITY, P_OPT_LAMB, false); else P_GO(true, P_MODE_IDENTITY, P_OPT_MOMENTUM, false); }
     else if (per_worker && rng16) P_GO_OPT(true, P_MODE_PER_WORKER);
     else if (per_worker) P_GO_OPT(false, P_MODE_PER_WORKER);
     else if (rng16) P_GO_OPT(true, P_MODE_SHARED);
@@ -792,6 +998,32 @@ extern "C" int dat_step_lamb(dat_plan_t *plan, float *theta, float *mom, float *
     const LambConst c = dat_lamb_const(hp, t);
     return p_launch(plan, theta, mom, var, grads, seed, step, nullptr, &c, hp->lr, hp->c_l, hp->c_u, code_sum_out,
                     layer_norms_out, scales_out, stream);
+}
+
+extern "C" int dat_step_two_sided(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
+                                  uint64_t seed, uint64_t step, const dat_hparams_t *hp, float *g_hat,
+                                  int32_t *code_sum_out, float *layer_norms_out, float *scales_out,
+                                  float *server_scales_out, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (!theta || !mom || !hp || !g_hat) return DAT_ERR_ARG;
+    return p_launch(plan, theta, mom, nullptr, grads, seed, step, hp, nullptr, hp->lr, hp->c_l, hp->c_u, code_sum_out,
+                    layer_norms_out, scales_out, stream, g_hat, server_scales_out);
+}
+
+extern "C" int dat_step_lamb_two_sided(dat_plan_t *plan, float *theta, float *mom, float *var, const float *const *grads,
+                                       uint64_t seed, uint64_t step, const dat_lamb_hparams_t *hp, int64_t t, float *g_hat,
+                                       int32_t *code_sum_out, float *layer_norms_out, float *scales_out,
+                                       float *server_scales_out, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (!theta || !mom || !var || !hp || !g_hat || t < 1) return DAT_ERR_ARG;
+    if (!(hp->beta1 > 0.0f && hp->beta1 < 1.0f && hp->beta2 > 0.0f && hp->beta2 < 1.0f)) return DAT_ERR_ARG;
+    const LambConst c = dat_lamb_const(hp, t);
+    return p_launch(plan, theta, mom, var, grads, seed, step, nullptr, &c, hp->lr, hp->c_l, hp->c_u, code_sum_out,
+                    layer_norms_out, scales_out, stream, g_hat, server_scales_out);
 }
 
 // Test hook (see dat.h): a short wait limit, and a layer whose norm never completes in the next call.

@@ -285,6 +285,98 @@ def test_step_lamb_parity_three_steps(api, oracle, mode):
         assert e.value.code == api.DAT_ERR_ARG
 
 
+def _two_sided_reference(oracle, offs, grads, bits, seed, step, M, sm, rng_bits, sc_gpu, sc2_gpu):
+    """Steps 7, 9 and 10 from the oracle's own operations: the workers' levels with the GPU's quantizer norms,
+    the aggregate, the server's Q(g_hat) with the GPU's server norms (each norm checked to the last place first)."""
+    sc_ref = oracle.scales(oracle.worker_norms(offs, grads), sm)
+    assert ulp_diff(sc_gpu.reshape(sc_ref.shape), sc_ref).max() <= 1
+    level, neg = oracle.quantize(offs, grads, bits, seed, step, sc_gpu, sm, rng_bits=rng_bits)
+    cs, gh = oracle.aggregate(offs, level, neg, sc_gpu, bits, sm)
+    _, sc2_ref, _, _ = oracle.requantize(offs, gh, bits, seed, step, stream=M, rng_bits=rng_bits)
+    assert ulp_diff(sc2_gpu, sc2_ref).max() <= 1
+    out, _, _, _ = oracle.requantize(offs, gh, bits, seed, step, stream=M, rng_bits=rng_bits, scales_in=sc2_gpu)
+    return cs, out
+
+
+@pytest.mark.parametrize("mode", ["shared", "per_worker"])
+@pytest.mark.parametrize("bits", [1, 2, 8, 16])
+def test_step_two_sided_parity(api, oracle, bits, mode, rng_bits):
+    """dat_step_two_sided: Steps 7, 9, 10 and 12 in the one launch, twice in a row on the same plan (fresh
+    gradients, advancing step counter).  The receiver's value and m' bit for bit, theta' within the tolerance."""
+    M = 5
+    sm = oracle.SCALE_PER_WORKER if mode == "per_worker" else oracle.SCALE_SHARED_MAX
+    sizes = SIZES_RAGGED + [50000]
+    offs, _, theta, mom = _random_problem(300 + bits, sizes, M)
+    d, h = int(offs[-1]), len(offs) - 1
+    theta[int(offs[4]):int(offs[5])] = 0.0                     # an all-zero parameter tensor
+    with GpuPlan(api, offs, M, bits, rng_bits, scale_mode=api.DAT_SCALE_PER_WORKER if mode == "per_worker" else 0) as P:
+        th_d, mo_d = torch.from_numpy(theta.copy()).cuda(), torch.from_numpy(mom.copy()).cuda()
+        gh_d = torch.full((d,), float("nan"), dtype=torch.float32, device="cuda")
+        cs_d = torch.zeros(d, dtype=torch.int32, device="cuda")
+        norms = torch.zeros(2 * h, dtype=torch.float32, device="cuda")
+        sc = torch.zeros(P.num_scales, dtype=torch.float32, device="cuda")
+        sc2 = torch.zeros(h, dtype=torch.float32, device="cuda")
+        mo_ref = mom
+        for step in (0, 1):
+            _, grads, _, _ = _random_problem(400 + bits + step, sizes, M, dist="t3" if step else "normal")
+            if step == 1:
+                for g in grads:
+                    g[int(offs[10]):int(offs[11])] = 0.0       # a layer with zero gradient: nu = nu^ = 0
+            th_in = np_of(th_d).copy()
+            api.dat_step_two_sided(P.plan, th_d, mo_d, [torch.from_numpy(g).cuda() for g in grads], 9, step, HP, gh_d,
+                                   cs_d, norms, sc, sc2)
+            torch.cuda.synchronize()
+            assert P.status() == 0
+            cs_ref, out = _two_sided_reference(oracle, offs, grads, bits, 9, step, M, sm, rng_bits, np_of(sc), np_of(sc2))
+            if mode == "shared":
+                assert np.array_equal(np_of(cs_d), cs_ref)
+            assert np.array_equal(np_of(gh_d).view(np.uint32), out.view(np.uint32)), "the receiver's value"
+            th_ref, mo_ref, n_ref = oracle.lalr(offs, th_in, mo_ref, out, *HP)
+            assert np.array_equal(np_of(mo_d).view(np.uint32), mo_ref.view(np.uint32))
+            assert ulp_diff(np_of(norms).reshape(-1, 2), n_ref).max() <= 1
+            assert_close_per_layer(np_of(th_d), th_ref, offs, "theta (dat_step_two_sided, step %d)" % step)
+        # the one-sided step on the same plan afterwards is the ordinary one
+        th1, mo1 = torch.from_numpy(theta.copy()).cuda(), torch.from_numpy(mom.copy()).cuda()
+        th2, mo2 = th1.clone(), mo1.clone()
+        gs = [torch.from_numpy(g).cuda() for g in grads]
+        api.dat_step(P.plan, th1, mo1, gs, 9, 5, HP)
+        with GpuPlan(api, offs, M, bits, rng_bits, scale_mode=api.DAT_SCALE_PER_WORKER if mode == "per_worker" else 0) as P2:
+            api.dat_step(P2.plan, th2, mo2, gs, 9, 5, HP)
+            torch.cuda.synchronize()
+        assert torch.equal(th1, th2) and torch.equal(mo1, mo2)
+
+
+def test_step_lamb_two_sided_parity(api, oracle):
+    M, bits = 4, 4
+    sizes = SIZES_RAGGED + [50000]
+    offs, grads, theta, _ = _random_problem(95, sizes, M)
+    d, h = int(offs[-1]), len(offs) - 1
+    mom, var = np.zeros(d, dtype=np.float32), np.zeros(d, dtype=np.float32)
+    with GpuPlan(api, offs, M, bits, 16) as P:
+        th_d, mo_d, va_d = (torch.from_numpy(x.copy()).cuda() for x in (theta, mom, var))
+        gh_d = torch.zeros(d, dtype=torch.float32, device="cuda")
+        norms = torch.zeros(2 * h, dtype=torch.float32, device="cuda")
+        sc = torch.zeros(P.num_scales, dtype=torch.float32, device="cuda")
+        sc2 = torch.zeros(h, dtype=torch.float32, device="cuda")
+        mo_ref, va_ref = mom, var
+        for t in (1, 2):
+            th_in = np_of(th_d).copy()
+            api.dat_step_lamb_two_sided(P.plan, th_d, mo_d, va_d, [torch.from_numpy(g).cuda() for g in grads], 7, t, LAMB_HP, t,
+                                        gh_d, None, norms, sc, sc2)
+            torch.cuda.synchronize()
+            assert P.status() == 0
+            _, out = _two_sided_reference(oracle, offs, grads, bits, 7, t, M, oracle.SCALE_SHARED_MAX, 16, np_of(sc), np_of(sc2))
+            th_ref, mo_ref, va_ref, n_ref = oracle.lamb(offs, th_in, mo_ref, va_ref, out, t, *LAMB_HP)
+            assert np.array_equal(np_of(mo_d).view(np.uint32), mo_ref.view(np.uint32))
+            assert np.array_equal(np_of(va_d).view(np.uint32), va_ref.view(np.uint32))
+            assert ulp_diff(np_of(norms).reshape(-1, 2), n_ref).max() <= 1
+            assert_close_per_layer(np_of(th_d), th_ref, offs, "theta (dat_step_lamb_two_sided, t = %d)" % t)
+    with GpuPlan(api, offs, M, 32, 16) as P:                    # b = 32: nothing to quantize with
+        with pytest.raises(api.DatError) as e:
+            api.dat_step_two_sided(P.plan, th_d, mo_d, [torch.from_numpy(g).cuda() for g in grads], 7, 0, HP, gh_d)
+        assert e.value.code == api.DAT_ERR_BITS
+
+
 @pytest.mark.parametrize("bits", [1, 2, 4, 8, 16, 32])
 def test_fused_parity_ragged(api, oracle, bits, rng_bits):
     offs, grads, theta, mom = _random_problem(100 + bits, SIZES_RAGGED, 3)
