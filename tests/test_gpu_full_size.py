@@ -114,3 +114,51 @@ def test_flat_1b_sampled_layers(oracle, bits, entry):
         sample = [l for l in sample if sizes[l] <= 2_000_000]
     _run_and_check(oracle, cfg, sample, entry=entry)
     torch.cuda.empty_cache()
+
+
+def test_resnet50_two_sided_sampled_layers(oracle):
+    """dat_step_two_sided on the bench workload.  The oracle's own operations, layer by layer on windows that
+    keep the global element index: the workers' levels, the aggregate, then -- on the full vector, with the
+    sampled layers filled in -- the server's Q(g_hat), and the update of each sampled layer."""
+    from paper_2206_06257_b200 import api, synth
+    cfg = synth.config("resnet50")
+    dev, step = "cuda", 2
+    theta, mom = synth.make_params(cfg, device=dev)
+    grads = synth.make_grads(cfg, step, device=dev)
+    hp = hp_tuple(cfg)
+    th0, mo0 = theta.clone(), mom.clone()
+    gh = torch.zeros(cfg.d, dtype=torch.float32, device=dev)
+    sc = torch.zeros(cfg.h, dtype=torch.float32, device=dev)
+    sc2 = torch.zeros(cfg.h, dtype=torch.float32, device=dev)
+    norms = torch.zeros(2 * cfg.h, dtype=torch.float32, device=dev)
+    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits, rng_bits=cfg.rng_bits)
+    try:
+        api.dat_step_two_sided(plan, theta, mom, grads, cfg.seed, step, hp, gh, None, norms, sc, sc2)
+        torch.cuda.synchronize()
+        assert api.dat_get_status(plan) == 0
+    finally:
+        api.dat_plan_destroy(plan)
+    offs = cfg.offsets
+    sizes = np.diff(offs)
+    sample = sorted(set(list(range(0, cfg.h, 9)) + [int(np.argmax(sizes)), int(np.argmin(sizes)), cfg.h - 2, cfg.h - 1]))
+    sc_h, sc2_h = np_of(sc), np_of(sc2)
+    gh_full = np.zeros(cfg.d, dtype=np.float32)
+    for l in sample:
+        a, b = int(offs[l]), int(offs[l + 1])
+        g_l = [np_of(g[a:b]) for g in grads]
+        nu = oracle.scales(oracle.worker_norms(offs, g_l, l0=l, l1=l + 1, window=True))
+        assert ulp_diff(sc_h[l:l + 1], nu[l:l + 1]).max() <= 1
+        level, neg = oracle.quantize(offs, g_l, cfg.bits, cfg.seed, step, sc_h, l0=l, l1=l + 1, window=True, rng_bits=cfg.rng_bits)
+        _, gh_full[a:b] = oracle.aggregate(offs, level, neg, sc_h, cfg.bits, l0=l, l1=l + 1, window=True)
+    _, sc2_ref, _, _ = oracle.requantize(offs, gh_full, cfg.bits, cfg.seed, step, stream=cfg.M, rng_bits=cfg.rng_bits)
+    out, _, _, _ = oracle.requantize(offs, gh_full, cfg.bits, cfg.seed, step, stream=cfg.M, rng_bits=cfg.rng_bits, scales_in=sc2_h)
+    gh_h, th_h, mo_h = np_of(gh), np_of(theta), np_of(mom)
+    norms_h = np_of(norms).reshape(-1, 2)
+    for l in sample:
+        a, b = int(offs[l]), int(offs[l + 1])
+        assert ulp_diff(sc2_h[l:l + 1], sc2_ref[l:l + 1]).max() <= 1
+        assert np.array_equal(gh_h[a:b].view(np.uint32), out[a:b].view(np.uint32)), "layer %d: the receiver's value" % l
+        th_ref, mo_ref, n_ref = oracle.lalr(offs, np_of(th0[a:b]), np_of(mo0[a:b]), out[a:b], *hp, l0=l, l1=l + 1, window=True)
+        assert np.array_equal(mo_h[a:b].view(np.uint32), mo_ref.view(np.uint32)), "layer %d momentum" % l
+        assert ulp_diff(norms_h[l], n_ref[l]).max() <= 1
+        assert_close_per_layer(th_h[a:b], th_ref, np.array([0, b - a]), "theta layer %d" % l)
