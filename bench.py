@@ -474,6 +474,7 @@ def run_sharded(args):
     hp = (cfg.lr, cfg.momentum, cfg.weight_decay, cfg.c_l, cfg.c_u)
     ops = CudaOps(api, cfg.offsets, cfg.M, M_loc, rank, world, cfg.bits, cfg.rng_bits)
     st = ShardedStep(ops, cfg.offsets, cfg.M, rank, world)
+    do_step = st.step_pull if args.exchange == "pull" else st.step
     mom_own = mom[st.own.a8:st.own.b].clone()
     stream = torch.cuda.current_stream()
 
@@ -484,7 +485,7 @@ def run_sharded(args):
 
     step_no = 0
     for _ in range(max(args.warmup, 3)):
-        st.step(theta, mom_own, grads, cfg.seed, step_no, hp)
+        do_step(theta, mom_own, grads, cfg.seed, step_no, hp)
         step_no += 1
     K = args.steps
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -493,7 +494,7 @@ def run_sharded(args):
     sampler.start()
     e0.record(stream)
     for _ in range(K):
-        st.step(theta, mom_own, grads, cfg.seed, step_no, hp)
+        do_step(theta, mom_own, grads, cfg.seed, step_no, hp)
         step_no += 1
     e1.record(stream)
     barrier()
@@ -509,7 +510,7 @@ def run_sharded(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": dict(workload_config(cfg, "inputs larger than L2, no flush"), parallelism="sharded: %d worker(s) and one layer range per rank" % M_loc,
+            "config": dict(workload_config(cfg, "inputs larger than L2, no flush"), parallelism="sharded: %d worker(s) and one layer range per rank, exchange %s" % (M_loc, args.exchange),
                            path="sharded (dat_worker_norms, dat_quantize, plane exchange, dat_aggregate, dat_lalr_step, theta broadcast)"),
             "roofline": None, "cpu_baseline": None, "e2e": None,
             "sent_plane_bytes_per_rank_and_step": int(own_bytes), "clocks": clocks, "outputs_finite": finite,
@@ -541,6 +542,9 @@ def main():
     ap.add_argument("--sharded", action="store_true",
                     help="the step sharded over the --gpus ranks (layer ranges owned by ranks, planes exchanged, "
                          "theta broadcast) instead of independent replicas; the M workers are divided over the ranks")
+    ap.add_argument("--exchange", default="sendrecv", choices=["sendrecv", "pull"],
+                    help="with --sharded: planes sent to their owners (NCCL point-to-point), or left in symmetric memory "
+                         "and read from there by the owner's aggregation kernel (dat_aggregate_gather)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

@@ -199,6 +199,18 @@ int dat_worker_norms(dat_plan_t *plan, const float *const *grads, float *norms_o
 int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint8_t *signs,
                   const float *scales, int32_t *code_sum, float *g_hat, void *stream);
 
+/* dat_aggregate_gather -- dat_aggregate with one pointer per worker instead of one buffer: worker i's level
+ * plane at level_planes[i] (level_bytes_per_worker bytes) and sign plane at sign_planes[i].  The planes may lie
+ * in this GPU's memory or in a peer GPU's memory that is mapped into the process (peer access, an IPC or
+ * symmetric-memory mapping): the kernel reads them with plain loads, so the owner of a layer range of a sharded
+ * step pulls the other ranks' messages over NVLink while it sums them -- exchange and Step 9 in one kernel.
+ * The caller guarantees that the planes are complete before the call's work starts (a barrier between the
+ * ranks) and are not rewritten before it ends.
+ *   level_planes, sign_planes   host arrays of M device pointers, each 16-byte aligned, read-only.
+ * Other arguments, results (bit for bit) and errors as dat_aggregate. */
+int dat_aggregate_gather(dat_plan_t *plan, const uint8_t *const *level_planes, const uint8_t *const *sign_planes,
+                         const float *scales, int32_t *code_sum, float *g_hat, void *stream);
+
 /* ---------------------------------------------------------------------------------------------
  * dat_requantize -- Algorithm A1 Step 10 (two-sided quantisation, the parameter-server setting):
  * the server quantizes the aggregate once more before sending it back, g_hat <- Q(g_hat).

@@ -30,7 +30,7 @@ DAT_STATIC_MAX_LAYERS, DAT_STATIC_MAX_TILES = 4096, 32768
 DAT_STATUS_NONFINITE, DAT_STATUS_TIMEOUT, DAT_STATUS_BOUNDS = 1, 2, 4
 
 # every symbol include/dat.h declares
-EXPORTS = ["dat_plan_create", "dat_plan_set_origin", "dat_plan_destroy", "dat_plan_sizes", "dat_worker_norms", "dat_quantize", "dat_aggregate", "dat_requantize",
+EXPORTS = ["dat_plan_create", "dat_plan_set_origin", "dat_plan_destroy", "dat_plan_sizes", "dat_worker_norms", "dat_quantize", "dat_aggregate", "dat_aggregate_gather", "dat_requantize",
            "dat_average", "dat_lalr_step", "dat_lamb_step", "dat_lalr_step_static", "dat_step", "dat_step_lamb", "dat_step_two_sided", "dat_step_lamb_two_sided", "dat_step_passes", "dat_step_pipelined", "dat_plan_test_stall", "dat_step_host", "dat_get_status",
            "dat_plan_launch_count", "dat_strerror", "dat_last_cuda_error"]
 
@@ -53,6 +53,7 @@ _lib.dat_worker_norms.argtypes = [_p, _p, _p, _p]
 _lib.dat_plan_sizes.argtypes = [_p, C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64), C.POINTER(_i64)]
 _lib.dat_quantize.argtypes = [_p, _p, _u64, _u64, _p, _p, _p, _p, _p]
 _lib.dat_aggregate.argtypes = [_p, _p, _p, _p, _p, _p, _p]
+_lib.dat_aggregate_gather.argtypes = [_p, _p, _p, _p, _p, _p, _p]
 _lib.dat_requantize.argtypes = [_p, _p, _u64, _u64, _p, _p, _p, _p, _p]
 _lib.dat_average.argtypes = [_p, _p, _p, _p]
 _lib.dat_lalr_step.argtypes = [_p, _p, _p, _p, C.POINTER(dat_hparams_t), _p, _p]
@@ -160,6 +161,12 @@ def dat_quantize(plan, grads, seed, step, levels, signs, scales, scales_in=None,
 def dat_aggregate(plan, levels, signs, scales, code_sum, g_hat, stream=None):
     _ok(_lib.dat_aggregate(_p(plan), _ptr(levels), _ptr(signs), _ptr(scales), _ptr(code_sum), _ptr(g_hat),
                            _stream(stream)), "dat_aggregate")
+
+
+def dat_aggregate_gather(plan, level_planes, sign_planes, scales, code_sum, g_hat, stream=None):
+    """level_planes, sign_planes: M tensors (or addresses), worker i's planes each."""
+    _ok(_lib.dat_aggregate_gather(_p(plan), _ptr_array(level_planes), _ptr_array(sign_planes), _ptr(scales),
+                                  _ptr(code_sum), _ptr(g_hat), _stream(stream)), "dat_aggregate_gather")
 
 
 def dat_requantize(plan, g_hat, seed, step, levels, signs, scales, scales_in=None, stream=None):

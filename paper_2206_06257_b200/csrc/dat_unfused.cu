@@ -289,10 +289,24 @@ __device__ __forceinline__ void dat_unpack8(const uint8_t *__restrict__ plane, i
     }
 }
 
-template <int BITS>
+// Where the M workers' planes are: one buffer with worker i at i * level_bytes (what dat_quantize writes), or
+// one pointer per worker -- this GPU's memory or a peer's mapped into the process, read with plain loads:
+// the owner of a layer range pulls the other ranks' planes itself instead of waiting for them to be sent.
+struct PlanesFlat {
+    const uint8_t *levels, *signs;
+    int64_t level_bytes, sign_bytes;
+    __device__ __forceinline__ const uint8_t *lv(int i) const { return levels + (int64_t)i * level_bytes; }
+    __device__ __forceinline__ const uint8_t *sg(int i) const { return signs + (int64_t)i * sign_bytes; }
+};
+struct PlanesTable {
+    const uint8_t *levels[DAT_MAX_WORKERS], *signs[DAT_MAX_WORKERS];
+    __device__ __forceinline__ const uint8_t *lv(int i) const { return levels[i]; }
+    __device__ __forceinline__ const uint8_t *sg(int i) const { return signs[i]; }
+};
+
+template <int BITS, class SRC>
 __global__ void __launch_bounds__(DAT_THREADS)
-k_aggregate(const uint8_t *__restrict__ levels, const uint8_t *__restrict__ signs, int64_t level_bytes,
-            int64_t sign_bytes, int M, const int64_t *__restrict__ off, int h, int64_t d,
+k_aggregate(const __grid_constant__ SRC src, int M, const int64_t *__restrict__ off, int h, int64_t d,
             const float *__restrict__ dq, int32_t *__restrict__ code_sum, float *__restrict__ g_hat)
 {
     __shared__ int s_first;
@@ -307,8 +321,8 @@ k_aggregate(const uint8_t *__restrict__ levels, const uint8_t *__restrict__ sign
 #pragma unroll 4
     for (int i = 0; i < M; ++i) {                // four workers' loads in flight at a time
         uint32_t lev[8];
-        dat_unpack8<BITS>(levels + (int64_t)i * level_bytes, e0, lev);
-        const uint32_t sg = signs[(int64_t)i * sign_bytes + (e0 >> 3)];
+        dat_unpack8<BITS>(src.lv(i), e0, lev);
+        const uint32_t sg = src.sg(i)[e0 >> 3];
 #pragma unroll
         for (int j = 0; j < 8; ++j) sum[j] += ((sg >> j) & 1u) ? -(int)lev[j] : (int)lev[j];
     }
@@ -344,10 +358,9 @@ k_aggregate(const uint8_t *__restrict__ levels, const uint8_t *__restrict__ sign
 // The same with one norm per worker (Eq. grad_agg as written): no integer sum exists;
 // g_hat = (sum_i nu_{i,l} * signed level_i) / (S*M), accumulated in fp32 with one fused
 // multiply-add per worker, in ascending worker order.
-template <int BITS>
+template <int BITS, class SRC>
 __global__ void __launch_bounds__(DAT_THREADS)
-k_aggregate_per_worker(const uint8_t *__restrict__ levels, const uint8_t *__restrict__ signs, int64_t level_bytes,
-                       int64_t sign_bytes, int M, const int64_t *__restrict__ off, int h, int64_t d,
+k_aggregate_per_worker(const __grid_constant__ SRC src, int M, const int64_t *__restrict__ off, int h, int64_t d,
                        const float *__restrict__ scales, float SM_f, float *__restrict__ g_hat)
 {
     __shared__ int s_first;
@@ -376,8 +389,8 @@ k_aggregate_per_worker(const uint8_t *__restrict__ levels, const uint8_t *__rest
 #pragma unroll 1
     for (int i = 0; i < M; ++i) {
         uint32_t lev[8];
-        dat_unpack8<BITS>(levels + (int64_t)i * level_bytes, e0, lev);
-        const uint32_t sg = signs[(int64_t)i * sign_bytes + (e0 >> 3)];
+        dat_unpack8<BITS>(src.lv(i), e0, lev);
+        const uint32_t sg = src.sg(i)[e0 >> 3];
         const float *__restrict__ nu_i = scales + (int64_t)i * h;
         const float nu0 = __ldg(nu_i + lidx[0]);
 #pragma unroll
@@ -449,8 +462,8 @@ extern "C" int dat_requantize(dat_plan_t *plan, float *g_hat, uint64_t seed, uin
                                                     signs, plan->level_bytes, plan->sign_bytes,                     \
                                                     plan->rng_bits == 16, false, plan->worker_base + (uint32_t)plan->M, plan->elem_base); \
         DAT_LAUNCHED(plan);                                                                                         \
-        k_aggregate<B><<<agrid, DAT_THREADS, 0, s>>>(levels, signs, plan->level_bytes, plan->sign_bytes, 1,          \
-                                                     plan->d_offsets, h, plan->d, plan->d_dq, nullptr, g_hat);      \
+        k_aggregate<B, PlanesFlat><<<agrid, DAT_THREADS, 0, s>>>(PlanesFlat{levels, signs, plan->level_bytes, plan->sign_bytes}, 1, \
+                                                                 plan->d_offsets, h, plan->d, plan->d_dq, nullptr, g_hat); \
     } while (0)
     switch (plan->bits) {
     case 1: DAT_RQ(1); break;
@@ -464,16 +477,9 @@ extern "C" int dat_requantize(dat_plan_t *plan, float *g_hat, uint64_t seed, uin
     return DAT_OK;
 }
 
-extern "C" int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint8_t *signs,
-                             const float *scales, int32_t *code_sum, float *g_hat, void *stream)
+template <class SRC>
+static int aggregate_launch(dat_plan_t *plan, const SRC &src, const float *scales, int32_t *code_sum, float *g_hat, void *stream)
 {
-    int rc = dat_check_plan(plan);
-    if (rc != DAT_OK) return rc;
-    if (plan->bits == 32) return DAT_ERR_BITS;
-    if (!levels || !signs || !scales || !g_hat) return DAT_ERR_ARG;
-    if (!dat_aligned16(levels) || !dat_aligned16(signs) || !dat_aligned16(scales) || !dat_aligned16(g_hat) ||
-        (code_sum && !dat_aligned16(code_sum)))
-        return DAT_ERR_ALIGN;
     cudaStream_t s = (cudaStream_t)stream;
     const int h = (int)plan->h;
     const float SM_f = (float)((uint64_t)plan->S * (uint64_t)plan->M);
@@ -481,8 +487,7 @@ extern "C" int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint
     if (plan->scale_mode == DAT_SCALE_PER_WORKER) {
         if (code_sum) return DAT_ERR_ARG;        // differently scaled codes have no integer sum
 #define DAT_APW(B)                                                                                                  \
-    k_aggregate_per_worker<B><<<grid, DAT_THREADS, 0, s>>>(levels, signs, plan->level_bytes, plan->sign_bytes, plan->M, \
-                                                           plan->d_offsets, h, plan->d, scales, SM_f, g_hat)
+    k_aggregate_per_worker<B, SRC><<<grid, DAT_THREADS, 0, s>>>(src, plan->M, plan->d_offsets, h, plan->d, scales, SM_f, g_hat)
         switch (plan->bits) {
         case 1: DAT_APW(1); break;
         case 2: DAT_APW(2); break;
@@ -497,8 +502,7 @@ extern "C" int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint
     k_dq_from_scales<<<(h + 255) / 256, 256, 0, s>>>(h, SM_f, scales, plan->d_dq);
     DAT_LAUNCHED(plan);
 #define DAT_A(B)                                                                                         \
-    k_aggregate<B><<<grid, DAT_THREADS, 0, s>>>(levels, signs, plan->level_bytes, plan->sign_bytes, plan->M, \
-                                                plan->d_offsets, h, plan->d, plan->d_dq, code_sum, g_hat)
+    k_aggregate<B, SRC><<<grid, DAT_THREADS, 0, s>>>(src, plan->M, plan->d_offsets, h, plan->d, plan->d_dq, code_sum, g_hat)
     switch (plan->bits) {
     case 1: DAT_A(1); break;
     case 2: DAT_A(2); break;
@@ -509,6 +513,38 @@ extern "C" int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint
 #undef DAT_A
     DAT_LAUNCHED(plan);
     return DAT_OK;
+}
+
+extern "C" int dat_aggregate(dat_plan_t *plan, const uint8_t *levels, const uint8_t *signs,
+                             const float *scales, int32_t *code_sum, float *g_hat, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (plan->bits == 32) return DAT_ERR_BITS;
+    if (!levels || !signs || !scales || !g_hat) return DAT_ERR_ARG;
+    if (!dat_aligned16(levels) || !dat_aligned16(signs) || !dat_aligned16(scales) || !dat_aligned16(g_hat) ||
+        (code_sum && !dat_aligned16(code_sum)))
+        return DAT_ERR_ALIGN;
+    return aggregate_launch(plan, PlanesFlat{levels, signs, plan->level_bytes, plan->sign_bytes}, scales, code_sum, g_hat, stream);
+}
+
+extern "C" int dat_aggregate_gather(dat_plan_t *plan, const uint8_t *const *level_planes, const uint8_t *const *sign_planes,
+                                    const float *scales, int32_t *code_sum, float *g_hat, void *stream)
+{
+    int rc = dat_check_plan(plan);
+    if (rc != DAT_OK) return rc;
+    if (plan->bits == 32) return DAT_ERR_BITS;
+    if (!level_planes || !sign_planes || !scales || !g_hat) return DAT_ERR_ARG;
+    if (!dat_aligned16(scales) || !dat_aligned16(g_hat) || (code_sum && !dat_aligned16(code_sum))) return DAT_ERR_ALIGN;
+    PlanesTable t;
+    for (int i = 0; i < DAT_MAX_WORKERS; ++i) { t.levels[i] = nullptr; t.signs[i] = nullptr; }
+    for (int i = 0; i < plan->M; ++i) {
+        if (!level_planes[i] || !sign_planes[i]) return DAT_ERR_ARG;
+        if (!dat_aligned16(level_planes[i]) || !dat_aligned16(sign_planes[i])) return DAT_ERR_ALIGN;
+        t.levels[i] = level_planes[i];
+        t.signs[i] = sign_planes[i];
+    }
+    return aggregate_launch(plan, t, scales, code_sum, g_hat, stream);
 }
 
 // Eq. grad_agg with Q = identity: ordered fp32 sum over workers, then one division by M.

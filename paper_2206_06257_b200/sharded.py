@@ -13,6 +13,11 @@ de-quantised (Step 9), and every machine applies the update (Step 12).  Here:
     layer-wise update to its range of theta and m (all layer norms are local to the owner);
   * the updated ranges of theta are broadcast by their owners.
 
+Two forms of the exchange: "sendrecv" (above), and "pull": every rank leaves its planes in a buffer of its own
+that the other ranks have mapped (symmetric memory), and the owner's aggregation kernel reads the M workers'
+planes of its range from where they lie -- its own memory and the peers' -- with plain loads
+(dat_aggregate_gather): exchange and Step 9 in one kernel, nothing is sent.
+
 Only the orchestration lives here; the arithmetic is done by an `ops` object -- `CudaOps` below calls
 the CUDA library through the C ABI (dat_worker_norms, dat_quantize with caller-supplied norms,
 dat_aggregate, dat_lalr_step on plans that cover one range each, with dat_plan_set_origin giving the
@@ -107,6 +112,69 @@ class ShardedStep:
         self.ops.aggregate_update(own, lv_all, sg_all, own.scales(nu), theta_own, mom_own, hp)
         theta[own.a:own.b].copy_(theta_own[own.pad:])
 
+    def update_pull(self, nu, planes_by_src, theta, mom_own, hp):
+        """Steps 9 and 12 on the owned range, the planes read where the ranks left them: planes_by_src[src] =
+        (levels, signs) of rank src's M/G workers for THIS rank's range (tensors, or base addresses of mapped
+        peer memory)."""
+        own = self.own
+        lb, sb = self.ops.plane_bytes(own)
+        lv_ptrs, sg_ptrs = [], []
+        for src in range(self.world):
+            lv, sg = planes_by_src[src]
+            lv0 = lv.data_ptr() if isinstance(lv, torch.Tensor) else int(lv)
+            sg0 = sg.data_ptr() if isinstance(sg, torch.Tensor) else int(sg)
+            lv_ptrs += [lv0 + j * lb for j in range(self.M_loc)]         # global worker order: rank-major
+            sg_ptrs += [sg0 + j * sb for j in range(self.M_loc)]
+        theta_own = theta[own.a8:own.b].clone()
+        self.ops.aggregate_update_gather(own, lv_ptrs, sg_ptrs, own.scales(nu), theta_own, mom_own, hp)
+        theta[own.a:own.b].copy_(theta_own[own.pad:])
+
+    def _pull_layout(self):
+        """Byte offsets, in every rank's outgoing buffer, of the level and sign planes meant for owner q."""
+        offs, at = [], 0
+        for q in range(self.world):
+            lb, sb = self.ops.plane_bytes(self.ranges[q])
+            offs.append((at, at + self.M_loc * lb))
+            at += self.M_loc * (lb + sb)                                  # (plane sizes are multiples of 16 bytes)
+        return offs, at
+
+    def step_pull(self, theta, mom_own, grads_local, seed, step, hp):
+        """The step with the "pull" exchange.  Needs CUDA ranks of one node with peer access.  Not run on more
+        than one GPU so far (one-GPU environment): the kernel path is covered by driving several ranks' objects
+        in one process, the mapping of the peers' buffers is not."""
+        layout, total = self._pull_layout()
+        multi = self.world > 1
+        if getattr(self, "_out", None) is None:
+            if multi:
+                import os
+                os.environ.setdefault("TORCH_SYMM_MEM_DISABLE_MULTICAST", "1")    # plain peer mappings, no NVLink multicast object
+                import torch.distributed._symmetric_memory as symm_mem
+                self._out = symm_mem.empty(total, dtype=torch.uint8, device=theta.device)
+                hdl = symm_mem.rendezvous(self._out, self.group if self.group is not None else dist.group.WORLD)
+                self._bases = [int(p) for p in hdl.buffer_ptrs]
+            else:
+                self._out = torch.empty(total, dtype=torch.uint8, device=theta.device)
+                self._bases = [self._out.data_ptr()]
+        nu = self.local_norms(grads_local)
+        if multi:
+            dist.all_reduce(nu, op=dist.ReduceOp.MAX, group=self.group)
+        for q in range(self.world):
+            lb, sb = self.ops.plane_bytes(self.ranges[q])
+            lo, so = layout[q]
+            self.ops.quantize_range(q, self.ranges[q], grads_local, self.ranges[q].scales(nu), seed, step,
+                                    out=(self._out[lo:lo + self.M_loc * lb], self._out[so:so + self.M_loc * sb]))
+        if multi:
+            torch.cuda.current_stream().synchronize()
+            dist.barrier(group=self.group)                                # every rank's planes are complete
+        lo, so = layout[self.rank]
+        self.update_pull(nu, [(b + lo, b + so) for b in self._bases], theta, mom_own, hp)
+        if multi:
+            torch.cuda.current_stream().synchronize()
+            dist.barrier(group=self.group)                                # nobody rewrites planes that are still being read
+            for r, rg in enumerate(self.ranges):
+                dist.broadcast(theta[rg.a:rg.b], src=r, group=self.group)
+        return nu
+
     def step(self, theta, mom_own, grads_local, seed, step, hp):
         """theta: the full parameter vector (updated in place on every rank); mom_own: the momentum of this
         rank's range, own.n elements with the pad in front (updated in place); grads_local: this rank's
@@ -170,15 +238,21 @@ class CudaOps:
         self.api.dat_worker_norms(self.plan_norms, grads_local, out)
         return out.view(self.M_loc, self.h)
 
-    def quantize_range(self, q, rg, grads_local, scales, seed, step):
+    def quantize_range(self, q, rg, grads_local, scales, seed, step, out=None):
         plan = self._plan(self.plans_q, rg, self.M_loc, self.rank * self.M_loc)
         lb, sb, ns, _ = self.api.dat_plan_sizes(plan)
         dev = grads_local[0].device
-        lv = torch.empty(self.M_loc * lb, dtype=torch.uint8, device=dev)
-        sg = torch.empty(self.M_loc * sb, dtype=torch.uint8, device=dev)
+        lv, sg = out if out is not None else (torch.empty(self.M_loc * lb, dtype=torch.uint8, device=dev),
+                                              torch.empty(self.M_loc * sb, dtype=torch.uint8, device=dev))
         sc = torch.empty(ns, dtype=torch.float32, device=dev)
         self.api.dat_quantize(plan, [g[rg.a8:rg.b] for g in grads_local], seed, step, lv, sg, sc, scales_in=scales.contiguous())
         return lv, sg
+
+    def aggregate_update_gather(self, rg, lv_ptrs, sg_ptrs, scales, theta_own, mom_own, hp):
+        plan = self._plan(self.plans_agg, rg, self.M, 0)
+        g_hat = torch.empty(rg.n, dtype=torch.float32, device=theta_own.device)
+        self.api.dat_aggregate_gather(plan, lv_ptrs, sg_ptrs, scales.contiguous(), None, g_hat)
+        self.api.dat_lalr_step(plan, theta_own, mom_own, g_hat, hp)
 
     def aggregate_update(self, rg, lv_all, sg_all, scales, theta_own, mom_own, hp):
         plan = self._plan(self.plans_agg, rg, self.M, 0)

@@ -285,6 +285,41 @@ def test_step_lamb_parity_three_steps(api, oracle, mode):
         assert e.value.code == api.DAT_ERR_ARG
 
 
+@pytest.mark.parametrize("mode", ["shared", "per_worker"])
+@pytest.mark.parametrize("bits", [1, 2, 4, 8, 16])
+def test_aggregate_gather_equals_aggregate(api, oracle, bits, mode):
+    """dat_aggregate_gather: every worker's planes in a buffer of its own (as a peer would hold them); the
+    result is dat_aggregate's bit for bit, and the oracle's."""
+    M = 5
+    sm = oracle.SCALE_PER_WORKER if mode == "per_worker" else oracle.SCALE_SHARED_MAX
+    offs, grads, _, _ = _random_problem(60 + bits, SIZES_RAGGED, M)
+    d = int(offs[-1])
+    with GpuPlan(api, offs, M, bits, 16, scale_mode=api.DAT_SCALE_PER_WORKER if mode == "per_worker" else 0) as P:
+        lv, sg, sc = P.alloc_message()
+        api.dat_quantize(P.plan, [torch.from_numpy(g).cuda() for g in grads], 3, 5, lv, sg, sc)
+        lb, sb, _, _ = api.dat_plan_sizes(P.plan)
+        pad = torch.empty(48, dtype=torch.uint8, device="cuda")          # (separate allocations, in scrambled order)
+        lvs = [lv[i * lb:(i + 1) * lb].clone() for i in reversed(range(M))][::-1]
+        sgs = [sg[i * sb:(i + 1) * sb].clone() for i in range(M)]
+        cs1 = None if mode == "per_worker" else torch.zeros(d, dtype=torch.int32, device="cuda")
+        cs2 = None if mode == "per_worker" else torch.zeros(d, dtype=torch.int32, device="cuda")
+        g1, g2 = torch.zeros(d, device="cuda"), torch.zeros(d, device="cuda")
+        api.dat_aggregate(P.plan, lv, sg, sc, cs1, g1)
+        api.dat_aggregate_gather(P.plan, lvs, sgs, sc, cs2, g2)
+        torch.cuda.synchronize()
+        assert torch.equal(g1, g2) and (cs1 is None or torch.equal(cs1, cs2))
+        level, neg = oracle.quantize(offs, grads, bits, 3, 5, np_of(sc), sm, rng_bits=16)
+        _, gh = oracle.aggregate(offs, level, neg, np_of(sc), bits, sm)
+        assert np.array_equal(np_of(g2).view(np.uint32), gh.view(np.uint32))
+        with pytest.raises(api.DatError) as e:                           # a worker without planes
+            api.dat_aggregate_gather(P.plan, lvs[:-1] + [None], sgs, sc, None, g2)
+        assert e.value.code == api.DAT_ERR_ARG
+        with pytest.raises(api.DatError) as e:                           # a plane that is not 16-byte aligned
+            api.dat_aggregate_gather(P.plan, [lvs[0].data_ptr() + 4] + lvs[1:], sgs, sc, None, g2)
+        assert e.value.code == api.DAT_ERR_ALIGN
+        del pad
+
+
 def _two_sided_reference(oracle, offs, grads, bits, seed, step, M, sm, rng_bits, sc_gpu, sc2_gpu):
     """Steps 7, 9 and 10 from the oracle's own operations: the workers' levels with the GPU's quantizer norms,
     the aggregate, the server's Q(g_hat) with the GPU's server norms (each norm checked to the last place first)."""

@@ -102,8 +102,9 @@ def test_sharded_step_on_gloo_ranks_equals_the_unsharded_oracle(oracle, world, M
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("exchange", ["sendrecv", "pull"])
 @pytest.mark.parametrize("world,M,bits", [(2, 4, 8), (4, 8, 2)])
-def test_sharded_step_cuda_ops_in_one_process(oracle, world, M, bits):
+def test_sharded_step_cuda_ops_in_one_process(oracle, world, M, bits, exchange):
     """The CUDA operations of the sharded step: `world` ranks' objects on one device, driven phase by phase."""
     sys.path.insert(0, ROOT)
     from paper_2206_06257_b200 import api
@@ -121,6 +122,9 @@ def test_sharded_step_cuda_ops_in_one_process(oracle, world, M, bits):
         nu = torch.stack(nus).max(dim=0).values                          # the all-reduce(max)
         planes = [s.quantize(nu, g[r], 11, 3) for r, s in enumerate(ranks)]
         for r, s in enumerate(ranks):
+            if exchange == "pull":      # the owner's kernel reads every rank's planes where that rank left them
+                s.update_pull(nu, [planes[src][r] for src in range(world)], th[r], mo[r], HP)
+                continue
             lv_all, sg_all = s.receive_buffers(nu.device)
             for src in range(world):                                     # the point-to-point exchange
                 lv_dst, sg_dst = s.slot(lv_all, sg_all, src)
