@@ -317,10 +317,13 @@ int dat_lalr_step_static(int64_t num_layers, const int64_t *layer_offsets, float
  * usual, DAT_STATUS_TIMEOUT is set in the status word, and the outputs of that call -- and of
  * later calls on the plan -- are undefined until dat_get_status has been called, which reports the
  * bit and restores the plan's counters.
+ * The call cannot be recorded into a CUDA graph (its epoch and the key of its random streams are launch
+ * parameters, which a replay would repeat): while `stream` is capturing it answers DAT_ERR_UNSUPPORTED and
+ * enqueues nothing.  The same holds for dat_step_lamb, dat_step_two_sided and dat_step_lamb_two_sided.
  * With a DAT_SCALE_PER_WORKER plan the step follows Eq. grad_agg as written (every worker on its own grid,
  * fp32 sum in ascending worker order): scales_out then has M*h entries (index i*h + l) and code_sum_out is
  * ignored (no integer sums exist).
- * Errors: ARG, ALIGN, CUDA.
+ * Errors: ARG, ALIGN, UNSUPPORTED (plan with an origin; capturing stream), CUDA.
  * ------------------------------------------------------------------------------------------- */
 int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
              uint64_t seed, uint64_t step, const dat_hparams_t *hp,

@@ -897,6 +897,11 @@ static int p_launch(dat_plan_t *plan, float *theta, float *mom, float *var, cons
         (g_hat && !dat_aligned16(g_hat)) || (server_scales_out && !dat_aligned16(server_scales_out)))
         return DAT_ERR_ALIGN;
     const bool two = (g_hat != nullptr);
+    {   // the call's epoch and the Philox key are launch parameters: a captured graph would replay them unchanged
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing((cudaStream_t)stream, &cap) != cudaSuccess) { (void)cudaGetLastError(); return DAT_ERR_CUDA; }
+        if (cap != cudaStreamCaptureStatusNone) return DAT_ERR_UNSUPPORTED;
+    }
     if (two && plan->bits == 32) return DAT_ERR_BITS;      // nothing to quantize with
     PArgs a;
     int rc = dat_check_grads(plan, grads, &a.gp);

@@ -320,6 +320,95 @@ def test_aggregate_gather_equals_aggregate(api, oracle, bits, mode):
         del pad
 
 
+class _Guarded:
+    """Buffers cut out of larger ones whose margins hold a pattern: nothing may write outside what it was given."""
+    MARGIN = 256                                                    # bytes on either side (keeps 16-byte alignment)
+
+    def __init__(self):
+        self.items = []
+
+    def make(self, n, dtype, fill=0):
+        nbytes = n * torch.empty((), dtype=dtype).element_size()
+        whole = torch.full((nbytes + 2 * self.MARGIN,), 0x5A, dtype=torch.uint8, device="cuda")
+        body = whole[self.MARGIN:self.MARGIN + nbytes]
+        body.fill_(0)
+        view = body.view(dtype)
+        if fill:
+            view.fill_(fill)
+        self.items.append(whole)
+        return view
+
+    def check(self):
+        torch.cuda.synchronize()
+        for whole in self.items:
+            assert bool((whole[:self.MARGIN] == 0x5A).all()) and bool((whole[-self.MARGIN:] == 0x5A).all()), "a write outside a buffer"
+
+
+@pytest.mark.parametrize("bits", [1, 4, 8])
+def test_nothing_is_written_outside_the_callers_buffers(api, bits, rng_bits):
+    """Every output of every entry point sits between two margins of a known pattern; ragged layers, M = 3."""
+    M = 3
+    offs, grads, theta, mom = _random_problem(70 + bits, SIZES_RAGGED, M)
+    d, h = int(offs[-1]), len(offs) - 1
+    gs = [torch.from_numpy(g).cuda() for g in grads]
+    for scale_mode in (0, api.DAT_SCALE_PER_WORKER):
+        with GpuPlan(api, offs, M, bits, rng_bits, scale_mode=scale_mode) as P:
+            lb, sb, ns, _ = api.dat_plan_sizes(P.plan)
+            G = _Guarded()
+            lv, sg, sc = G.make(M * lb, torch.uint8), G.make(M * sb, torch.uint8), G.make(ns, torch.float32)
+            wn = G.make(M * h, torch.float32)
+            cs = None if scale_mode else G.make(d, torch.int32)
+            gh, gh2 = G.make(d, torch.float32), G.make(d, torch.float32)
+            th, mo, va = G.make(d, torch.float32), G.make(d, torch.float32), G.make(d, torch.float32)
+            th.copy_(torch.from_numpy(theta)); mo.copy_(torch.from_numpy(mom))
+            norms, sc_out, sc2 = G.make(2 * h, torch.float32), G.make(ns, torch.float32), G.make(h, torch.float32)
+            slv, ssg, ssc = G.make(lb, torch.uint8), G.make(sb, torch.uint8), G.make(h, torch.float32)
+            api.dat_worker_norms(P.plan, gs, wn)
+            api.dat_quantize(P.plan, gs, 3, 0, lv, sg, sc)
+            api.dat_aggregate(P.plan, lv, sg, sc, cs, gh)
+            api.dat_aggregate_gather(P.plan, [lv[i * lb:(i + 1) * lb] for i in range(M)], [sg[i * sb:(i + 1) * sb] for i in range(M)], sc, cs, gh)
+            api.dat_requantize(P.plan, gh, 3, 0, slv, ssg, ssc)
+            api.dat_lalr_step(P.plan, th, mo, gh, HP, norms)
+            api.dat_lamb_step(P.plan, th, mo, va, gh, LAMB_HP, 1, norms)
+            api.dat_step(P.plan, th, mo, gs, 3, 1, HP, cs, norms, sc_out)
+            api.dat_step_lamb(P.plan, th, mo, va, gs, 3, 2, LAMB_HP, 2, cs, norms, sc_out)
+            api.dat_step_two_sided(P.plan, th, mo, gs, 3, 3, HP, gh2, cs, norms, sc_out, sc2)
+            api.dat_step_lamb_two_sided(P.plan, th, mo, va, gs, 3, 4, LAMB_HP, 3, gh2, cs, norms, sc_out, sc2)
+            if not scale_mode:
+                api.dat_step_passes(P.plan, th, mo, gs, 3, 5, HP, cs, norms, sc_out)
+            assert P.status() == 0
+            G.check()
+
+
+def test_step_refuses_stream_capture(api):
+    """The one-launch step carries its epoch and its Philox key as launch parameters: it must not end up in a graph."""
+    offs, grads, theta, mom = _random_problem(5, [1000, 5000], 2)
+    with GpuPlan(api, offs, 2, 8, 16) as P:
+        th, mo = torch.from_numpy(theta).cuda(), torch.from_numpy(mom).cuda()
+        gs = [torch.from_numpy(g).cuda() for g in grads]
+        api.dat_step(P.plan, th, mo, gs, 1, 0, HP)
+        torch.cuda.synchronize()
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(s):
+            g.capture_begin()
+            try:
+                th.add_(0.0)                                        # something to capture
+                with pytest.raises(api.DatError) as e:
+                    api.dat_step(P.plan, th, mo, gs, 1, 1, HP, stream=s)
+                assert e.value.code == api.DAT_ERR_UNSUPPORTED
+            finally:
+                g.capture_end()
+        torch.cuda.synchronize()
+        th2, mo2 = th.clone(), mo.clone()
+        api.dat_step(P.plan, th, mo, gs, 1, 1, HP)                  # the plan is as it was
+        with GpuPlan(api, offs, 2, 8, 16) as P2:
+            api.dat_step(P2.plan, th2, mo2, gs, 1, 1, HP)
+            torch.cuda.synchronize()
+        assert torch.equal(th, th2) and torch.equal(mo, mo2)
+
+
 def _two_sided_reference(oracle, offs, grads, bits, seed, step, M, sm, rng_bits, sc_gpu, sc2_gpu):
     """Steps 7, 9 and 10 from the oracle's own operations: the workers' levels with the GPU's quantizer norms,
     the aggregate, the server's Q(g_hat) with the GPU's server norms (each norm checked to the last place first)."""
