@@ -162,3 +162,74 @@ def test_resnet50_two_sided_sampled_layers(oracle):
         assert np.array_equal(mo_h[a:b].view(np.uint32), mo_ref.view(np.uint32)), "layer %d momentum" % l
         assert ulp_diff(norms_h[l], n_ref[l]).max() <= 1
         assert_close_per_layer(th_h[a:b], th_ref, np.array([0, b - a]), "theta layer %d" % l)
+
+
+def _sample_layers(cfg):
+    sizes = np.diff(cfg.offsets)
+    return sorted(set(list(range(0, cfg.h, 9)) + [int(np.argmax(sizes)), int(np.argmin(sizes)), cfg.h - 2, cfg.h - 1]))
+
+
+def test_resnet50_per_worker_norms_sampled_layers(oracle):
+    """dat_step on a plan with one quantizer norm per worker (Eq. grad_agg as written) at the bench size."""
+    from paper_2206_06257_b200 import api, synth
+    cfg = synth.config("resnet50")
+    dev, step = "cuda", 1
+    theta, mom = synth.make_params(cfg, device=dev)
+    grads = synth.make_grads(cfg, step, device=dev)
+    hp = hp_tuple(cfg)
+    th0, mo0 = theta.clone(), mom.clone()
+    sc = torch.zeros(cfg.M * cfg.h, dtype=torch.float32, device=dev)
+    norms = torch.zeros(2 * cfg.h, dtype=torch.float32, device=dev)
+    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits, rng_bits=cfg.rng_bits, scale_mode=api.DAT_SCALE_PER_WORKER)
+    try:
+        api.dat_step(plan, theta, mom, grads, cfg.seed, step, hp, None, norms, sc)
+        torch.cuda.synchronize()
+        assert api.dat_get_status(plan) == 0
+    finally:
+        api.dat_plan_destroy(plan)
+    offs, sc_h = cfg.offsets, np_of(sc)
+    for l in _sample_layers(cfg):
+        a, b = int(offs[l]), int(offs[l + 1])
+        g_l = [np_of(g[a:b]) for g in grads]
+        nu = oracle.worker_norms(offs, g_l, l0=l, l1=l + 1, window=True)
+        assert ulp_diff(sc_h.reshape(cfg.M, cfg.h)[:, l], nu[:, l]).max() <= 1
+        ref = oracle.step(offs, np_of(th0[a:b]), np_of(mo0[a:b]), g_l, cfg.bits, cfg.seed, step, *hp, l0=l, l1=l + 1,
+                          window=True, scale_mode=oracle.SCALE_PER_WORKER, scales_in=sc_h, rng_bits=cfg.rng_bits)
+        assert np.array_equal(np_of(mom[a:b]).view(np.uint32), ref["mom"].view(np.uint32)), "layer %d momentum" % l
+        assert_close_per_layer(np_of(theta[a:b]), ref["theta"], np.array([0, b - a]), "theta layer %d" % l)
+
+
+def test_resnet50_lamb_sampled_layers(oracle):
+    """dat_step_lamb (Algorithm A2 in the one launch) at the bench size, t = 1 and t = 2 on one plan."""
+    from paper_2206_06257_b200 import api, synth
+    cfg = synth.config("resnet50")
+    dev = "cuda"
+    theta, mom = synth.make_params(cfg, device=dev)
+    var = torch.zeros_like(mom)
+    lamb_hp = (cfg.lr, 0.9, 0.999, 1e-6, 1e-4, cfg.c_l, cfg.c_u)
+    sc = torch.zeros(cfg.h, dtype=torch.float32, device=dev)
+    norms = torch.zeros(2 * cfg.h, dtype=torch.float32, device=dev)
+    offs = cfg.offsets
+    plan = api.dat_plan_create(cfg.offsets, cfg.M, cfg.bits, rng_bits=cfg.rng_bits)
+    try:
+        for t in (1, 2):
+            grads = synth.make_grads(cfg, t, device=dev)
+            th0, mo0, va0 = theta.clone(), mom.clone(), var.clone()
+            api.dat_step_lamb(plan, theta, mom, var, grads, cfg.seed, t, lamb_hp, t, None, norms, sc)
+            torch.cuda.synchronize()
+            assert api.dat_get_status(plan) == 0
+            sc_h, norms_h = np_of(sc), np_of(norms).reshape(-1, 2)
+            for l in _sample_layers(cfg):
+                a, b = int(offs[l]), int(offs[l + 1])
+                g_l = [np_of(g[a:b]) for g in grads]
+                nu = oracle.scales(oracle.worker_norms(offs, g_l, l0=l, l1=l + 1, window=True))
+                assert ulp_diff(sc_h[l:l + 1], nu[l:l + 1]).max() <= 1
+                level, neg = oracle.quantize(offs, g_l, cfg.bits, cfg.seed, t, sc_h, l0=l, l1=l + 1, window=True, rng_bits=cfg.rng_bits)
+                _, gh = oracle.aggregate(offs, level, neg, sc_h, cfg.bits, l0=l, l1=l + 1, window=True)
+                th_ref, mo_ref, va_ref, n_ref = oracle.lamb(np.array([0, b - a]), np_of(th0[a:b]), np_of(mo0[a:b]), np_of(va0[a:b]), gh, t, *lamb_hp)
+                assert np.array_equal(np_of(mom[a:b]).view(np.uint32), mo_ref.view(np.uint32)), "layer %d m', t = %d" % (l, t)
+                assert np.array_equal(np_of(var[a:b]).view(np.uint32), va_ref.view(np.uint32)), "layer %d v', t = %d" % (l, t)
+                assert ulp_diff(norms_h[l], n_ref[0]).max() <= 1
+                assert_close_per_layer(np_of(theta[a:b]), th_ref, np.array([0, b - a]), "theta layer %d, t = %d" % (l, t))
+    finally:
+        api.dat_plan_destroy(plan)
