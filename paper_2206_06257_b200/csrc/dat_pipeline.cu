@@ -478,10 +478,18 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
         // arithmetic as p_direction, spelled out so that the loads are issued before g_hat is scaled: the step
         // is 3 % slower with the call.)
         float th[8], m[8];
-        p_load4_cg(a.theta, e0, lo, hi, th);
-        p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
-        p_load4_cg(a.mom, e0, lo, hi, m);
-        p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
+        if (full) {                                 // (evict-first: by the time the U part wants them they are gone anyway)
+            const uint64_t pf = dat_policy_evict_first();
+            const float4 t0 = dat_ld4_hint(a.theta + e0, pf), t1 = dat_ld4_hint(a.theta + e0 + 4, pf);
+            const float4 m0 = dat_ld4_hint(a.mom + e0, pf), m1 = dat_ld4_hint(a.mom + e0 + 4, pf);
+            th[0] = t0.x; th[1] = t0.y; th[2] = t0.z; th[3] = t0.w; th[4] = t1.x; th[5] = t1.y; th[6] = t1.z; th[7] = t1.w;
+            m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
+        } else {
+            p_load4_cg(a.theta, e0, lo, hi, th);
+            p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
+            p_load4_cg(a.mom, e0, lo, hi, m);
+            p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
+        }
         if (MODE == P_MODE_SHARED && a.code_sum) {
 #pragma unroll
             for (int j = 0; j < 8; ++j)
@@ -513,8 +521,14 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
                 ss_u = fma((double)m[j], (double)m[j], ss_u);
             }
         }
-        dat_store4(a.mom, e0, lo, hi, m);
-        dat_store4(a.mom, e0 + 4, lo, hi, m + 4);
+        if (full) {
+            const uint64_t pf = dat_policy_evict_first();
+            dat_st4_hint(a.mom + e0, make_float4(m[0], m[1], m[2], m[3]), pf);
+            dat_st4_hint(a.mom + e0 + 4, make_float4(m[4], m[5], m[6], m[7]), pf);
+        } else {
+            dat_store4(a.mom, e0, lo, hi, m);
+            dat_store4(a.mom, e0 + 4, lo, hi, m + 4);
+        }
     }
     __threadfence();                               // m' (and v'), or g_hat, are read by a later part of another CTA
     ss_theta = dat_warp_sum(ss_theta);
