@@ -333,7 +333,9 @@ int dat_step(dat_plan_t *plan, float *theta, float *mom, const float *const *gra
  * vector is cut into per-layer tiles; a work item holds one tile for each of three phases -- sums of
  * squares for the quantizer norms (N), levels + signed sum + g_hat + m' + layer sums (Q), parameter
  * update (U) -- with the Q tiles running a fixed distance behind the N tiles and the U tiles behind the
- * Q tiles, so that a gradient read for its norm is still in the L2 cache when its level is drawn.
+ * Q tiles, far enough that a part seldom has to wait for the layer-wide result it needs.  The gradients are
+ * read twice (norm, then levels; from the L2 cache the second time only for small layers); codes, sums and
+ * g_hat stay in registers.
  * Same arguments, results and errors as dat_step. */
 int dat_step_pipelined(dat_plan_t *plan, float *theta, float *mom, const float *const *grads,
                        uint64_t seed, uint64_t step, const dat_hparams_t *hp, int32_t *code_sum_out,

@@ -1,14 +1,16 @@
 // dat_step_pipelined: Steps 7, 9 and 12 of Algorithm A1 in ONE launch of ordinary (non-persistent)
-// CTAs that reads every gradient from HBM once.
+// CTAs.  Codes, integer sums and g_hat never reach memory; the gradients are read twice (for the norm, then
+// for the levels), the second time from L2 only where a layer is small enough to still be there.
 //
 // The quantizer norm of a layer (Eq. rand_q) must be known before the first level of that layer
 // (Eq. xi) can be drawn, and the two layer norms of Eq. 3 before the first parameter moves: three
 // phases per layer, each needing the previous one complete for the whole layer.  The flat vector is
 // cut into per-layer tiles, and the host lays three streams of tiles side by side in one list of
 // work items: item s holds (at most) one tile for each phase,
-//     N  sums of squares of the gradients of a tile          (gradients come from HBM),
-//     Q  levels, signed sum, g_hat, m', layer sums of a tile  (the same gradients, now from L2),
-//     U  theta update of a tile                               (theta and m' still in L2),
+//     N  sums of squares of the gradients of a tile          (gradients from HBM, L2 evict-first),
+//     Q  levels, signed sum, g_hat, m', layer sums of a tile  (the same gradients once more: from L2 for
+//                                                             small layers, from HBM for the others),
+//     U  theta update of a tile                               (theta and m' kept in L2 with evict-last),
 // where the Q stream runs behind the N stream, and the U stream behind the Q stream, by the size of
 // the layer plus a fixed number of items.  A CTA takes the next item by an atomic ticket, so items
 // start in list order, and does its N part first: the sums a later item waits for are produced by
@@ -37,7 +39,7 @@
 #define DAT_P_MINB (1024 / DAT_P_THREADS)         // 64 registers per thread
 #endif
 #ifndef DAT_P_LAG                                 // items between the last N tile of a layer and its first Q tile
-#define DAT_P_LAG 256
+#define DAT_P_LAG 384
 #endif
 #ifndef DAT_P_LAG_U                               // items between the last Q tile of a layer and its first U tile
 #define DAT_P_LAG_U DAT_P_LAG
@@ -177,9 +179,10 @@ __device__ __forceinline__ void p_norm_sums(const PArgs &a, const PipePart &pt, 
     int run = u0;
     if (p_tile_inside(pt)) {
 #ifndef DAT_P_N_POLICY
-#define DAT_P_N_POLICY dat_policy_evict_last
+#define DAT_P_N_POLICY dat_policy_evict_first
 #endif
-        const uint64_t pol = DAT_P_N_POLICY();         // the Q part of a later item reads these lines again
+        const uint64_t pol = DAT_P_N_POLICY();         // by the time the Q part of a later item wants these lines they are gone anyway:
+                                                       // better they leave first than push out theta and m', which the U part can still find
 #pragma unroll 1
         for (int ub = u0; ub < u1; ub += UPB) {
             float4 v[8];
@@ -478,9 +481,9 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
         // arithmetic as p_direction, spelled out so that the loads are issued before g_hat is scaled: the step
         // is 3 % slower with the call.)
         float th[8], m[8];
-        if (full) {                                 // (evict-first: by the time the U part wants them they are gone anyway)
-            const uint64_t pf = dat_policy_evict_first();
-            const float4 t0 = dat_ld4_hint(a.theta + e0, pf), t1 = dat_ld4_hint(a.theta + e0 + 4, pf);
+        if (full) {                                 // theta is read again by the U part (evict-last), m is dead (evict-first)
+            const uint64_t pf = dat_policy_evict_first(), pth = dat_policy_evict_last();
+            const float4 t0 = dat_ld4_hint(a.theta + e0, pth), t1 = dat_ld4_hint(a.theta + e0 + 4, pth);
             const float4 m0 = dat_ld4_hint(a.mom + e0, pf), m1 = dat_ld4_hint(a.mom + e0 + 4, pf);
             th[0] = t0.x; th[1] = t0.y; th[2] = t0.z; th[3] = t0.w; th[4] = t1.x; th[5] = t1.y; th[6] = t1.z; th[7] = t1.w;
             m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
@@ -522,7 +525,7 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
             }
         }
         if (full) {
-            const uint64_t pf = dat_policy_evict_first();
+            const uint64_t pf = dat_policy_evict_last();   // the U part of a later item reads m' again
             dat_st4_hint(a.mom + e0, make_float4(m[0], m[1], m[2], m[3]), pf);
             dat_st4_hint(a.mom + e0 + 4, make_float4(m[4], m[5], m[6], m[7]), pf);
         } else {
