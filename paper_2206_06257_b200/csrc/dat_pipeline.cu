@@ -44,6 +44,9 @@
 #ifndef DAT_P_LAG_U                               // items between the last Q tile of a layer and its first U tile
 #define DAT_P_LAG_U DAT_P_LAG
 #endif
+#ifndef DAT_P_KEEP_T                              // layers of at most this many tiles: the first reads stay in L2 for the second
+#define DAT_P_KEEP_T 72
+#endif
 #ifndef DAT_P_REVERSE_FROM                        // layers of at least this many tiles: Q walks back from the last tile
 #define DAT_P_REVERSE_FROM 320
 #endif
@@ -124,6 +127,29 @@ __device__ __forceinline__ void p_load4_cg(const float *__restrict__ p, int64_t 
     }
 }
 
+// Eight consecutive elements with an L2 eviction hint: two 16-byte accesses where the group lies inside the
+// layer, element accesses (no hint) at a layer's ragged ends.
+__device__ __forceinline__ void p_ld8(const float *p, int64_t e0, int64_t lo, int64_t hi, float v[8], uint64_t pol)
+{
+    if (e0 >= lo && e0 + 8 <= hi) {
+        const float4 x = dat_ld4_hint(p + e0, pol), y = dat_ld4_hint(p + e0 + 4, pol);
+        v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
+    } else {
+        p_load4_cg(p, e0, lo, hi, v);
+        p_load4_cg(p, e0 + 4, lo, hi, v + 4);
+    }
+}
+__device__ __forceinline__ void p_st8(float *p, int64_t e0, int64_t lo, int64_t hi, const float v[8], uint64_t pol)
+{
+    if (e0 >= lo && e0 + 8 <= hi) {
+        dat_st4_hint(p + e0, make_float4(v[0], v[1], v[2], v[3]), pol);
+        dat_st4_hint(p + e0 + 4, make_float4(v[4], v[5], v[6], v[7]), pol);
+    } else {
+        dat_store4(p, e0, lo, hi, v);
+        dat_store4(p, e0 + 4, lo, hi, v + 4);
+    }
+}
+
 // One thread: waits until `word` carries this call's epoch.  Bounded: when the limit runs out the status
 // word gets DAT_STATUS_TIMEOUT and the call's abort word is set, which ends every other wait at once.
 // Returns false if the part that needs the word must be skipped.
@@ -181,8 +207,9 @@ __device__ __forceinline__ void p_norm_sums(const PArgs &a, const PipePart &pt, 
 #ifndef DAT_P_N_POLICY
 #define DAT_P_N_POLICY dat_policy_evict_first
 #endif
-        const uint64_t pol = DAT_P_N_POLICY();         // by the time the Q part of a later item wants these lines they are gone anyway:
-                                                       // better they leave first than push out theta and m', which the U part can still find
+        // A small layer's lines are still in L2 when the Q part of a later item reads them again; a large layer's
+        // are gone by then anyway: better they leave first than push out theta and m', which the U part can still find.
+        const uint64_t pol = (pt.T <= DAT_P_KEEP_T) ? dat_policy_evict_normal() : DAT_P_N_POLICY();
 #pragma unroll 1
         for (int ub = u0; ub < u1; ub += UPB) {
             float4 v[8];
@@ -390,16 +417,15 @@ template <int OPT>
 __device__ __forceinline__ void p_direction(const PArgs &a, int64_t e0, int64_t lo, int64_t hi, const float ghat[8],
                                             double &ss_theta, double &ss_u)
 {
+    // what the U part reads again (theta, m', v') is kept in L2 (evict-last); the old m is dead (evict-first)
+    const uint64_t keep = dat_policy_evict_last();
     float th[8], m[8];
-    p_load4_cg(a.theta, e0, lo, hi, th);
-    p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
-    p_load4_cg(a.mom, e0, lo, hi, m);
-    p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
+    p_ld8(a.theta, e0, lo, hi, th, keep);
+    p_ld8(a.mom, e0, lo, hi, m, dat_policy_evict_first());
     if (OPT == P_OPT_LAMB) {
         // Algorithm A2: both moments are stored, the direction is formed on the fly for the layer sums
         float v[8];
-        p_load4_cg(a.var, e0, lo, hi, v);
-        p_load4_cg(a.var, e0 + 4, lo, hi, v + 4);
+        p_ld8(a.var, e0, lo, hi, v, keep);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             m[j] = __fmaf_rn(a.lamb.beta1, m[j], __fmul_rn(a.lamb.om1, ghat[j]));
@@ -409,8 +435,7 @@ __device__ __forceinline__ void p_direction(const PArgs &a, int64_t e0, int64_t 
             ss_theta = fma((double)th[j], (double)th[j], ss_theta);
             ss_u = fma((double)u, (double)u, ss_u);
         }
-        dat_store4(a.var, e0, lo, hi, v);
-        dat_store4(a.var, e0 + 4, lo, hi, v + 4);
+        p_st8(a.var, e0, lo, hi, v, keep);
     } else {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -419,8 +444,7 @@ __device__ __forceinline__ void p_direction(const PArgs &a, int64_t e0, int64_t 
             ss_u = fma((double)m[j], (double)m[j], ss_u);
         }
     }
-    dat_store4(a.mom, e0, lo, hi, m);
-    dat_store4(a.mom, e0 + 4, lo, hi, m + 4);
+    p_st8(a.mom, e0, lo, hi, m, keep);
 }
 
 // ---- Q: levels (Eq. xi), signed sum over the workers and g_hat (Eq. grad_agg), m' and the layer sums
@@ -471,8 +495,7 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
 #pragma unroll
             for (int j = 0; j < 8; ++j)
                 acc[j] = (MODE == P_MODE_IDENTITY) ? acc[j] / a.M_f : (MODE == P_MODE_PER_WORKER) ? acc[j] / a.SM_f : acc[j] * f;
-            dat_store4(a.ghat, e0, lo, hi, acc);
-            dat_store4(a.ghat, e0 + 4, lo, hi, acc + 4);
+            p_st8(a.ghat, e0, lo, hi, acc, dat_policy_evict_last());   // the R part of a later item reads it again
 #pragma unroll
             for (int j = 0; j < 8; ++j) ss_theta = fma((double)acc[j], (double)acc[j], ss_theta);
             continue;
@@ -501,8 +524,7 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
         if (OPT == P_OPT_LAMB) {
             // Algorithm A2: both moments are stored, the direction is formed on the fly for the layer sums
             float v[8];
-            p_load4_cg(a.var, e0, lo, hi, v);
-            p_load4_cg(a.var, e0 + 4, lo, hi, v + 4);
+            p_ld8(a.var, e0, lo, hi, v, dat_policy_evict_last());
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const float ghat = (MODE == P_MODE_IDENTITY) ? acc[j] / a.M_f : (MODE == P_MODE_PER_WORKER) ? acc[j] / a.SM_f : acc[j] * f;
@@ -513,8 +535,7 @@ __device__ __forceinline__ void p_part_quant(const PArgs &a, const PipePart &pt,
                 ss_theta = fma((double)th[j], (double)th[j], ss_theta);
                 ss_u = fma((double)u, (double)u, ss_u);
             }
-            dat_store4(a.var, e0, lo, hi, v);
-            dat_store4(a.var, e0 + 4, lo, hi, v + 4);
+            p_st8(a.var, e0, lo, hi, v, dat_policy_evict_last());
         } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -558,8 +579,7 @@ __device__ __forceinline__ void p_part_requant(const PArgs &a, const PipePart &p
         const int64_t e0 = begin + 8 * (int64_t)(k * DAT_P_THREADS + threadIdx.x);
         if (e0 >= hi) continue;
         float v[8];
-        p_load4_cg(a.ghat, e0, lo, hi, v);
-        p_load4_cg(a.ghat, e0 + 4, lo, hi, v + 4);
+        p_ld8(a.ghat, e0, lo, hi, v, dat_policy_evict_first());
         uint32_t w[8];
         if (RNG16) {
             dat_random_words((uint64_t)e0 >> 3, (uint32_t)a.M, a.keys, w);
@@ -573,8 +593,7 @@ __device__ __forceinline__ void p_part_requant(const PArgs &a, const PipePart &p
             const int lev = (int)dat_level_u1(v[j], t, two_b, u1);
             v[j] = (float)((v[j] < 0.0f) ? -lev : lev) * f;
         }
-        dat_store4(a.ghat, e0, lo, hi, v);          // the receiver's value
-        dat_store4(a.ghat, e0 + 4, lo, hi, v + 4);
+        p_st8(a.ghat, e0, lo, hi, v, dat_policy_evict_first());   // the receiver's value
         p_direction<OPT>(a, e0, lo, hi, v, ss_theta, ss_u);
     }
     __threadfence();
@@ -655,20 +674,16 @@ __device__ __forceinline__ void p_part_update(const PArgs &a, const PipePart &pt
         if (OPT == P_OPT_LAMB) {
             // the direction once more from the stored moments: the same fp32 operations give the same bits
             float th[8], m[8], v[8];
-            p_load4_cg(a.theta, e0, lo, hi, th);
-            p_load4_cg(a.theta, e0 + 4, lo, hi, th + 4);
-            p_load4_cg(a.mom, e0, lo, hi, m);
-            p_load4_cg(a.mom, e0 + 4, lo, hi, m + 4);
-            p_load4_cg(a.var, e0, lo, hi, v);
-            p_load4_cg(a.var, e0 + 4, lo, hi, v + 4);
+            p_ld8(a.theta, e0, lo, hi, th, pol_first);
+            p_ld8(a.mom, e0, lo, hi, m, pol_first);
+            p_ld8(a.var, e0, lo, hi, v, pol_first);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const bool inside = (e0 + j >= lo && e0 + j < hi);
                 const float u = inside ? dat_lamb_direction(a.lamb, m[j], v[j], th[j]) : 0.0f;
                 th[j] = __fmaf_rn(na, u, th[j]);
             }
-            dat_store4(a.theta, e0, lo, hi, th);
-            dat_store4(a.theta, e0 + 4, lo, hi, th + 4);
+            p_st8(a.theta, e0, lo, hi, th, pol_first);
         } else if (e0 >= lo && e0 + 8 <= hi) {
             float4 t0 = dat_ld4_hint(a.theta + e0, pol_first), t1 = dat_ld4_hint(a.theta + e0 + 4, pol_first);
             const float4 m0 = dat_ld4_hint(a.mom + e0, pol_first), m1 = dat_ld4_hint(a.mom + e0 + 4, pol_first);
