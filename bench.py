@@ -524,8 +524,9 @@ def run_sharded(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200,
-                    help="timed steps (about a thousand back-to-back steps and more bring the GPU under its power cap: lower clocks)")
+    ap.add_argument("--steps", type=int, default=100,
+                    help="timed steps (after about 60 ms of back-to-back steps the GPU comes under its power cap and the clocks drop: "
+                         "the measured peak this is compared with is a burst figure too)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="resnet50",
                     choices=["tiny_mlp", "resnet18", "resnet50", "resnet50_m32", "flat1b", "flat_small"])
