@@ -39,16 +39,19 @@
 #define DAT_P_MINB (1024 / DAT_P_THREADS)         // 64 registers per thread
 #endif
 #ifndef DAT_P_LAG                                 // items between the last N tile of a layer and its first Q tile
-#define DAT_P_LAG 384
+#define DAT_P_LAG 256
 #endif
 #ifndef DAT_P_LAG_U                               // items between the last Q tile of a layer and its first U tile
-#define DAT_P_LAG_U DAT_P_LAG
+#define DAT_P_LAG_U 512
 #endif
 #ifndef DAT_P_KEEP_T                              // layers of at most this many tiles: the first reads stay in L2 for the second
 #define DAT_P_KEEP_T 72
 #endif
+#ifndef DAT_P_KEEP_TAIL                           // of a larger layer, the first reads of this many last tiles stay in L2 too
+#define DAT_P_KEEP_TAIL 64
+#endif
 #ifndef DAT_P_REVERSE_FROM                        // layers of at least this many tiles: Q walks back from the last tile
-#define DAT_P_REVERSE_FROM 320
+#define DAT_P_REVERSE_FROM (DAT_P_KEEP_T + 1)
 #endif
 #define DAT_P_WAIT_CYCLES (4000000000ll)          // about two seconds
 
@@ -207,9 +210,10 @@ __device__ __forceinline__ void p_norm_sums(const PArgs &a, const PipePart &pt, 
 #ifndef DAT_P_N_POLICY
 #define DAT_P_N_POLICY dat_policy_evict_first
 #endif
-        // A small layer's lines are still in L2 when the Q part of a later item reads them again; a large layer's
-        // are gone by then anyway: better they leave first than push out theta and m', which the U part can still find.
-        const uint64_t pol = (pt.T <= DAT_P_KEEP_T) ? dat_policy_evict_normal() : DAT_P_N_POLICY();
+        // A small layer's lines are still in L2 when the Q part of a later item reads them again, and so are those of
+        // a larger layer's last tiles, which the Q stream (walking back from the last tile) reads first; the rest of a
+        // large layer is gone by then anyway: better it leaves first than push out those lines, theta and m'.
+        const uint64_t pol = (pt.T <= DAT_P_KEEP_T || pt.tile >= pt.T - DAT_P_KEEP_TAIL) ? dat_policy_evict_normal() : DAT_P_N_POLICY();
 #pragma unroll 1
         for (int ub = u0; ub < u1; ub += UPB) {
             float4 v[8];
@@ -849,7 +853,7 @@ int dat_pipe_build(dat_plan_t *plan)
                 const int64_t T = tb[l + 1] - tb[l];
                 slot = std::max(slot, done_n[l] + DAT_P_LAG + 1);
                 // a layer that L2 cannot hold next to what streams in meanwhile is walked back from its last
-                // tile (what N read last is read first); the others in N's order, every tile at the same distance
+                // tile (what N read last, and marked to stay, is read first); the others in N's order
                 const bool reverse = T >= DAT_P_REVERSE_FROM;
                 for (int64_t t = 0; t < T; ++t) { at(slot).q = part(l, reverse ? T - 1 - t : t); done_q[l] = slot++; }
             }
